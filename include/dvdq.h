@@ -1,0 +1,179 @@
+/*
+ * dvdq.h -- C ABI of the B200 (sm_100a) quantized-linear library for DVD-Quant.
+ *
+ * The library runs the per-layer hot path of DVD-Quant's quantized inference:
+ *
+ *   (1) online activation transform (Sec. 3.2 "Auto-scaling Rotated Quantization",
+ *       Eq. 10): rotate each token by a block Hadamard matrix, take one absmax
+ *       scale per token, round to b-bit signed codes and pack them;
+ *   (2) an integer GEMM of those codes against 4-bit weights stored in the
+ *       Quant/DeQuant format of Sec. 3.1 (unsigned code, integer zero point and
+ *       step size per output channel) with a dequantizing bf16 epilogue,
+ *       Y = X^ Lambda W^^T (Eq. 10).
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller unless a
+ *     parameter says "host".  The library never allocates device memory.
+ *   - Calls are asynchronous on the CUDA stream passed as `cuda_stream`
+ *     (a cudaStream_t cast to void*; NULL is the default stream).
+ *   - The return value covers host-side argument validation and launch errors.
+ *     A kernel that gives up on a device-side wait records that in a status word
+ *     read by dvdq_last_device_status().
+ *   - Packed code buffers are opaque; use the pack/unpack entry points to read or
+ *     write them.  Row-major everywhere; "ld" arguments count ELEMENTS.
+ *   - Only sm_100 devices are accepted (DVDQ_ERR_ARCH otherwise).  There is no
+ *     fallback path of any kind.
+ */
+#ifndef DVDQ_H_
+#define DVDQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    DVDQ_OK = 0,
+    DVDQ_ERR_NULL = 1,           /* a required pointer is NULL */
+    DVDQ_ERR_SHAPE = 2,          /* M, N, K or a leading dimension is not supported */
+    DVDQ_ERR_BITS = 3,           /* activation bit width is not 4 or 6 */
+    DVDQ_ERR_ROT_BLOCK = 4,      /* rotation block invalid, or activations and weights disagree on it */
+    DVDQ_ERR_ALIGN = 5,          /* a pointer or pitch misses its alignment requirement */
+    DVDQ_ERR_WORKSPACE = 6,      /* workspace too small */
+    DVDQ_ERR_BLOB = 7,           /* weight handle / blob header is not one this library wrote */
+    DVDQ_ERR_ARCH = 8,           /* current device is not sm_100 */
+    DVDQ_ERR_CUDA = 9,           /* a CUDA runtime or driver call failed */
+    DVDQ_ERR_DEVICE_TIMEOUT = 10,/* a kernel gave up on a bounded device-side wait */
+    DVDQ_ERR_UNSUPPORTED = 11    /* a reserved option (scale_group != 0, bits == 8) */
+} dvdq_status;
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* dvdq_status_string(dvdq_status s);
+
+/*
+ * The activation quantizer of Eq. 10, X^ = Q(X H Lambda^-1):
+ *   bits        b, the code width: 4 (codes in [-8,7]) or 6 (codes in [-32,31]).
+ *               The quantizer is symmetric with qmax = 2^(b-1) - 1.
+ *   rot_block   B, the order of the Hadamard blocks of the rotation
+ *               R = I_{K/B} (x) H_B / sqrt(B); a power of two in [64, 1024] that
+ *               divides K.  0 means no rotation (R = I).
+ *   scale_group granularity of Lambda: 0 = one absmax scale per token over all K
+ *               channels (the only built value; others give DVDQ_ERR_UNSUPPORTED).
+ */
+typedef struct {
+    int32_t bits;
+    int32_t rot_block;
+    int32_t scale_group;
+} dvdq_act_quant;
+
+/*
+ * Host-side handle of a packed weight matrix.  Filled by dvdq_pack_weights();
+ * `blob` is the device buffer the caller passed there.  Plain data: it may be
+ * copied, and it stays valid as long as the device buffer does.
+ */
+typedef struct {
+    uint32_t magic;      /* 'DVDQ' */
+    uint32_t version;
+    int64_t  N;          /* output channels (rows of W) */
+    int64_t  K;          /* input channels */
+    int32_t  rot_block;  /* B the weights were rotated with (recorded, not applied) */
+    int32_t  k_layout;   /* storage order of the K axis shared with the activation codes */
+    const void* blob;    /* device */
+    uint64_t blob_bytes;
+} dvdq_weights;
+
+/* ---- size queries (host only, no CUDA calls) ------------------------------------ */
+
+/* Bytes of the packed activation codes of an [M, K] tensor: M * K * bits / 8. 0 on bad input. */
+size_t dvdq_act_codes_bytes(int64_t M, int64_t K, int32_t bits);
+/* Bytes of the device blob that dvdq_pack_weights() writes for an [N, K] matrix. 0 on bad input. */
+size_t dvdq_weight_blob_bytes(int64_t N, int64_t K);
+/* Bytes of the workspace dvdq_qlinear() needs (codes, scales and code sums of X). 0 on bad input. */
+size_t dvdq_qlinear_workspace_bytes(int64_t M, int64_t K, const dvdq_act_quant* q);
+
+/* ---- (1) online activation transform: Sec. 3.2, Eq. 10 ---------------------------
+ *
+ * For every token i (row of X):  x~_i = x_i R  (fast Walsh-Hadamard butterflies in fp32),
+ * a_i = max_k |x~_ik|, s_i = a_i / qmax, c_ik = round_half_even(x~_ik / s_i).
+ *
+ *   X_bf16         [M, K] bf16, row pitch ldx elements; 16-byte aligned, ldx % 8 == 0
+ *   codes_out      dvdq_act_codes_bytes(M, K, bits) bytes, 16-byte aligned (opaque layout)
+ *   scales_out     [M] fp32, s_i  (0 for an all-zero token, whose codes are all 0)
+ *   code_sums_out  [M] int32, sum_k c_ik (used by the GEMM for the weight zero point)
+ * K % 64 == 0, K <= 32768.  M == 0 is a no-op.
+ */
+dvdq_status dvdq_rotate_quantize(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
+                                 const dvdq_act_quant* q, void* codes_out, float* scales_out,
+                                 int32_t* code_sums_out, void* cuda_stream);
+
+/* ---- (0) offline weight packing: Sec. 3.1 Quant/DeQuant format, Eq. 10 W^ ----------
+ *
+ * Takes weights that are ALREADY rotated (W~ = W R, same B as the activations) and
+ * quantized to the format W^ = Delta (W_q - z):
+ *   Wq     [N, K] uint8, values 0..15 (upper bits ignored)
+ *   delta  [N] fp32 step sizes
+ *   zero   [N] int32 zero points, 0..15
+ *   blob_out  dvdq_weight_blob_bytes(N, K) bytes, 256-byte aligned
+ *   out    host handle describing the blob (written synchronously)
+ * N % 8 == 0, K % 64 == 0.  rot_block is recorded so that dvdq_qgemm can refuse
+ * activations rotated with a different block.
+ */
+dvdq_status dvdq_pack_weights(const uint8_t* Wq, const float* delta, const int32_t* zero,
+                              int64_t N, int64_t K, int32_t rot_block,
+                              void* blob_out, dvdq_weights* out /* host */, void* cuda_stream);
+
+/* ---- (2) low-bit GEMM + dequantizing epilogue: Eq. 10, Y = X^ Lambda W^^T ----------
+ *
+ *   acc_in = sum_k c_ik (u_nk - z_n)      exact int32 (tensor cores, int8 operands)
+ *   y_in   = bf16( acc_in * s_i * Delta_n + bias_n )   fp32 arithmetic, one rounding
+ *   act == 1 applies tanh-GELU to the rounded value and rounds to bf16 again.
+ *
+ *   codes, scales, code_sums   outputs of dvdq_rotate_quantize for the same M, K, q
+ *   w            host handle from dvdq_pack_weights
+ *   bias_bf16    [N] bf16 or NULL
+ *   Y_bf16       [M, N] bf16, row pitch ldy elements; 16-byte aligned, ldy % 8 == 0
+ */
+dvdq_status dvdq_qgemm(const void* codes, const float* scales, const int32_t* code_sums,
+                       int64_t M, const dvdq_act_quant* q, const dvdq_weights* w /* host */,
+                       const void* bias_bf16, int32_t act, void* Y_bf16, int64_t ldy,
+                       void* cuda_stream);
+
+/* ---- (1)+(2): one quantized linear layer ------------------------------------------
+ * workspace: dvdq_qlinear_workspace_bytes(M, K, q) bytes, 256-byte aligned. */
+dvdq_status dvdq_qlinear(const void* X_bf16, int64_t M, int64_t ldx, const dvdq_act_quant* q,
+                         const dvdq_weights* w /* host */, const void* bias_bf16, int32_t act,
+                         void* Y_bf16, int64_t ldy, void* workspace, size_t workspace_bytes,
+                         void* cuda_stream);
+
+/* ---- test / debug entry points (so that no caller depends on the packed layouts) ---- */
+
+/* The raw accumulators of dvdq_qgemm: acc_out [M, N] int32, row pitch ldacc elements. */
+dvdq_status dvdq_qgemm_int32(const void* codes, const int32_t* code_sums, int64_t M,
+                             const dvdq_act_quant* q, const dvdq_weights* w /* host */,
+                             int32_t* acc_out, int64_t ldacc, void* cuda_stream);
+
+/* Natural-order codes [M, K] int8 -> packed buffer (+ code sums); the inverse of the next one. */
+dvdq_status dvdq_pack_act_codes(const int8_t* codes_nat, int64_t M, int64_t K,
+                                const dvdq_act_quant* q, void* codes_out, int32_t* code_sums_out,
+                                void* cuda_stream);
+/* Packed buffer -> natural-order codes [M, K] int8. */
+dvdq_status dvdq_unpack_act_codes(const void* codes, int64_t M, int64_t K,
+                                  const dvdq_act_quant* q, int8_t* codes_nat, void* cuda_stream);
+/* Blob -> Wq [N, K] uint8 (0..15), delta [N], zero [N]. */
+dvdq_status dvdq_unpack_weights(const dvdq_weights* w /* host */, uint8_t* Wq, float* delta,
+                                int32_t* zero, void* cuda_stream);
+
+/* Reads (and clears) the device-side status word of the current device; synchronizes
+ * the device.  DVDQ_OK, or DVDQ_ERR_DEVICE_TIMEOUT with `detail` (host, may be NULL)
+ * set to a code identifying the wait that gave up. */
+dvdq_status dvdq_last_device_status(uint32_t* detail /* host */);
+
+/* Library version, for the Python binding's sanity check. */
+int32_t dvdq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DVDQ_H_ */
