@@ -102,7 +102,7 @@ size_t dvdq_qlinear_workspace_bytes(int64_t M, int64_t K, const dvdq_act_quant* 
  *   codes_out      dvdq_act_codes_bytes(M, K, bits) bytes, 16-byte aligned (opaque layout)
  *   scales_out     [M] fp32, s_i  (0 for an all-zero token, whose codes are all 0)
  *   code_sums_out  [M] int32, sum_k c_ik (used by the GEMM for the weight zero point)
- * K % 64 == 0, K <= 32768.  M == 0 is a no-op.
+ * K % 64 == 0, K <= 16384.  M == 0 is a no-op.
  */
 dvdq_status dvdq_rotate_quantize(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
                                  const dvdq_act_quant* q, void* codes_out, float* scales_out,

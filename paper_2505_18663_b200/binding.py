@@ -1,0 +1,228 @@
+"""Thin ctypes binding of the C ABI declared in ``include/dvdq.h``.
+
+Argument marshalling only: every function takes torch CUDA tensors (device memory) and a
+stream, checks dtypes, passes raw pointers and raises :class:`DvdqError` on a non-zero
+status.  No step of the path runs in Python or on the CPU, and there is no fallback: if the
+CUDA library is missing, importing the functions fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+# status codes of include/dvdq.h
+OK, ERR_NULL, ERR_SHAPE, ERR_BITS, ERR_ROT_BLOCK, ERR_ALIGN, ERR_WORKSPACE, ERR_BLOB, ERR_ARCH, \
+    ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_UNSUPPORTED = range(12)
+
+EXPORTS = [
+    "dvdq_status_string", "dvdq_version", "dvdq_act_codes_bytes", "dvdq_weight_blob_bytes",
+    "dvdq_qlinear_workspace_bytes", "dvdq_rotate_quantize", "dvdq_pack_weights", "dvdq_qgemm",
+    "dvdq_qlinear", "dvdq_qgemm_int32", "dvdq_pack_act_codes", "dvdq_unpack_act_codes",
+    "dvdq_unpack_weights", "dvdq_last_device_status",
+]
+
+
+class DvdqError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({status_string(status)})")
+
+
+class ActQuant(C.Structure):
+    """dvdq_act_quant: the activation quantizer of Eq. 10 (bits, rotation block, scale granularity)."""
+    _fields_ = [("bits", C.c_int32), ("rot_block", C.c_int32), ("scale_group", C.c_int32)]
+
+
+class Weights(C.Structure):
+    """dvdq_weights: host handle of a packed weight blob."""
+    _fields_ = [("magic", C.c_uint32), ("version", C.c_uint32), ("N", C.c_int64), ("K", C.c_int64),
+                ("rot_block", C.c_int32), ("k_layout", C.c_int32), ("blob", C.c_void_p),
+                ("blob_bytes", C.c_uint64)]
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB_PATH
+
+
+def load():
+    """dlopen the in-tree library (building it first if the sources are newer)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB_PATH
+    if _build.is_stale():
+        try:
+            path = _build.build_library()
+        except Exception as e:  # no nvcc on this machine and no prebuilt library
+            if not os.path.exists(path):
+                raise RuntimeError(f"CUDA library {path} is missing and cannot be built: {e}") from e
+    lib = C.CDLL(path)
+    i32, i64, p, sz = C.c_int32, C.c_int64, C.c_void_p, C.c_size_t
+    aq, wp = C.POINTER(ActQuant), C.POINTER(Weights)
+    sig = {
+        "dvdq_status_string": (C.c_char_p, [C.c_int]),
+        "dvdq_version": (i32, []),
+        "dvdq_act_codes_bytes": (sz, [i64, i64, i32]),
+        "dvdq_weight_blob_bytes": (sz, [i64, i64]),
+        "dvdq_qlinear_workspace_bytes": (sz, [i64, i64, aq]),
+        "dvdq_rotate_quantize": (C.c_int, [p, i64, i64, i64, aq, p, p, p, p]),
+        "dvdq_pack_weights": (C.c_int, [p, p, p, i64, i64, i32, p, wp, p]),
+        "dvdq_qgemm": (C.c_int, [p, p, p, i64, aq, wp, p, i32, p, i64, p]),
+        "dvdq_qlinear": (C.c_int, [p, i64, i64, aq, wp, p, i32, p, i64, p, sz, p]),
+        "dvdq_qgemm_int32": (C.c_int, [p, p, i64, aq, wp, p, i64, p]),
+        "dvdq_pack_act_codes": (C.c_int, [p, i64, i64, aq, p, p, p]),
+        "dvdq_unpack_act_codes": (C.c_int, [p, i64, i64, aq, p, p]),
+        "dvdq_unpack_weights": (C.c_int, [wp, p, p, p, p]),
+        "dvdq_last_device_status": (C.c_int, [C.POINTER(C.c_uint32)]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load().dvdq_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise DvdqError(status, where)
+
+
+def _ptr(t: Optional[torch.Tensor], dtype=None, name="tensor"):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _row_major(t: torch.Tensor, name: str) -> int:
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise TypeError(f"{name} must be 2-D with unit inner stride")
+    return t.stride(0)
+
+
+# ------------------------------------------------------------------ size queries
+
+def dvdq_version() -> int:
+    return int(load().dvdq_version())
+
+
+def dvdq_act_codes_bytes(M: int, K: int, bits: int) -> int:
+    return int(load().dvdq_act_codes_bytes(M, K, bits))
+
+
+def dvdq_weight_blob_bytes(N: int, K: int) -> int:
+    return int(load().dvdq_weight_blob_bytes(N, K))
+
+
+def dvdq_qlinear_workspace_bytes(M: int, K: int, q: ActQuant) -> int:
+    return int(load().dvdq_qlinear_workspace_bytes(M, K, C.byref(q)))
+
+
+# ------------------------------------------------------------------ the path
+
+def dvdq_rotate_quantize(X: torch.Tensor, q: ActQuant, codes: torch.Tensor, scales: torch.Tensor,
+                         code_sums: torch.Tensor, stream=None) -> None:
+    ldx = _row_major(X, "X")
+    M, K = X.shape
+    _check(load().dvdq_rotate_quantize(_ptr(X, torch.bfloat16, "X"), M, K, ldx, C.byref(q),
+                                       _ptr(codes, torch.uint8, "codes"), _ptr(scales, torch.float32, "scales"),
+                                       _ptr(code_sums, torch.int32, "code_sums"), _stream(stream)),
+           "dvdq_rotate_quantize")
+
+
+def dvdq_pack_weights(Wq: torch.Tensor, delta: torch.Tensor, zero: torch.Tensor, rot_block: int,
+                      blob: torch.Tensor, stream=None) -> Weights:
+    N, K = Wq.shape
+    if not Wq.is_contiguous():
+        raise TypeError("Wq must be contiguous")
+    w = Weights()
+    _check(load().dvdq_pack_weights(_ptr(Wq, torch.uint8, "Wq"), _ptr(delta, torch.float32, "delta"),
+                                    _ptr(zero, torch.int32, "zero"), N, K, rot_block,
+                                    _ptr(blob, torch.uint8, "blob"), C.byref(w), _stream(stream)),
+           "dvdq_pack_weights")
+    return w
+
+
+def dvdq_qgemm(codes: torch.Tensor, scales: torch.Tensor, code_sums: torch.Tensor, M: int, q: ActQuant,
+               w: Weights, bias: Optional[torch.Tensor], act: int, Y: torch.Tensor, stream=None) -> None:
+    ldy = _row_major(Y, "Y")
+    _check(load().dvdq_qgemm(_ptr(codes, torch.uint8, "codes"), _ptr(scales, torch.float32, "scales"),
+                             _ptr(code_sums, torch.int32, "code_sums"), M, C.byref(q), C.byref(w),
+                             _ptr(bias, torch.bfloat16, "bias"), act, _ptr(Y, torch.bfloat16, "Y"), ldy,
+                             _stream(stream)), "dvdq_qgemm")
+
+
+def dvdq_qlinear(X: torch.Tensor, q: ActQuant, w: Weights, bias: Optional[torch.Tensor], act: int,
+                 Y: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    ldx = _row_major(X, "X")
+    ldy = _row_major(Y, "Y")
+    M = X.shape[0]
+    _check(load().dvdq_qlinear(_ptr(X, torch.bfloat16, "X"), M, ldx, C.byref(q), C.byref(w),
+                               _ptr(bias, torch.bfloat16, "bias"), act, _ptr(Y, torch.bfloat16, "Y"), ldy,
+                               _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)),
+           "dvdq_qlinear")
+
+
+# ------------------------------------------------------------------ test / debug entry points
+
+def dvdq_qgemm_int32(codes: torch.Tensor, code_sums: torch.Tensor, M: int, q: ActQuant, w: Weights,
+                     acc: torch.Tensor, stream=None) -> None:
+    ld = _row_major(acc, "acc")
+    _check(load().dvdq_qgemm_int32(_ptr(codes, torch.uint8, "codes"), _ptr(code_sums, torch.int32, "code_sums"),
+                                   M, C.byref(q), C.byref(w), _ptr(acc, torch.int32, "acc"), ld, _stream(stream)),
+           "dvdq_qgemm_int32")
+
+
+def dvdq_pack_act_codes(codes_nat: torch.Tensor, q: ActQuant, codes: torch.Tensor, code_sums: torch.Tensor,
+                        stream=None) -> None:
+    M, K = codes_nat.shape
+    if not codes_nat.is_contiguous():
+        raise TypeError("codes_nat must be contiguous")
+    _check(load().dvdq_pack_act_codes(_ptr(codes_nat, torch.int8, "codes_nat"), M, K, C.byref(q),
+                                      _ptr(codes, torch.uint8, "codes"), _ptr(code_sums, torch.int32, "code_sums"),
+                                      _stream(stream)), "dvdq_pack_act_codes")
+
+
+def dvdq_unpack_act_codes(codes: torch.Tensor, M: int, K: int, q: ActQuant, codes_nat: torch.Tensor,
+                          stream=None) -> None:
+    if not codes_nat.is_contiguous() or tuple(codes_nat.shape) != (M, K):
+        raise TypeError("codes_nat must be contiguous [M, K]")
+    _check(load().dvdq_unpack_act_codes(_ptr(codes, torch.uint8, "codes"), M, K, C.byref(q),
+                                        _ptr(codes_nat, torch.int8, "codes_nat"), _stream(stream)),
+           "dvdq_unpack_act_codes")
+
+
+def dvdq_unpack_weights(w: Weights, Wq: torch.Tensor, delta: torch.Tensor, zero: torch.Tensor, stream=None) -> None:
+    if not Wq.is_contiguous():
+        raise TypeError("Wq must be contiguous")
+    _check(load().dvdq_unpack_weights(C.byref(w), _ptr(Wq, torch.uint8, "Wq"), _ptr(delta, torch.float32, "delta"),
+                                      _ptr(zero, torch.int32, "zero"), _stream(stream)), "dvdq_unpack_weights")
+
+
+def dvdq_last_device_status():
+    """(status, detail) of the device-side status word; synchronizes the device and clears it."""
+    d = C.c_uint32(0)
+    s = load().dvdq_last_device_status(C.byref(d))
+    return int(s), int(d.value)

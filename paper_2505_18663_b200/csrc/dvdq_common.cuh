@@ -1,0 +1,205 @@
+// Shared declarations of the CUDA sources: packed-format constants, the device status
+// word, and thin wrappers around the sm_100a PTX the kernels use (mbarrier, TMA,
+// tcgen05).  Nothing here is shared with the CPU oracle.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/dvdq.h"
+
+namespace dvdq {
+
+// ------------------------------------------------------------------ formats
+
+constexpr uint32_t kBlobMagic = 0x51445644u;  // "DVDQ" little endian
+constexpr uint32_t kBlobVersion = 1u;
+constexpr int64_t kBlobHeaderBytes = 256;     // header padded so that the codes stay 256-byte aligned
+constexpr int32_t kLibVersion = 1;
+
+// Storage order of the K axis, shared by activation codes and weight codes.  The integer
+// GEMM is a dot product over k, so any permutation applied to both operands gives the same
+// accumulators.
+constexpr int32_t kKLayoutNatural = 0;        // position p holds logical channel p
+
+__host__ __device__ inline int64_t align_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+
+// Device copy of the blob header (the host handle dvdq_weights mirrors it).
+struct BlobHeader {
+    uint32_t magic, version;
+    int64_t N, K;
+    int32_t rot_block, k_layout;
+    int64_t codes_offset, delta_offset, zc_offset;
+};
+
+struct BlobLayout {
+    int64_t codes_offset, delta_offset, zc_offset, total;
+};
+
+__host__ __device__ inline BlobLayout blob_layout(int64_t N, int64_t K) {
+    BlobLayout L;
+    L.codes_offset = kBlobHeaderBytes;
+    L.delta_offset = L.codes_offset + align_up(N * (K / 2), 256);
+    L.zc_offset = L.delta_offset + align_up(N * 4, 256);
+    L.total = L.zc_offset + align_up(N * 4, 256);
+    return L;
+}
+
+// Activation code rows: A4 = K/2 bytes (two's-complement nibbles, position 2t in the low
+// nibble of byte t).  A6 = a low plane in exactly the A4 format holding the low 4 bits of
+// each code, followed by a high plane of K/4 bytes with bits 5:4.  In the high plane one
+// 32-bit word covers 16 consecutive positions p = 16m + 8a + i (a in {0,1}, i in 0..7):
+// the 2-bit field sits at bit 2*(4*(i>>1) + 2*a + (i&1)).  That order makes the GEMM's
+// widening of 16 codes into four int8 words a shift and a mask per word.
+__host__ __device__ inline int64_t act_row_bytes(int64_t K, int bits) { return K * bits / 8; }
+__host__ __device__ inline int hi_field_shift(int a, int i) { return 2 * (4 * (i >> 1) + 2 * a + (i & 1)); }
+
+// ------------------------------------------------------------------ device status word
+
+// [0] = status (0 ok, else dvdq_status), [1] = detail of the first failure.  The library is a
+// single translation unit, so this is the one copy.
+__device__ uint32_t g_device_status[2] = {0u, 0u};
+
+enum WaitId : uint32_t {
+    kWaitPackedEmpty = 1, kWaitPackedFull = 2, kWaitWideEmpty = 3, kWaitWideFull = 4,
+    kWaitAccEmpty = 5, kWaitAccFull = 6, kWaitDrain = 7
+};
+
+__device__ __forceinline__ void report_timeout(uint32_t detail) {
+    if (atomicCAS(&g_device_status[0], 0u, (uint32_t)DVDQ_ERR_DEVICE_TIMEOUT) == 0u) g_device_status[1] = detail;
+}
+
+// ------------------------------------------------------------------ PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Every wait in the kernels is bounded: it gives up when another role has already given up
+// (abort flag in shared memory) or after kWaitLimitNs, records which wait it was, raises the
+// abort flag and returns false.  The caller then leaves its loop and walks to the common exit.
+constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t wait_id) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 0xFFu) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1u;
+                report_timeout(wait_id);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
+}
+// 2-D tiled TMA load global -> shared, completion counted in bytes on an mbarrier.
+// x is the innermost coordinate; x * element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* m, uint32_t bar, int32_t x, int32_t y) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+
+// ---- tensor memory and tcgen05
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// Arrives once on the mbarrier when every tcgen05.mma issued so far by this thread has finished.
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, int8 operands, int32 accumulators, issued by ONE thread.
+__device__ __forceinline__ void tc_mma_i8_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread t of the warp receives lane (base_lane + t).
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major int8 tile whose rows are 128 bytes wide and
+// stored with the 128-byte swizzle: 8-row groups are 1024 bytes apart (stride byte offset),
+// the leading byte offset is unused for this layout (set to 16 bytes), descriptor version 1.
+__device__ __forceinline__ uint64_t umma_desc_sw128_kmajor(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)1u << 16;
+    d |= (uint64_t)(1024u >> 4) << 32;
+    d |= (uint64_t)1u << 46;
+    d |= (uint64_t)2u << 61;
+    return d;
+}
+// Instruction descriptor for kind::i8: signed int8 A and B, both K-major, int32 accumulator.
+__host__ __device__ constexpr uint32_t umma_idesc_s8s8s32(int m, int n) {
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// ------------------------------------------------------------------ host helpers (api.cu)
+
+dvdq_status check_device_arch();
+dvdq_status validate_act_quant(const dvdq_act_quant* q, int64_t K);
+dvdq_status validate_weights(const dvdq_weights* w);
+dvdq_status cuda_status(cudaError_t e);
+
+}  // namespace dvdq

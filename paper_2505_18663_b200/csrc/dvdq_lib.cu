@@ -1,0 +1,260 @@
+// C ABI of the library (see include/dvdq.h): argument validation, size queries and the
+// launches of the kernels in rotate_quantize.cuh, pack.cuh and qgemm.cuh.  One translation
+// unit, so that the device status word is a single symbol.
+#include "dvdq_common.cuh"
+
+#include "pack.cuh"
+#include "qgemm.cuh"
+#include "rotate_quantize.cuh"
+
+namespace dvdq {
+
+dvdq_status cuda_status(cudaError_t e) { return e == cudaSuccess ? DVDQ_OK : DVDQ_ERR_CUDA; }
+
+dvdq_status check_device_arch() {
+    static int cached_dev = -1;
+    static dvdq_status cached = DVDQ_ERR_ARCH;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DVDQ_ERR_CUDA;
+    if (dev == cached_dev) return cached;
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return DVDQ_ERR_CUDA;
+    cached_dev = dev;
+    cached = (major == 10) ? DVDQ_OK : DVDQ_ERR_ARCH;
+    return cached;
+}
+
+static bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
+static bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+// Shape rules shared by every entry point: K a multiple of 64 (16-byte TMA pitches for both
+// code widths and whole 16-code groups of the 6-bit high plane), K <= 16384 (one CTA holds a
+// token), rot_block 0 or a power of two in [64, 1024] dividing K.
+static dvdq_status validate_k(int64_t K) {
+    if (K <= 0 || K % 64 != 0 || K > 16384) return DVDQ_ERR_SHAPE;
+    return DVDQ_OK;
+}
+
+dvdq_status validate_act_quant(const dvdq_act_quant* q, int64_t K) {
+    if (!q) return DVDQ_ERR_NULL;
+    if (q->bits == 8) return DVDQ_ERR_UNSUPPORTED;
+    if (q->bits != 4 && q->bits != 6) return DVDQ_ERR_BITS;
+    if (q->scale_group != 0) return DVDQ_ERR_UNSUPPORTED;
+    if (q->rot_block != 0) {
+        if (!is_pow2(q->rot_block) || q->rot_block < 64 || q->rot_block > 1024) return DVDQ_ERR_ROT_BLOCK;
+        if (K % q->rot_block != 0) return DVDQ_ERR_ROT_BLOCK;
+    }
+    return DVDQ_OK;
+}
+
+dvdq_status validate_weights(const dvdq_weights* w) {
+    if (!w) return DVDQ_ERR_NULL;
+    if (w->magic != kBlobMagic || w->version != kBlobVersion || !w->blob) return DVDQ_ERR_BLOB;
+    if (w->N <= 0 || w->N % 8 != 0 || validate_k(w->K) != DVDQ_OK) return DVDQ_ERR_BLOB;
+    if (w->blob_bytes != (uint64_t)blob_layout(w->N, w->K).total) return DVDQ_ERR_BLOB;
+    if (w->k_layout != kKLayoutNatural) return DVDQ_ERR_BLOB;
+    if (!aligned(w->blob, 256)) return DVDQ_ERR_ALIGN;
+    return DVDQ_OK;
+}
+
+struct WorkspacePlan {
+    int64_t codes_off, scales_off, sums_off, total;
+};
+static WorkspacePlan workspace_plan(int64_t M, int64_t K, int bits) {
+    WorkspacePlan p;
+    p.codes_off = 0;
+    p.scales_off = align_up(M * act_row_bytes(K, bits), 256);
+    p.sums_off = p.scales_off + align_up(M * 4, 256);
+    p.total = p.sums_off + align_up(M * 4, 256);
+    return p;
+}
+
+}  // namespace dvdq
+
+using namespace dvdq;
+
+extern "C" {
+
+const char* dvdq_status_string(dvdq_status s) {
+    switch (s) {
+        case DVDQ_OK: return "ok";
+        case DVDQ_ERR_NULL: return "required pointer is NULL";
+        case DVDQ_ERR_SHAPE: return "unsupported shape or leading dimension";
+        case DVDQ_ERR_BITS: return "activation bit width must be 4 or 6";
+        case DVDQ_ERR_ROT_BLOCK: return "rotation block invalid or inconsistent between activations and weights";
+        case DVDQ_ERR_ALIGN: return "pointer or pitch not aligned as required";
+        case DVDQ_ERR_WORKSPACE: return "workspace too small";
+        case DVDQ_ERR_BLOB: return "weight handle was not produced by this library version";
+        case DVDQ_ERR_ARCH: return "device is not sm_100";
+        case DVDQ_ERR_CUDA: return "CUDA call failed";
+        case DVDQ_ERR_DEVICE_TIMEOUT: return "a kernel gave up on a bounded device-side wait";
+        case DVDQ_ERR_UNSUPPORTED: return "reserved option is not built";
+    }
+    return "unknown status";
+}
+
+int32_t dvdq_version(void) { return kLibVersion; }
+
+size_t dvdq_act_codes_bytes(int64_t M, int64_t K, int32_t bits) {
+    if (M < 0 || validate_k(K) != DVDQ_OK || (bits != 4 && bits != 6)) return 0;
+    return (size_t)(M * act_row_bytes(K, bits));
+}
+
+size_t dvdq_weight_blob_bytes(int64_t N, int64_t K) {
+    if (N <= 0 || N % 8 != 0 || validate_k(K) != DVDQ_OK) return 0;
+    return (size_t)blob_layout(N, K).total;
+}
+
+size_t dvdq_qlinear_workspace_bytes(int64_t M, int64_t K, const dvdq_act_quant* q) {
+    if (M < 0 || validate_k(K) != DVDQ_OK || validate_act_quant(q, K) != DVDQ_OK) return 0;
+    return (size_t)workspace_plan(M, K, q->bits).total;
+}
+
+dvdq_status dvdq_rotate_quantize(const void* X, int64_t M, int64_t K, int64_t ldx, const dvdq_act_quant* q,
+                                 void* codes_out, float* scales_out, int32_t* code_sums_out, void* stream) {
+    if (!q) return DVDQ_ERR_NULL;
+    if (M < 0 || validate_k(K) != DVDQ_OK || ldx < K || ldx % 8 != 0) return DVDQ_ERR_SHAPE;
+    dvdq_status s = validate_act_quant(q, K);
+    if (s != DVDQ_OK) return s;
+    if (M == 0) return DVDQ_OK;
+    if (!X || !codes_out || !scales_out || !code_sums_out) return DVDQ_ERR_NULL;
+    if (!aligned(X, 16) || !aligned(codes_out, 16) || !aligned(scales_out, 4) || !aligned(code_sums_out, 4)) return DVDQ_ERR_ALIGN;
+    if ((s = check_device_arch()) != DVDQ_OK) return s;
+    return launch_rotate_quantize(X, M, K, ldx, *q, codes_out, scales_out, code_sums_out, (cudaStream_t)stream);
+}
+
+dvdq_status dvdq_pack_weights(const uint8_t* Wq, const float* delta, const int32_t* zero, int64_t N, int64_t K,
+                              int32_t rot_block, void* blob_out, dvdq_weights* out, void* stream) {
+    if (!Wq || !delta || !zero || !blob_out || !out) return DVDQ_ERR_NULL;
+    if (N <= 0 || N % 8 != 0 || validate_k(K) != DVDQ_OK) return DVDQ_ERR_SHAPE;
+    dvdq_act_quant probe = {4, rot_block, 0};
+    dvdq_status s = validate_act_quant(&probe, K);
+    if (s != DVDQ_OK) return s;
+    if (!aligned(blob_out, 256)) return DVDQ_ERR_ALIGN;
+    if ((s = check_device_arch()) != DVDQ_OK) return s;
+    pack_weights_kernel<<<grid_for(N * (K / 2), 256), 256, 0, (cudaStream_t)stream>>>(
+        Wq, delta, zero, N, K, rot_block, kKLayoutNatural, static_cast<uint8_t*>(blob_out));
+    if ((s = cuda_status(cudaGetLastError())) != DVDQ_OK) return s;
+    out->magic = kBlobMagic;
+    out->version = kBlobVersion;
+    out->N = N;
+    out->K = K;
+    out->rot_block = rot_block;
+    out->k_layout = kKLayoutNatural;
+    out->blob = blob_out;
+    out->blob_bytes = (uint64_t)blob_layout(N, K).total;
+    return DVDQ_OK;
+}
+
+static dvdq_status check_gemm_args(const void* codes, const int32_t* sums, int64_t M, const dvdq_act_quant* q,
+                                   const dvdq_weights* w) {
+    dvdq_status s = validate_weights(w);
+    if (s != DVDQ_OK) return s;
+    if ((s = validate_act_quant(q, w->K)) != DVDQ_OK) return s;
+    if (q->rot_block != w->rot_block) return DVDQ_ERR_ROT_BLOCK;
+    if (M < 0 || M > 0x7FFFFF00ll) return DVDQ_ERR_SHAPE;
+    if (M == 0) return DVDQ_OK;
+    if (!codes || !sums) return DVDQ_ERR_NULL;
+    if (!aligned(codes, 16) || !aligned(sums, 4)) return DVDQ_ERR_ALIGN;
+    return check_device_arch();
+}
+
+dvdq_status dvdq_qgemm(const void* codes, const float* scales, const int32_t* code_sums, int64_t M,
+                       const dvdq_act_quant* q, const dvdq_weights* w, const void* bias, int32_t act,
+                       void* Y, int64_t ldy, void* stream) {
+    dvdq_status s = check_gemm_args(codes, code_sums, M, q, w);
+    if (s != DVDQ_OK) return s;
+    if (act != 0 && act != 1) return DVDQ_ERR_UNSUPPORTED;
+    if (ldy < w->N || ldy % 8 != 0) return DVDQ_ERR_SHAPE;
+    if (M == 0) return DVDQ_OK;
+    if (!scales || !Y) return DVDQ_ERR_NULL;
+    if (!aligned(Y, 16) || !aligned(scales, 4) || (bias && !aligned(bias, 2))) return DVDQ_ERR_ALIGN;
+    return launch_qgemm(codes, scales, code_sums, M, *q, *w, bias, act, Y, ldy, nullptr, 0, (cudaStream_t)stream);
+}
+
+dvdq_status dvdq_qgemm_int32(const void* codes, const int32_t* code_sums, int64_t M, const dvdq_act_quant* q,
+                             const dvdq_weights* w, int32_t* acc_out, int64_t ldacc, void* stream) {
+    dvdq_status s = check_gemm_args(codes, code_sums, M, q, w);
+    if (s != DVDQ_OK) return s;
+    if (ldacc < w->N || ldacc % 4 != 0) return DVDQ_ERR_SHAPE;
+    if (M == 0) return DVDQ_OK;
+    if (!acc_out) return DVDQ_ERR_NULL;
+    if (!aligned(acc_out, 16)) return DVDQ_ERR_ALIGN;
+    return launch_qgemm(codes, nullptr, code_sums, M, *q, *w, nullptr, 0, nullptr, 0, acc_out, ldacc, (cudaStream_t)stream);
+}
+
+dvdq_status dvdq_qlinear(const void* X, int64_t M, int64_t ldx, const dvdq_act_quant* q, const dvdq_weights* w,
+                         const void* bias, int32_t act, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+    dvdq_status s = validate_weights(w);
+    if (s != DVDQ_OK) return s;
+    if ((s = validate_act_quant(q, w->K)) != DVDQ_OK) return s;
+    if (M < 0) return DVDQ_ERR_SHAPE;
+    if (M == 0) return DVDQ_OK;
+    if (!workspace) return DVDQ_ERR_NULL;
+    if (!aligned(workspace, 256)) return DVDQ_ERR_ALIGN;
+    const WorkspacePlan p = workspace_plan(M, w->K, q->bits);
+    if (workspace_bytes < (size_t)p.total) return DVDQ_ERR_WORKSPACE;
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    void* codes = ws + p.codes_off;
+    float* scales = reinterpret_cast<float*>(ws + p.scales_off);
+    int32_t* sums = reinterpret_cast<int32_t*>(ws + p.sums_off);
+    if ((s = dvdq_rotate_quantize(X, M, w->K, ldx, q, codes, scales, sums, stream)) != DVDQ_OK) return s;
+    return dvdq_qgemm(codes, scales, sums, M, q, w, bias, act, Y, ldy, stream);
+}
+
+dvdq_status dvdq_pack_act_codes(const int8_t* codes_nat, int64_t M, int64_t K, const dvdq_act_quant* q,
+                                void* codes_out, int32_t* code_sums_out, void* stream) {
+    if (M < 0 || validate_k(K) != DVDQ_OK) return DVDQ_ERR_SHAPE;
+    dvdq_status s = validate_act_quant(q, K);
+    if (s != DVDQ_OK) return s;
+    if (M == 0) return DVDQ_OK;
+    if (!codes_nat || !codes_out || !code_sums_out) return DVDQ_ERR_NULL;
+    if (!aligned(codes_out, 16)) return DVDQ_ERR_ALIGN;
+    if ((s = check_device_arch()) != DVDQ_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    const unsigned g = grid_for(M * (K / 16), 256);
+    if (q->bits == 4) pack_act_codes_kernel<4><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
+    else pack_act_codes_kernel<6><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
+    code_sums_kernel<<<(unsigned)((M * 32 + 255) / 256), 256, 0, st>>>(codes_nat, M, K, code_sums_out);
+    return cuda_status(cudaGetLastError());
+}
+
+dvdq_status dvdq_unpack_act_codes(const void* codes, int64_t M, int64_t K, const dvdq_act_quant* q,
+                                  int8_t* codes_nat, void* stream) {
+    if (M < 0 || validate_k(K) != DVDQ_OK) return DVDQ_ERR_SHAPE;
+    dvdq_status s = validate_act_quant(q, K);
+    if (s != DVDQ_OK) return s;
+    if (M == 0) return DVDQ_OK;
+    if (!codes || !codes_nat) return DVDQ_ERR_NULL;
+    if (!aligned(codes, 16)) return DVDQ_ERR_ALIGN;
+    if ((s = check_device_arch()) != DVDQ_OK) return s;
+    const unsigned g = grid_for(M * (K / 16), 256);
+    if (q->bits == 4) unpack_act_codes_kernel<4><<<g, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint8_t*>(codes), M, K, codes_nat);
+    else unpack_act_codes_kernel<6><<<g, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint8_t*>(codes), M, K, codes_nat);
+    return cuda_status(cudaGetLastError());
+}
+
+dvdq_status dvdq_unpack_weights(const dvdq_weights* w, uint8_t* Wq, float* delta, int32_t* zero, void* stream) {
+    dvdq_status s = validate_weights(w);
+    if (s != DVDQ_OK) return s;
+    if (!Wq || !delta || !zero) return DVDQ_ERR_NULL;
+    if ((s = check_device_arch()) != DVDQ_OK) return s;
+    unpack_weights_kernel<<<grid_for(w->N * (w->K / 2), 256), 256, 0, (cudaStream_t)stream>>>(
+        static_cast<const uint8_t*>(w->blob), w->N, w->K, Wq, delta, zero);
+    return cuda_status(cudaGetLastError());
+}
+
+dvdq_status dvdq_last_device_status(uint32_t* detail) {
+    uint32_t h[2] = {0u, 0u};
+    if (cudaDeviceSynchronize() != cudaSuccess) return DVDQ_ERR_CUDA;
+    if (cudaMemcpyFromSymbol(h, g_device_status, sizeof h) != cudaSuccess) return DVDQ_ERR_CUDA;
+    if (h[0] != 0u) {
+        const uint32_t zero[2] = {0u, 0u};
+        if (cudaMemcpyToSymbol(g_device_status, zero, sizeof zero) != cudaSuccess) return DVDQ_ERR_CUDA;
+    }
+    if (detail) *detail = h[1];
+    return (dvdq_status)h[0];
+}
+
+}  // extern "C"
