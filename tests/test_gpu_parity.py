@@ -230,8 +230,10 @@ def test_bf16_output_on_oracle_codes_and_scales(M, N, K, Bk, bits, mode, act):
     y = Y.to(torch.float64).cpu().numpy()
     assert np.abs(y - y_or).max() <= Y_MAXNORM_RTOL * np.abs(y_or).max()
     # identical integer inputs: only the fp32-vs-fp64 epilogue differs, i.e. at most one bf16 ulp
-    ulp = np.maximum(np.abs(y_or), 2.0 ** -100) * 2.0 ** -7
-    assert np.all(np.abs(y - y_or) <= ulp)
+    # of the linear output; through GELU (slope <= 1.13) that ulp plus the second rounding.
+    y0_or = bf16_values(orc.epilogue(orc.int_gemm(codes, u, z), s32, d, to_bits(bias), 0))
+    ulp = np.maximum(np.abs(y0_or), 2.0 ** -100) * 2.0 ** -7
+    assert np.all(np.abs(y - y_or) <= (ulp if act == 0 else 3 * ulp))
     assert np.mean(y != y_or) < 0.02
 
 
