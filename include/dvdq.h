@@ -147,6 +147,32 @@ dvdq_status dvdq_qlinear(const void* X_bf16, int64_t M, int64_t ldx, const dvdq_
                          void* Y_bf16, int64_t ldy, void* workspace, size_t workspace_bytes,
                          void* cuda_stream);
 
+/* ---- (1)+(2) for callers that cannot allocate device memory -------------------------
+ *
+ * The paper has no counterpart to this entry point; it exists for integration reasons only.
+ *
+ * Some hosts of this library cannot hand it a workspace: code running inside a region where
+ * cudaMalloc is forbidden or would synchronise the device (a plugin called from another
+ * framework's execution engine, a real-time loop that must not touch the allocator, a
+ * process whose memory pool is owned and sized by someone else).  For them this variant of
+ * dvdq_qlinear keeps the intermediate activation codes, scales and code sums in a fixed
+ * array that is part of the library image itself: DVDQ_STATIC_SCRATCH_BYTES of device
+ * memory, reserved on every GPU that loads the library for as long as the process lives.
+ * The call allocates nothing and frees nothing.  Inputs and outputs are still the caller's.
+ *
+ *   - The problem must fit: dvdq_qlinear_workspace_bytes(M, K, q) <= DVDQ_STATIC_SCRATCH_BYTES,
+ *     otherwise DVDQ_ERR_WORKSPACE is returned and nothing is launched.
+ *   - The first call on each device looks up the array's device address (once per device,
+ *     with that device current).  Make that first call outside any stream capture.
+ *   - Every call on a device uses the SAME array.  Calls that may overlap on the GPU (two
+ *     streams, two host threads) race on it; serialise them.  The array keeps the previous
+ *     call's contents; the call overwrites every byte it later reads, so nothing needs clearing.
+ * All other arguments and rules are those of dvdq_qlinear. */
+#define DVDQ_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+dvdq_status dvdq_qlinear_static(const void* X_bf16, int64_t M, int64_t ldx, const dvdq_act_quant* q,
+                                const dvdq_weights* w /* host */, const void* bias_bf16, int32_t act,
+                                void* Y_bf16, int64_t ldy, void* cuda_stream);
+
 /* ---- test / debug entry points (so that no caller depends on the packed layouts) ---- */
 
 /* The raw accumulators of dvdq_qgemm: acc_out [M, N] int32, row pitch ldacc elements. */

@@ -22,7 +22,7 @@ OK, ERR_NULL, ERR_SHAPE, ERR_BITS, ERR_ROT_BLOCK, ERR_ALIGN, ERR_WORKSPACE, ERR_
 EXPORTS = [
     "dvdq_status_string", "dvdq_version", "dvdq_act_codes_bytes", "dvdq_weight_blob_bytes",
     "dvdq_qlinear_workspace_bytes", "dvdq_rotate_quantize", "dvdq_pack_weights", "dvdq_qgemm",
-    "dvdq_qlinear", "dvdq_qgemm_int32", "dvdq_pack_act_codes", "dvdq_unpack_act_codes",
+    "dvdq_qlinear", "dvdq_qlinear_static", "dvdq_qgemm_int32", "dvdq_pack_act_codes", "dvdq_unpack_act_codes",
     "dvdq_unpack_weights", "dvdq_last_device_status",
 ]
 
@@ -77,6 +77,7 @@ def load():
         "dvdq_pack_weights": (C.c_int, [p, p, p, i64, i64, i32, p, wp, p]),
         "dvdq_qgemm": (C.c_int, [p, p, p, i64, aq, wp, p, i32, p, i64, p]),
         "dvdq_qlinear": (C.c_int, [p, i64, i64, aq, wp, p, i32, p, i64, p, sz, p]),
+        "dvdq_qlinear_static": (C.c_int, [p, i64, i64, aq, wp, p, i32, p, i64, p]),
         "dvdq_qgemm_int32": (C.c_int, [p, p, i64, aq, wp, p, i64, p]),
         "dvdq_pack_act_codes": (C.c_int, [p, i64, i64, aq, p, p, p]),
         "dvdq_unpack_act_codes": (C.c_int, [p, i64, i64, aq, p, p]),
@@ -183,6 +184,21 @@ def dvdq_qlinear(X: torch.Tensor, q: ActQuant, w: Weights, bias: Optional[torch.
                                _ptr(bias, torch.bfloat16, "bias"), act, _ptr(Y, torch.bfloat16, "Y"), ldy,
                                _ptr(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)),
            "dvdq_qlinear")
+
+
+STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+
+def dvdq_qlinear_static(X: torch.Tensor, q: ActQuant, w: Weights, bias: Optional[torch.Tensor], act: int,
+                        Y: torch.Tensor, stream=None) -> None:
+    """dvdq_qlinear for callers that cannot allocate: the intermediate codes live in a fixed
+    STATIC_SCRATCH_BYTES array inside the library (shared by all calls on a device, so calls
+    must not overlap; larger problems are refused with ERR_WORKSPACE)."""
+    ldx = _row_major(X, "X")
+    ldy = _row_major(Y, "Y")
+    _check(load().dvdq_qlinear_static(_ptr(X, torch.bfloat16, "X"), X.shape[0], ldx, C.byref(q), C.byref(w),
+                                      _ptr(bias, torch.bfloat16, "bias"), act, _ptr(Y, torch.bfloat16, "Y"), ldy,
+                                      _stream(stream)), "dvdq_qlinear_static")
 
 
 # ------------------------------------------------------------------ test / debug entry points

@@ -203,6 +203,36 @@ dvdq_status dvdq_qlinear(const void* X, int64_t M, int64_t ldx, const dvdq_act_q
     return dvdq_qgemm(codes, scales, sums, M, q, w, bias, act, Y, ldy, stream);
 }
 
+// Scratch of dvdq_qlinear_static: part of the library image, so no allocation is ever needed.
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) uint8_t g_static_scratch[DVDQ_STATIC_SCRATCH_BYTES];
+
+dvdq_status dvdq_qlinear_static(const void* X, int64_t M, int64_t ldx, const dvdq_act_quant* q, const dvdq_weights* w,
+                                const void* bias, int32_t act, void* Y, int64_t ldy, void* stream) {
+    constexpr int kMaxDevices = 64;
+    static void* scratch_of_device[kMaxDevices] = {nullptr};
+    dvdq_status s = validate_weights(w);
+    if (s != DVDQ_OK) return s;
+    if ((s = validate_act_quant(q, w->K)) != DVDQ_OK) return s;
+    if (M < 0) return DVDQ_ERR_SHAPE;
+    if (M == 0) return DVDQ_OK;
+    const WorkspacePlan p = workspace_plan(M, w->K, q->bits);
+    if (p.total > (int64_t)DVDQ_STATIC_SCRATCH_BYTES) return DVDQ_ERR_WORKSPACE;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DVDQ_ERR_CUDA;
+    if (scratch_of_device[dev] == nullptr) {  // set-up, once per device, with that device current
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return DVDQ_ERR_CUDA;
+        scratch_of_device[dev] = ptr;
+    }
+    uint8_t* ws = static_cast<uint8_t*>(scratch_of_device[dev]);
+    void* codes = ws + p.codes_off;
+    float* scales = reinterpret_cast<float*>(ws + p.scales_off);
+    int32_t* sums = reinterpret_cast<int32_t*>(ws + p.sums_off);
+    if ((s = dvdq_rotate_quantize(X, M, w->K, ldx, q, codes, scales, sums, stream)) != DVDQ_OK) return s;
+    return dvdq_qgemm(codes, scales, sums, M, q, w, bias, act, Y, ldy, stream);
+}
+
 dvdq_status dvdq_pack_act_codes(const int8_t* codes_nat, int64_t M, int64_t K, const dvdq_act_quant* q,
                                 void* codes_out, int32_t* code_sums_out, void* stream) {
     if (M < 0 || validate_k(K) != DVDQ_OK) return DVDQ_ERR_SHAPE;
