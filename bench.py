@@ -177,6 +177,7 @@ def config_of(wl, args):
 
 def run_cuda(args, wl):
     from paper_2505_18663_b200 import binding as B
+    from paper_2505_18663_b200 import dist as D
     from paper_2505_18663_b200 import workloads as W
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -251,18 +252,14 @@ def run_cuda(args, wl):
     t_end.record()
     barrier()
     clocks = sampler.stop() if rank == 0 else None
-    elapsed_ms = t_begin.elapsed_time(t_end)
-    if dist is not None:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = D.max_over_ranks(t_begin.elapsed_time(t_end), dist, dev)
     status, detail = B.dvdq_last_device_status()
     if status != B.OK:
         raise SystemExit(f"device status {status} ({B.status_string(status)}), wait id {detail}")
 
     ms_per_step = elapsed_ms / args.steps
     ops_per_step = sum(layer_ops(M, L["layer"]) for L in layers)
-    value = world * ops_per_step / (ms_per_step * 1e-3) / 1e12
+    value = D.aggregate_rate(ops_per_step, ms_per_step, world) / 1e12
 
     # ---- per-kernel durations from the events of the timed region (this rank)
     rq_ms = [sum(ev[s][li][0].elapsed_time(ev[s][li][1]) for s in range(args.steps)) / args.steps for li in range(len(layers))]
@@ -282,7 +279,7 @@ def run_cuda(args, wl):
 
     # ---- end to end through dvdq_qlinear with HOST buffers (pinned), copies inside the timed region
     e2e = None
-    if rank == 0 or world > 1:
+    if not args.no_e2e:
         e2e = run_e2e(args, wl, layers, xs, dev, B, dist, world)
 
     if rank != 0:
@@ -355,11 +352,8 @@ def run_e2e(args, wl, layers, xs, dev, B, dist, world):
         step()
     t1.record()
     torch.cuda.synchronize()
-    ms = t0.elapsed_time(t1) / steps
-    if dist is not None:
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    from paper_2505_18663_b200 import dist as D
+    ms = D.max_over_ranks(t0.elapsed_time(t1) / steps, dist, dev)
     ops = sum(layer_ops(M, L["layer"]) for L in layers)
     return {"value": world * ops / (ms * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": ms, "steps": steps,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "api": "dvdq_qlinear, pinned host buffers"}
@@ -374,9 +368,14 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=384, help="token sample timed on the CPU oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling runs)")
     args = ap.parse_args()
     from paper_2505_18663_b200 import workloads as W
     wl = W.WORKLOADS[args.workload]
+    if args.tokens > 0:
+        import dataclasses
+        wl = dataclasses.replace(wl, M=args.tokens)
     if args.impl == "reference":
         run_reference(args, wl)
     else:

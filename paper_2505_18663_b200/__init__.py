@@ -3,6 +3,6 @@
 ``binding`` exposes the C ABI of ``include/dvdq.h`` with the same names; ``build``
 compiles the CUDA library in-tree; ``workloads`` holds the seeded synthetic inputs.
 """
-from . import binding, build, workloads  # noqa: F401
+from . import binding, build, dist, workloads  # noqa: F401
 
-__all__ = ["binding", "build", "workloads"]
+__all__ = ["binding", "build", "dist", "workloads"]

@@ -30,7 +30,7 @@
 namespace dvdq {
 
 constexpr int kBM = 128, kBN = 256, kBK = 128;
-constexpr int kPackedStages = 4, kWideStages = 2;
+constexpr int kWideStages = 2;
 constexpr int kUnpackWarps = 8, kEpilogueWarps = 4;
 constexpr int kFirstEpilogueWarp = 2, kFirstUnpackWarp = 6;
 constexpr int kGemmThreads = (2 + kEpilogueWarps + kUnpackWarps) * 32;
@@ -38,6 +38,7 @@ constexpr int kTmemCols = 512;
 
 template <int BITS>
 struct GemmSmem {
+    static constexpr int kPackedStages = (BITS == 4) ? 4 : 3;     // what fits beside the other buffers
     static constexpr int kALo = kBM * kBK / 2;                    // packed low plane / A4 codes
     static constexpr int kAHi = (BITS == 6) ? kBM * kBK / 4 : 0;  // packed high plane
     static constexpr int kW = kBN * kBK / 2;
@@ -46,8 +47,10 @@ struct GemmSmem {
     static constexpr int kWideStage = kWideA + kWideW;
     static constexpr int kWideOff = 0;  // 1024-byte aligned tiles first
     static constexpr int kPackedOff = kWideOff + kWideStages * kWideStage;
-    static constexpr int kConstOff = kPackedOff + kPackedStages * kPackedStage;
-    static constexpr int kConstPerWarp = 3 * kBN * 4;  // delta, zc, bias for 256 channels
+    static constexpr int kStageOutOff = kPackedOff + kPackedStages * kPackedStage;  // 1024-byte aligned
+    static constexpr int kStageOutPerWarp = 2 * 32 * 64;  // two buffers of 32 rows x 32 bf16
+    static constexpr int kConstOff = kStageOutOff + kEpilogueWarps * kStageOutPerWarp;
+    static constexpr int kConstPerWarp = 3 * kBN * 4;  // delta, zero-point rest, bias for 256 channels
     static constexpr int kBarOff = kConstOff + kEpilogueWarps * kConstPerWarp;
     static constexpr int kNumBars = 2 * kPackedStages + 2 * kWideStages + 4;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
@@ -62,11 +65,13 @@ __device__ __forceinline__ float gelu_tanh_f32(float y) {
 template <int BITS, bool RAW>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmAhi,
-             const __grid_constant__ CUtensorMap tmW, const float* __restrict__ scales,
+             const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmY,
+             const float* __restrict__ scales,
              const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
              const __nv_bfloat16* __restrict__ bias, __nv_bfloat16* __restrict__ Y, int64_t ldy,
              int32_t* __restrict__ acc_out, int64_t ldacc, int M, int N, int K, int act) {
     using S = GemmSmem<BITS>;
+    constexpr int kPackedStages = S::kPackedStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -164,11 +169,15 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     } else if (warp < kFirstUnpackWarp) {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;  // tensor-memory lane quarter this warp may read
-        float* c_delta = reinterpret_cast<float*>(smem + S::kConstOff + (warp - kFirstEpilogueWarp) * S::kConstPerWarp);
-        int32_t* c_zc = reinterpret_cast<int32_t*>(c_delta + kBN);
-        float* c_bias = reinterpret_cast<float*>(c_zc + kBN);
+        const int ew = warp - kFirstEpilogueWarp;
+        float* c_delta = reinterpret_cast<float*>(smem + S::kConstOff + ew * S::kConstPerWarp);
+        float* c_zc = c_delta + kBN;    // (z_n - 8) as a float: exact, |.| <= 8
+        float* c_bias = c_zc + kBN;
+        const uint32_t stg0 = sbase + S::kStageOutOff + ew * S::kStageOutPerWarp;
+        uint8_t* stg_ptr = smem + S::kStageOutOff + ew * S::kStageOutPerWarp;
         constexpr int kShift = (BITS == 4) ? 8 : 6;
-        uint32_t lt = 0;
+        if (!RAW && lane == 0) tma_prefetch_desc(&tmY);
+        uint32_t lt = 0, nstore = 0;
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++lt) {
             const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
             const int m0 = (tile / num_n) * kBM, n0 = (tile % num_n) * kBN;
@@ -177,7 +186,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 const int n = n0 + c;
                 const bool okn = n < N;
                 c_delta[c] = okn ? delta[n] : 0.f;
-                c_zc[c] = okn ? zc[n] : 0;
+                c_zc[c] = okn ? (float)zc[n] : 0.f;
                 c_bias[c] = (okn && bias != nullptr) ? __bfloat162float(bias[n]) : 0.f;
             }
             __syncwarp();
@@ -187,6 +196,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const bool row_ok = row < M;
             const float s_i = (!RAW && row_ok) ? scales[row] : 0.f;
             const int32_t S_i = row_ok ? sums[row] : 0;
+            const float S_f = (float)S_i;  // |sum of codes| <= K * 32 < 2^24: exact
 #pragma unroll 1
             for (int c = 0; c < kBN / 32; ++c) {
                 uint32_t r[32];
@@ -198,39 +208,65 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) {
                         int4 o;
-                        o.x = ((int32_t)r[j] >> kShift) - c_zc[c * 32 + j] * S_i;
-                        o.y = ((int32_t)r[j + 1] >> kShift) - c_zc[c * 32 + j + 1] * S_i;
-                        o.z = ((int32_t)r[j + 2] >> kShift) - c_zc[c * 32 + j + 2] * S_i;
-                        o.w = ((int32_t)r[j + 3] >> kShift) - c_zc[c * 32 + j + 3] * S_i;
+                        o.x = ((int32_t)r[j] >> kShift) - __float2int_rn(c_zc[c * 32 + j]) * S_i;
+                        o.y = ((int32_t)r[j + 1] >> kShift) - __float2int_rn(c_zc[c * 32 + j + 1]) * S_i;
+                        o.z = ((int32_t)r[j + 2] >> kShift) - __float2int_rn(c_zc[c * 32 + j + 2]) * S_i;
+                        o.w = ((int32_t)r[j + 3] >> kShift) - __float2int_rn(c_zc[c * 32 + j + 3]) * S_i;
                         if (row_ok && nb + j < N) *reinterpret_cast<int4*>(dst + j) = o;
                     }
                 } else {
-                    __nv_bfloat16* dst = Y + (int64_t)row * ldy + nb;
+                    // The staging buffer used two chunks ago must have been read by its TMA store.
+                    if (lane == 0) tma_store_wait_read<1>();
+                    __syncwarp();
+                    uint8_t* buf = stg_ptr + (nstore & 1u) * (32 * 64);
 #pragma unroll
                     for (int j = 0; j < 32; j += 8) {
+                        const float4 d0 = *reinterpret_cast<const float4*>(c_delta + c * 32 + j);
+                        const float4 d1 = *reinterpret_cast<const float4*>(c_delta + c * 32 + j + 4);
+                        const float4 z0 = *reinterpret_cast<const float4*>(c_zc + c * 32 + j);
+                        const float4 z1 = *reinterpret_cast<const float4*>(c_zc + c * 32 + j + 4);
+                        const float4 b0 = *reinterpret_cast<const float4*>(c_bias + c * 32 + j);
+                        const float4 b1 = *reinterpret_cast<const float4*>(c_bias + c * 32 + j + 4);
+                        const float dl[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+                        const float zz[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
+                        const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                        float v[8];
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) {
+                            // int -> float without the conversion pipe: |acc >> shift| <= K*32*8 <= 2^22
+                            const int32_t sh = (int32_t)r[j + t] >> kShift;
+                            float f = __int_as_float(sh + 0x4B400000) - 12582912.0f;
+                            f = fmaf(-zz[t], S_f, f);                 // rest of the zero point, exact
+                            float y = fmaf(f, s_i * dl[t], bb[t]);
+                            if (act == 1) y = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(y)));
+                            v[t] = y;
+                        }
                         uint32_t pk[4];
 #pragma unroll
                         for (int t = 0; t < 4; ++t) {
-                            float v[2];
-#pragma unroll
-                            for (int h = 0; h < 2; ++h) {
-                                const int col = c * 32 + j + 2 * t + h;
-                                const int32_t acc = ((int32_t)r[j + 2 * t + h] >> kShift) - c_zc[col] * S_i;
-                                float y = fmaf((float)acc, s_i * c_delta[col], c_bias[col]);
-                                if (act == 1) y = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(y)));
-                                v[h] = y;
-                            }
-                            __nv_bfloat162 b2 = __floats2bfloat162_rn(v[0], v[1]);
+                            __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * t], v[2 * t + 1]);
                             pk[t] = *reinterpret_cast<uint32_t*>(&b2);
                         }
-                        if (row_ok && nb + j < N) *reinterpret_cast<uint4*>(dst + j) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        // 64-byte rows, 16-byte chunk index XORed with (row >> 1) & 3: the layout a
+                        // 64B-swizzled TMA store reads, and conflict-free for this per-row write.
+                        const int ch = (j >> 3) ^ ((lane >> 1) & 3);
+                        *reinterpret_cast<uint4*>(buf + lane * 64 + ch * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && nb < N && m0 + q * 32 < M) {
+                        tma_store_2d(&tmY, stg0 + (nstore & 1u) * (32 * 64), nb, m0 + q * 32);
+                        tma_store_commit();
+                    }
+                    ++nstore;
                 }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty(a));
         }
+        if (!RAW && lane == 0) tma_store_wait_all();
+        __syncwarp();
     } else {
         // ------------------------------------------------------------ widen 4/6-bit codes to int8
         const int u = threadIdx.x - kFirstUnpackWarp * 32;  // 0..255
@@ -318,6 +354,20 @@ inline PFN_encodeTiled get_encode_tiled() {
 
 // Byte matrix [rows, row_len] with row pitch `pitch`, tiles of box_rows x box_bytes, no swizzle,
 // out-of-range bytes read as zero.
+// bf16 matrix [rows, cols] with row pitch ld elements, tiles of 32 x 32, 64-byte swizzle
+// (the layout the epilogue stages its output in).
+inline bool make_out_map(CUtensorMap* tm, const void* base, uint64_t cols, uint64_t rows, uint64_t ld) {
+    PFN_encodeTiled enc = get_encode_tiled();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {ld * 2};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 inline bool make_byte_map(CUtensorMap* tm, const void* base, uint64_t row_len, uint64_t rows, uint64_t pitch,
                           uint32_t box_bytes, uint32_t box_rows) {
     PFN_encodeTiled enc = get_encode_tiled();
@@ -340,7 +390,7 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
     const BlobLayout L = blob_layout(N, K);
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
     const uint64_t pitch = (uint64_t)act_row_bytes(K, BITS);
-    CUtensorMap tmA, tmAhi, tmW;
+    CUtensorMap tmA, tmAhi, tmW, tmY;
     if (!make_byte_map(&tmA, codes, (uint64_t)K / 2, (uint64_t)M, pitch, kBK / 2, kBM)) return DVDQ_ERR_CUDA;
     if (BITS == 6) {
         if (!make_byte_map(&tmAhi, static_cast<const uint8_t*>(codes) + K / 2, (uint64_t)K / 4, (uint64_t)M, pitch, kBK / 4, kBM))
@@ -349,6 +399,12 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
         tmAhi = tmA;
     }
     if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, kBN)) return DVDQ_ERR_CUDA;
+
+    if (RAW) {
+        tmY = tmA;  // unused
+    } else if (!make_out_map(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)) {
+        return DVDQ_ERR_CUDA;
+    }
 
     static int sm_count = 0;
     if (sm_count == 0) {
@@ -364,7 +420,7 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
     }
     const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
     const unsigned grid = (unsigned)(tiles < sm_count ? tiles : sm_count);
-    kern<<<grid, kGemmThreads, S::kTotal, st>>>(tmA, tmAhi, tmW, scales, sums,
+    kern<<<grid, kGemmThreads, S::kTotal, st>>>(tmA, tmAhi, tmW, tmY, scales, sums,
                                                 reinterpret_cast<const float*>(blob + L.delta_offset),
                                                 reinterpret_cast<const int32_t*>(blob + L.zc_offset),
                                                 static_cast<const __nv_bfloat16*>(bias), static_cast<__nv_bfloat16*>(Y), ldy,
