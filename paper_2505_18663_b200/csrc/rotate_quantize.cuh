@@ -1,12 +1,29 @@
 // Online activation transform (Sec. 3.2, Eq. 10): rotate -> auto-scale -> quantize -> pack,
 // one kernel, bound by HBM traffic (2K bytes read, K*b/8 + 8 bytes written per token).
 //
-// General-shape kernel, natural K order.  A warp owns a span of 1024 consecutive channels of
-// one token: lane L holds four 16-byte chunks, channels c*256 + 8L + j (c chunk, j in 0..7),
-// as 32 fp32 registers.  The Walsh-Hadamard butterflies over channel-index bits 0..log2(B)-1
-// run in registers: bits 0-2 inside a chunk, bits 3-7 across lanes with shuffles, bits 8-9
-// between chunks.  Blocks smaller than 1024 simply skip the upper stages, so one span holds
-// 1024/B whole blocks.  The 1/sqrt(B) normalisation is folded into the scale.
+// A warp owns a span of 1024 consecutive channels of one token (index bits 0..9 below are the
+// bits of the channel index inside the span).  The Walsh-Hadamard transform over those bits is
+// split so that no butterfly ever needs a warp shuffle:
+//
+//   load     lane L reads four 16-byte chunks, channels c*256 + 8L + e: bits 0-2 in the chunk,
+//            bits 3-7 = lane, bits 8-9 = chunk number.
+//   stage A  bits {0,1,3,4}: the raw bf16 words are the B operand of mma.sync.m16n8k16 and the
+//            A operand is the +-1 matrix H_16, so D = H_16 * B holds the four butterflies.
+//            bf16 inputs and +-1 factors make every product exact; the sums accumulate in fp32.
+//            The MMA also moves data: afterwards a lane holds bits {1,2,5,8,9} in registers.
+//   stage B  bits {2,8,9} as packed f32x2 adds/subs on register pairs, bit 5 as scalar add/sub.
+//   turn     one conflict-free transposition through shared memory (8 x 16-byte stores and loads
+//            per lane) brings bits {6,7} and {0,1,2} into registers.
+//   stage C  bits {6,7} as packed f32x2 adds/subs.
+//
+// After stage C a lane holds, for each j = bits 7:6, eight channels that are consecutive in
+// memory, i.e. exactly one 32-bit word of packed 4-bit codes (or of the low plane of 6-bit
+// codes), so the packed layout stays in natural channel order.  Blocks smaller than 1024 skip
+// the stages of the upper bits; no rotation (B = 0) runs the same data path with the identity
+// in place of H_16.  The 1/sqrt(B) normalisation is folded into the scale.
+//
+// Rounding: c = rne(x~ * (qmax / absmax)) as one fused multiply-add onto 1.5 * 2^23, which
+// leaves the two's-complement code in the low mantissa bits.  (B = 0 divides instead.)
 #pragma once
 
 #include "dvdq_common.cuh"
@@ -14,151 +31,352 @@
 namespace dvdq {
 
 constexpr int kRqSpan = 1024;
+constexpr int kRqMaxWarps = 16;
 
-template <int LOG2B, int BITS>
-__global__ void __launch_bounds__(512)
-rq_natural_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
-                  uint8_t* __restrict__ codes, float* __restrict__ scales, int32_t* __restrict__ sums,
-                  int spans, int tokens_per_cta) {
-    __shared__ float s_max[32];
-    __shared__ int s_sum[32];
+__device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+// (a, b) -> (a + b, a - b) on packed pairs
+__device__ __forceinline__ void f2_butterfly(uint64_t& a, uint64_t& b) {
+    const uint64_t s = f2_add(a, b), d = f2_sub(a, b);
+    a = s;
+    b = d;
+}
+
+// D = A * B with A 16x16 (row major), B 16x8 (column major), bf16 inputs, fp32 result, C = 0.
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%10, %10, %10, %10};"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.0f));
+}
+
+// Entry (m, s) of the stage-A matrix as bf16 bits: the Sylvester sign (-1)^popcount(m & s), or the
+// identity when there is no rotation.
+template <bool ROTATE>
+__device__ __forceinline__ uint32_t stage_a_entry(int m, int s) {
+    if (ROTATE) return (__popc(m & s) & 1) ? 0xBF80u : 0x3F80u;
+    return m == s ? 0x3F80u : 0u;
+}
+
+// One warp-span of work per loop iteration; CTAs are persistent and walk over groups of
+// tokens_per_cta tokens.  FULL = every span is complete (K a multiple of 1024): no per-chunk
+// predicates.  Per iteration there is ONE CTA barrier (the token absmax); the code sums of
+// iteration i are finalised after the barrier of iteration i + 1 from double-buffered slots.
+template <int LOG2B, int BITS, bool FULL>
+__global__ void __maxnreg__(80)  // two CTAs of 12 warps per SM
+rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
+          uint8_t* __restrict__ codes, float* __restrict__ scales, int32_t* __restrict__ sums,
+          int spans, int tokens_per_cta, int num_groups) {
+    extern __shared__ float4 s_turn[];  // 256 float4 per warp
+    __shared__ float s_max[2][kRqMaxWarps];
+    __shared__ int s_sum[2][kRqMaxWarps];
+    constexpr bool kRot = LOG2B > 0;
+    constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
+    constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: ulp 1, so the fma rounds to an integer
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int tl = warp / spans, sp = warp - tl * spans;
-    const int64_t token = (int64_t)blockIdx.x * tokens_per_cta + tl;
-    const bool tok_ok = token < M;
+    const int g = lane >> 2, t = lane & 3;
 
-    float v[32];
-    const __nv_bfloat16* xrow = X + (tok_ok ? token : 0) * ldx;
+    // ---- loop invariants
+    // stage-A matrix fragment (H_16, or the identity without a rotation)
+    uint32_t afrag[4];
+    afrag[0] = stage_a_entry<kRot>(g, 2 * t) | (stage_a_entry<kRot>(g, 2 * t + 1) << 16);
+    afrag[1] = stage_a_entry<kRot>(g + 8, 2 * t) | (stage_a_entry<kRot>(g + 8, 2 * t + 1) << 16);
+    afrag[2] = stage_a_entry<kRot>(g, 2 * t + 8) | (stage_a_entry<kRot>(g, 2 * t + 9) << 16);
+    afrag[3] = stage_a_entry<kRot>(g + 8, 2 * t + 8) | (stage_a_entry<kRot>(g + 8, 2 * t + 9) << 16);
+    // channel of the lane's first load chunk and of its first output word
+    const int ld_e0 = sp * kRqSpan + lane * 8;                                   // + c * 256
+    const int st_e0 = sp * kRqSpan + ((lane >> 3) * 32 + (lane & 7)) * 8;        // + j * 64
+    uint32_t ld_ok = 0xFu, st_ok = 0xFu;
+    if (!FULL) {
+        ld_ok = st_ok = 0u;
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        const int e0 = sp * kRqSpan + c * 256 + lane * 8;
-        uint4 raw = make_uint4(0u, 0u, 0u, 0u);
-        if (tok_ok && e0 < K) raw = __ldg(reinterpret_cast<const uint4*>(xrow + e0));
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {  // a bf16 is the upper half of an fp32
-            v[c * 8 + 2 * j] = __uint_as_float(w[j] << 16);
-            v[c * 8 + 2 * j + 1] = __uint_as_float(w[j] & 0xFFFF0000u);
+        for (int c = 0; c < 4; ++c) {
+            if (ld_e0 + c * 256 < K) ld_ok |= 1u << c;
+            if (st_e0 + c * 64 < K) st_ok |= 1u << c;
         }
     }
-
-    // in-chunk stages: index bits 0,1,2
-#pragma unroll
-    for (int h = 1; h < 8; h <<= 1) {
-        if (h < (1 << LOG2B)) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                if ((i & h) == 0) {
-                    const float a = v[i], b = v[i + h];
-                    v[i] = a + b;
-                    v[i + h] = a - b;
-                }
-            }
-        }
+    // turn addresses (float4 units): write = wr[r0] + 64 c, read = rd ^ (j | i0 << 2)
+    float4* turn = s_turn + warp * 256;
+    int wr[2];
+    {
+        const int b34 = lane >> 3, b0 = (lane >> 2) & 1, b67 = lane & 3;
+        const int low = (b67 | (b0 << 2)) ^ b34;
+        wr[0] = b34 * 8 + low;
+        wr[1] = (b34 + 4) * 8 + (low ^ 4);
     }
-    // cross-lane stages: index bits 3..7 are lane bits 0..4
-#pragma unroll
-    for (int bit = 3; bit < 8; ++bit) {
-        if (bit < LOG2B) {
-            const int m = 1 << (bit - 3);
-            const bool upper = (lane & m) != 0;
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const float o = __shfl_xor_sync(0xFFFFFFFFu, v[i], m);
-                v[i] = upper ? (o - v[i]) : (v[i] + o);
-            }
-        }
-    }
-    // cross-chunk stages: index bits 8,9
-#pragma unroll
-    for (int bit = 8; bit < 10; ++bit) {
-        if (bit < LOG2B) {
-            const int h = 8 << (bit - 8);
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                if ((i & h) == 0) {
-                    const float a = v[i], b = v[i + h];
-                    v[i] = a + b;
-                    v[i + h] = a - b;
-                }
-            }
-        }
-    }
-
-    // per-token absmax (of the un-normalised transform)
-    float amax = 0.f;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) amax = fmaxf(amax, fabsf(v[i]));
-#pragma unroll
-    for (int m = 16; m > 0; m >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, m));
-    if (lane == 0) s_max[warp] = amax;
-    __syncthreads();
-    amax = 0.f;
-    for (int s = 0; s < spans; ++s) amax = fmaxf(amax, s_max[tl * spans + s]);
-
-    constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
-    const float inv = amax > 0.f ? qmax / amax : 0.f;
-
-    int q[32];
-    int lsum = 0;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        q[i] = __float2int_rn(v[i] * inv);
-        lsum += q[i];
-    }
-#pragma unroll
-    for (int m = 16; m > 0; m >>= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, m);
-    if (lane == 0) s_sum[warp] = lsum;
-
-    // pack + store
+    const int rd = lane * 8 + (lane & 7);
     const int64_t row_bytes = act_row_bytes(K, BITS);
-    uint8_t* crow = codes + (tok_ok ? token : 0) * row_bytes;
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        const int e0 = sp * kRqSpan + c * 256 + lane * 8;
-        const bool ok = tok_ok && e0 < K;
-        uint32_t lo = 0u;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) lo |= ((uint32_t)q[c * 8 + j] & 0xFu) << (4 * j);
-        if (ok) *reinterpret_cast<uint32_t*>(crow + (e0 >> 1)) = lo;
-        if (BITS == 6) {
-            const int a = lane & 1;
-            uint32_t hi = 0u;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) hi |= (((uint32_t)q[c * 8 + j] >> 4) & 0x3u) << (2 * (4 * (j >> 1) + (j & 1)));
-            hi <<= 4 * a;  // hi_field_shift(a, j) = hi_field_shift(0, j) + 4a
-            hi |= __shfl_xor_sync(0xFFFFFFFFu, hi, 1);
-            if (ok && ((c ^ lane) & 1) == 0) *reinterpret_cast<uint32_t*>(crow + (K >> 1) + ((e0 >> 4) << 2)) = hi;
-        }
-    }
+    const float rs = (LOG2B & 1) ? rsqrtf((float)(1 << LOG2B)) : 1.0f / (float)(1 << (LOG2B / 2));
 
-    __syncthreads();
-    if (sp == 0 && lane == 0 && tok_ok) {
-        int tsum = 0;
-        for (int s = 0; s < spans; ++s) tsum += s_sum[tl * spans + s];
-        // s_i = (absmax / sqrt(B)) / qmax
-        const float rs = (LOG2B & 1) ? rsqrtf((float)(1 << LOG2B)) : 1.0f / (float)(1 << (LOG2B / 2));
-        scales[token] = (amax * rs) / qmax;
-        sums[token] = tsum;
+    auto load_span = [&](uint4 (&raw)[4], int group) {
+        int64_t token = (int64_t)group * tokens_per_cta + tl;
+        if (token >= M) token = M - 1;  // a clamped duplicate; its results are never stored
+        const uint4* src = reinterpret_cast<const uint4*>(X + token * ldx + ld_e0);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            raw[c] = make_uint4(0u, 0u, 0u, 0u);
+            if (FULL || (ld_ok >> c & 1u)) raw[c] = __ldg(src + c * 32);
+        }
+    };
+
+    uint4 raw[4];
+    int group = blockIdx.x;
+    if (group < num_groups) load_span(raw, group);
+    int64_t prev_token = -1;
+    float prev_amax = 0.f;
+    uint32_t it = 0;
+    for (; group < num_groups; group += gridDim.x, ++it) {
+        const uint32_t buf = it & 1u;
+        const int64_t token = (int64_t)group * tokens_per_cta + tl;
+        const bool tok_ok = token < M;
+
+        // ---- stage A: D = H_16 * B on index bits {0, 3, 4, 1} (k-slot bit 0 = half of a word,
+        // bits 1-2 = lane & 3, bit 3 = which of the two words).  Word pair p = bit 2.
+        // acc[c][p][r]: c = bits 9:8, p = bit 2, r & 1 = bit 5, r >> 1 = bit 1.
+        // The lane now stands for bits 7:6 (lane & 3), bit 0 (lane >> 2 & 1), bits 4:3 (lane >> 3).
+        float acc[4][2][4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            mma_bf16_16816(acc[c][0], afrag, raw[c].x, raw[c].y);
+            mma_bf16_16816(acc[c][1], afrag, raw[c].z, raw[c].w);
+        }
+        // the next group's loads fly while this one is transformed
+        if (group + (int)gridDim.x < num_groups) load_span(raw, group + gridDim.x);
+
+        // ---- stage B: bits 2, 8, 9 on packed pairs (the pair is bit 5), then bit 5 itself
+        uint64_t P[4][2][2];
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int p = 0; p < 2; ++p)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) P[c][p][h] = f2_pack(acc[c][p][2 * h], acc[c][p][2 * h + 1]);
+        if (kRot) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) f2_butterfly(P[c][0][h], P[c][1][h]);
+        }
+        if (LOG2B > 8) {
+#pragma unroll
+            for (int c = 0; c < 4; c += 2)
+#pragma unroll
+                for (int p = 0; p < 2; ++p)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) f2_butterfly(P[c][p][h], P[c + 1][p][h]);
+        }
+        if (LOG2B > 9) {
+#pragma unroll
+            for (int c = 0; c < 2; ++c)
+#pragma unroll
+                for (int p = 0; p < 2; ++p)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) f2_butterfly(P[c][p][h], P[c + 2][p][h]);
+        }
+
+        // ---- turn: float4 = bits (1, 2) varying; address = [bits 9 8 5 4 3 | (bits 0 7 6) ^ (bits 5 4 3)]
+        __syncwarp();  // the previous iteration's reads of this warp's turn buffer are done
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            float v[2][2][2];  // [p][h][r0]
+#pragma unroll
+            for (int p = 0; p < 2; ++p)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    float lo, hi;
+                    f2_unpack(P[c][p][h], lo, hi);
+                    v[p][h][0] = kRot ? lo + hi : lo;
+                    v[p][h][1] = kRot ? lo - hi : hi;
+                }
+#pragma unroll
+            for (int r0 = 0; r0 < 2; ++r0)
+                turn[wr[r0] + 64 * c] = make_float4(v[0][0][r0], v[0][1][r0], v[1][0][r0], v[1][1][r0]);
+        }
+        __syncwarp();
+        // The lane now stands for bits 5:3 (lane & 7) and bits 9:8 (lane >> 3);
+        // W[j][i0][h]: j = bits 7:6, i0 = bit 0, h = bit 2, the pair is bit 1.
+        uint64_t W[4][2][2];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int i0 = 0; i0 < 2; ++i0) {
+                const float4 f = turn[rd ^ (j | (i0 << 2))];
+                W[j][i0][0] = f2_pack(f.x, f.y);
+                W[j][i0][1] = f2_pack(f.z, f.w);
+            }
+
+        // ---- stage C: bits 6 and 7
+        if (LOG2B > 6) {
+#pragma unroll
+            for (int j = 0; j < 4; j += 2)
+#pragma unroll
+                for (int i0 = 0; i0 < 2; ++i0)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) f2_butterfly(W[j][i0][h], W[j + 1][i0][h]);
+        }
+        if (LOG2B > 7) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+                for (int i0 = 0; i0 < 2; ++i0)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) f2_butterfly(W[j][i0][h], W[j + 2][i0][h]);
+        }
+
+        // val[j][e]: channel (lane >> 3) * 256 + j * 64 + (lane & 7) * 8 + e of the span,
+        // e = i0 + 2 * bit1 + 4 * h
+        float val[4][8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int i0 = 0; i0 < 2; ++i0)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) f2_unpack(W[j][i0][h], val[j][i0 + 4 * h], val[j][i0 + 4 * h + 2]);
+
+        // ---- per-token absmax (of the un-normalised transform)
+        float amax = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(val[j][e]));
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, m));
+        if (lane == 0) s_max[buf][warp] = amax;
+        __syncthreads();
+        if (spans > 1) {
+            amax = 0.f;
+            for (int s = 0; s < spans; ++s) amax = fmaxf(amax, s_max[buf][tl * spans + s]);
+        }
+        // the previous iteration's token: all its code sums are in shared memory by now
+        if (sp == 0 && lane == 0 && prev_token >= 0) {
+            int tsum = 0;
+            for (int s = 0; s < spans; ++s) tsum += s_sum[buf ^ 1u][tl * spans + s];
+            scales[prev_token] = (prev_amax * rs) / qmax;  // s_i = (absmax / sqrt(B)) / qmax
+            sums[prev_token] = tsum;
+        }
+        const float inv = amax > 0.f ? qmax / amax : 0.f;
+
+        // ---- quantize, sum, pack, store
+        uint8_t* crow = codes + (tok_ok ? token : 0) * row_bytes;
+        int lsum = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t b[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                if (kRot) {
+                    b[e] = __float_as_uint(fmaf(val[j][e], inv, kMagic));
+                } else {
+                    // Without a rotation x~ is a bf16 value, x~ * qmax is exact and exact half-way
+                    // quotients are common: take the correctly rounded quotient so that they survive.
+                    const float quo = amax > 0.f ? __fdiv_rn(val[j][e] * qmax, amax) : 0.f;
+                    b[e] = __float_as_uint(quo + kMagic);
+                }
+            }
+            // low bytes (= the codes as int8) of the even and of the odd channels
+            const uint32_t E = __byte_perm(__byte_perm(b[0], b[2], 0x0040), __byte_perm(b[4], b[6], 0x0040), 0x5410);
+            const uint32_t O = __byte_perm(__byte_perm(b[1], b[3], 0x0040), __byte_perm(b[5], b[7], 0x0040), 0x5410);
+            lsum = __dp4a((int)E, 0x01010101, lsum);
+            lsum = __dp4a((int)O, 0x01010101, lsum);
+            const uint32_t lo = (E & 0x0F0F0F0Fu) | ((O << 4) & 0xF0F0F0F0u);
+            const int e0 = st_e0 + j * 64;
+            const bool ok = tok_ok && (FULL || (st_ok >> j & 1u));
+            if (ok) *reinterpret_cast<uint32_t*>(crow + (e0 >> 1)) = lo;
+            if (BITS == 6) {
+                // bits 5:4 of 16 consecutive channels share one word of the high plane; the two
+                // halves sit in neighbouring lanes
+                uint32_t hi = ((E >> 4) & 0x03030303u) | ((O >> 2) & 0x0C0C0C0Cu);
+                hi <<= 4 * (lane & 1);
+                hi |= __shfl_xor_sync(0xFFFFFFFFu, hi, 1);
+                if (ok && ((j ^ lane) & 1) == 0) *reinterpret_cast<uint32_t*>(crow + (K >> 1) + ((e0 >> 4) << 2)) = hi;
+            }
+        }
+#pragma unroll
+        for (int m = 16; m > 0; m >>= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, m);
+        if (lane == 0) s_sum[buf][warp] = lsum;
+        prev_token = tok_ok ? token : -1;
+        prev_amax = amax;
     }
+    __syncthreads();
+    if (sp == 0 && lane == 0 && prev_token >= 0) {
+        const uint32_t buf = (it & 1u) ^ 1u;  // the last iteration's slots
+        int tsum = 0;
+        for (int s = 0; s < spans; ++s) tsum += s_sum[buf][tl * spans + s];
+        scales[prev_token] = (prev_amax * rs) / qmax;
+        sums[prev_token] = tsum;
+    }
+}
+
+template <int LOG2B, int BITS, bool FULL>
+static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t ldx, void* codes, float* scales,
+                                    int32_t* sums, cudaStream_t st) {
+    const int spans = (int)((K + kRqSpan - 1) / kRqSpan);
+    if (spans > kRqMaxWarps) return DVDQ_ERR_SHAPE;
+    int tpc = 12 / spans;
+    if (tpc < 1) tpc = 1;
+    const int warps = spans * tpc;
+    const int threads = warps * 32;
+    const size_t smem = (size_t)warps * 256 * sizeof(float4);
+    const int64_t groups = (M + tpc - 1) / tpc;
+    if (groups > 0x7FFFFFFFll) return DVDQ_ERR_SHAPE;
+    auto kern = rq_kernel<LOG2B, BITS, FULL>;
+    static bool attr_set = false;
+    static int sm_count = 0;
+    static int blocks_per_sm[kRqMaxWarps + 1] = {0};
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 kRqMaxWarps * 256 * (int)sizeof(float4)) != cudaSuccess)
+            return DVDQ_ERR_CUDA;
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return DVDQ_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DVDQ_ERR_CUDA;
+        attr_set = true;
+    }
+    if (blocks_per_sm[warps] == 0) {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, threads, smem) != cudaSuccess || n < 1) return DVDQ_ERR_CUDA;
+        blocks_per_sm[warps] = n;
+    }
+    const int64_t resident = (int64_t)sm_count * blocks_per_sm[warps];
+    const unsigned grid = (unsigned)(groups < resident ? groups : resident);
+    kern<<<grid, threads, smem, st>>>((const __nv_bfloat16*)X, M, (int)K, ldx, (uint8_t*)codes, scales, sums, spans, tpc,
+                                      (int)groups);
+    return cuda_status(cudaGetLastError());
 }
 
 template <int BITS>
 static dvdq_status launch_rq_bits(const void* X, int64_t M, int64_t K, int64_t ldx, int rot_block, void* codes,
                                   float* scales, int32_t* sums, cudaStream_t st) {
-    const int spans = (int)((K + kRqSpan - 1) / kRqSpan);
-    int tpc = 8 / spans;
-    if (tpc < 1) tpc = 1;
-    const int threads = spans * tpc * 32;
-    const int64_t grid = (M + tpc - 1) / tpc;
-    if (grid > 0x7FFFFFFFll) return DVDQ_ERR_SHAPE;
     int log2b = 0;
     while ((1 << log2b) < rot_block) ++log2b;
-#define DVDQ_RQ_CASE(L)                                                                                   \
-    case L:                                                                                               \
-        rq_natural_kernel<L, BITS><<<(unsigned)grid, threads, 0, st>>>(                                   \
-            (const __nv_bfloat16*)X, M, (int)K, ldx, (uint8_t*)codes, scales, sums, spans, tpc);          \
-        break;
+    const bool full = K % kRqSpan == 0;
+#define DVDQ_RQ_CASE(L)                                                                              \
+    case L:                                                                                          \
+        return full ? launch_rq_kernel<L, BITS, true>(X, M, K, ldx, codes, scales, sums, st)         \
+                    : launch_rq_kernel<L, BITS, false>(X, M, K, ldx, codes, scales, sums, st);
     switch (log2b) {
         DVDQ_RQ_CASE(0)
         DVDQ_RQ_CASE(6)
@@ -170,7 +388,6 @@ static dvdq_status launch_rq_bits(const void* X, int64_t M, int64_t K, int64_t l
             return DVDQ_ERR_ROT_BLOCK;
     }
 #undef DVDQ_RQ_CASE
-    return cuda_status(cudaGetLastError());
 }
 
 inline dvdq_status launch_rotate_quantize(const void* X, int64_t M, int64_t K, int64_t ldx, const dvdq_act_quant& q,

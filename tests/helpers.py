@@ -69,3 +69,19 @@ def check_codes_against_oracle(nat_gpu: np.ndarray, codes_or: np.ndarray, xt: np
         mid = (nat_gpu[i, k].astype(np.float64) + codes_or[i, k]) / 2.0
         assert np.abs(ratio - mid).max() < 1e-4, np.abs(ratio - mid).max()
     return frac
+
+
+def oracle_y_for_validated_codes(nat_gpu: np.ndarray, out: dict, u, d, z, bias_bits=None, act: int = 0) -> np.ndarray:
+    """bf16 values the oracle gives for the layer output when its quantizer takes the GPU's side
+    on rounding ties.  A code whose x~/s sits on a half-way point has two correct values (fp32
+    and fp64 transforms land on different sides of it), and one flipped code moves a whole output
+    row by s_i * Delta_n * (u - z): on a token with a large scale that alone can exceed the
+    output tolerance.  So the codes are first validated (equal, or +-1 on a tie: see
+    check_codes_against_oracle), and the rest of the path -- integer GEMM and epilogue, where
+    nothing is ambiguous -- is then evaluated by the oracle on the validated codes."""
+    from oracle import dvdq_oracle as orc
+    check_codes_against_oracle(nat_gpu, out["codes"], out["xt"], out["scale64"])
+    if np.array_equal(nat_gpu.astype(np.int32), out["codes"]):
+        return bf16_values(out["y"])
+    acc = orc.int_gemm(nat_gpu.astype(np.int32), u, z)
+    return bf16_values(orc.epilogue(acc, out["scale32"], d, bias_bits, act))

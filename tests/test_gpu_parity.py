@@ -5,7 +5,8 @@ seeded inputs.  Bars (written here once):
   * scales: 1e-6 relative;
   * codes: equal on >= 99.99 % of the elements, every mismatch +-1 on a rounding tie;
   * bf16 outputs: 4e-3 relative in max-norm (and <= 1 bf16 ulp elementwise when the GEMM is
-    fed the oracle's own codes and scales).
+    fed the oracle's own codes and scales).  Whole-layer comparisons validate the codes first
+    and let the oracle take the GPU's side on rounding ties (oracle_y_for_validated_codes).
 """
 import ctypes as C
 
@@ -18,7 +19,7 @@ from paper_2505_18663_b200 import binding as B
 from paper_2505_18663_b200 import workloads as W
 
 from helpers import (act_quant, bf16_values, check_codes_against_oracle, from_bits, gpu_pack_codes,
-                     gpu_pack_weights, gpu_rotate_quantize, to_bits)
+                     gpu_pack_weights, gpu_rotate_quantize, oracle_y_for_validated_codes, to_bits)
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -240,22 +241,27 @@ def test_bf16_output_on_oracle_codes_and_scales(M, N, K, Bk, bits, mode, act):
 # ------------------------------------------------------------------ the whole layer
 
 def run_qlinear(x_dev, w, bits, Bk, bias_dev, act, N):
+    """dvdq_qlinear; returns (Y, natural-order codes read back from the head of the workspace)."""
     M, K = x_dev.shape
     q = act_quant(bits, Bk)
     ws = torch.empty(B.dvdq_qlinear_workspace_bytes(M, K, q), dtype=torch.uint8, device=DEV)
     Y = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
     B.dvdq_qlinear(x_dev, q, w, bias_dev, act, Y, ws)
-    return Y
+    nat = torch.empty(M, K, dtype=torch.int8, device=DEV)
+    B.dvdq_unpack_act_codes(ws, M, K, q, nat)
+    return Y, nat.cpu().numpy()
 
 
 @pytest.mark.parametrize("M,N,K,Bk,bits,mode", [GEMM_CASES[0], GEMM_CASES[3], GEMM_CASES[4]])
 def test_qlinear_matches_oracle_end_to_end(M, N, K, Bk, bits, mode):
     x, u, d, z, codes, s64, s32, xt = oracle_layer(M, N, K, Bk, bits, mode, seed=7 * M + N)
-    y_or = bf16_values(orc.epilogue(orc.int_gemm(codes, u, z), s32, d, None, 0))
+    out = {"codes": codes, "xt": xt, "scale64": s64, "scale32": s32,
+           "y": orc.epilogue(orc.int_gemm(codes, u, z), s32, d, None, 0)}
     w, blob = gpu_pack_weights(u, d, z, Bk)
-    Y = run_qlinear(x.to(DEV), w, bits, Bk, None, 0, N)
+    Y, nat = run_qlinear(x.to(DEV), w, bits, Bk, None, 0, N)
     assert_device_ok()
     y = Y.to(torch.float64).cpu().numpy()
+    y_or = oracle_y_for_validated_codes(nat, out, u, d, z)
     assert np.abs(y - y_or).max() <= Y_MAXNORM_RTOL * np.abs(y_or).max()
 
 
@@ -271,9 +277,9 @@ def test_tiny_config_full_comparison():
     _, scales, _, nat = gpu_rotate_quantize(x.to(DEV), layer.bits, layer.rot_block)
     assert np.abs(scales.cpu().numpy().astype(np.float64) / out["scale64"] - 1).max() <= SCALE_RTOL
     check_codes_against_oracle(nat.cpu().numpy(), out["codes"], out["xt"], out["scale64"])
-    Y = run_qlinear(x.to(DEV), w, layer.bits, layer.rot_block, None, 0, layer.N)
+    Y, nat_q = run_qlinear(x.to(DEV), w, layer.bits, layer.rot_block, None, 0, layer.N)
     assert_device_ok()
-    y, y_or = Y.to(torch.float64).cpu().numpy(), bf16_values(out["y"])
+    y, y_or = Y.to(torch.float64).cpu().numpy(), oracle_y_for_validated_codes(nat_q, out, u, d, z)
     assert np.abs(y - y_or).max() <= Y_MAXNORM_RTOL * np.abs(y_or).max()
     exact = x.to(torch.float64).numpy() @ wb.to(torch.float64).numpy().T
     rel = np.linalg.norm(y - exact) / np.linalg.norm(exact)
@@ -295,14 +301,14 @@ def test_ffn_chain_stage_by_stage():
     u2, d2, z2 = orc.prepare_weights(to_bits(w2), down.rot_block)
     h1, blob1 = gpu_pack_weights(u1, d1, z1, up.rot_block)
     h2, blob2 = gpu_pack_weights(u2, d2, z2, down.rot_block)
-    Y1 = run_qlinear(x.to(DEV), h1, up.bits, up.rot_block, None, up.act, up.N)
-    Y2 = run_qlinear(Y1, h2, down.bits, down.rot_block, bias.to(DEV), down.act, down.N)
+    Y1, nat1 = run_qlinear(x.to(DEV), h1, up.bits, up.rot_block, None, up.act, up.N)
+    Y2, nat2 = run_qlinear(Y1, h2, down.bits, down.rot_block, bias.to(DEV), down.act, down.N)
     assert_device_ok()
     o1 = orc.qlinear(to_bits(x), u1, d1, z1, up.rot_block, up.bits, None, up.act)
-    y1, y1_or = Y1.to(torch.float64).cpu().numpy(), bf16_values(o1["y"])
+    y1, y1_or = Y1.to(torch.float64).cpu().numpy(), oracle_y_for_validated_codes(nat1, o1, u1, d1, z1, None, up.act)
     assert np.abs(y1 - y1_or).max() <= Y_MAXNORM_RTOL * np.abs(y1_or).max()
     o2 = orc.qlinear(to_bits(Y1), u2, d2, z2, down.rot_block, down.bits, to_bits(bias), down.act)
-    y2, y2_or = Y2.to(torch.float64).cpu().numpy(), bf16_values(o2["y"])
+    y2, y2_or = Y2.to(torch.float64).cpu().numpy(), oracle_y_for_validated_codes(nat2, o2, u2, d2, z2, to_bits(bias), down.act)
     assert np.abs(y2 - y2_or).max() <= Y_MAXNORM_RTOL * np.abs(y2_or).max()
 
 
@@ -332,9 +338,8 @@ def test_full_size_hunyuan_layer_on_sampled_rows(layer_idx):
     nat = torch.empty(M, layer.K, dtype=torch.int8, device=DEV)
     B.dvdq_unpack_act_codes(ws, M, layer.K, q, nat)
     nat_s = nat[rows.to(DEV)].cpu().numpy()
-    check_codes_against_oracle(nat_s, out["codes"], out["xt"], out["scale64"])
     y = Y[rows.to(DEV)].to(torch.float64).cpu().numpy()
-    y_or = bf16_values(out["y"])
+    y_or = oracle_y_for_validated_codes(nat_s, out, u.cpu().numpy(), d.cpu().numpy(), z.cpu().numpy())
     assert np.abs(y - y_or).max() <= Y_MAXNORM_RTOL * np.abs(y_or).max()
     # a property that holds at any size: no NaN/Inf anywhere in the full output
     assert bool(torch.isfinite(Y).all())
