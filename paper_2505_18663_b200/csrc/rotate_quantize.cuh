@@ -11,7 +11,8 @@
 //            A operand is the +-1 matrix H_16, so D = H_16 * B holds the four butterflies.
 //            bf16 inputs and +-1 factors make every product exact; the sums accumulate in fp32.
 //            The MMA also moves data: afterwards a lane holds bits {1,2,5,8,9} in registers.
-//   stage B  bits {2,8,9} as packed f32x2 adds/subs on register pairs, bit 5 as scalar add/sub.
+//   stage B  bit 2 through the accumulator input of further MMAs (H*B0 +- H*B1), bits {8,9} as
+//            packed f32x2 adds/subs on register pairs, bit 5 as scalar add/sub.
 //   turn     one conflict-free transposition through shared memory (8 x 16-byte stores and loads
 //            per lane) brings bits {6,7} and {0,1,2} into registers.
 //   stage C  bits {6,7} as packed f32x2 adds/subs.
@@ -63,13 +64,13 @@ __device__ __forceinline__ void f2_butterfly(uint64_t& a, uint64_t& b) {
     b = d;
 }
 
-// D = A * B with A 16x16 (row major), B 16x8 (column major), bf16 inputs, fp32 result, C = 0.
-__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
-    asm(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-        "{%10, %10, %10, %10};"
+// D = A * B + C with A 16x16 (row major), B 16x8 (column major), bf16 inputs, fp32 C and D.
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1,
+                                               const float (&c)[4]) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%10, %11, %12, %13};"
         : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.0f));
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(c[0]), "f"(c[1]), "f"(c[2]), "f"(c[3]));
 }
 
 // Entry (m, s) of the stage-A matrix as bf16 bits: the Sylvester sign (-1)^popcount(m & s), or the
@@ -106,6 +107,13 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
     afrag[1] = stage_a_entry<kRot>(g + 8, 2 * t) | (stage_a_entry<kRot>(g + 8, 2 * t + 1) << 16);
     afrag[2] = stage_a_entry<kRot>(g, 2 * t + 8) | (stage_a_entry<kRot>(g, 2 * t + 9) << 16);
     afrag[3] = stage_a_entry<kRot>(g + 8, 2 * t + 8) | (stage_a_entry<kRot>(g + 8, 2 * t + 9) << 16);
+    uint32_t afrag_neg[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) afrag_neg[i] = afrag[i] ^ 0x80008000u;
+    // a zero accumulator the compiler cannot fold, so that it stays in four registers
+    float zero4[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) asm volatile("mov.f32 %0, 0f00000000;" : "=f"(zero4[i]));
     // channel of the lane's first load chunk and of its first output word
     const int ld_e0 = sp * kRqSpan + lane * 8;                                   // + c * 256
     const int st_e0 = sp * kRqSpan + ((lane >> 3) * 32 + (lane & 7)) * 8;        // + j * 64
@@ -150,23 +158,34 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
     uint32_t it = 0;
     for (; group < num_groups; group += gridDim.x, ++it) {
         const uint32_t buf = it & 1u;
-        const int64_t token = (int64_t)group * tokens_per_cta + tl;
-        const bool tok_ok = token < M;
+        // A token past the end is a clamped duplicate of the last one: it computes and stores
+        // the same bytes to the same places, which needs no predicate.
+        int64_t token = (int64_t)group * tokens_per_cta + tl;
+        if (token >= M) token = M - 1;
 
         // ---- stage A: D = H_16 * B on index bits {0, 3, 4, 1} (k-slot bit 0 = half of a word,
         // bits 1-2 = lane & 3, bit 3 = which of the two words).  Word pair p = bit 2.
         // acc[c][p][r]: c = bits 9:8, p = bit 2, r & 1 = bit 5, r >> 1 = bit 1.
         // The lane now stands for bits 7:6 (lane & 3), bit 0 (lane >> 2 & 1), bits 4:3 (lane >> 3).
+        // With a rotation the butterfly on bit 2 rides on the accumulator input:
+        // acc[c][0] = H*B0 + H*B1, acc[c][1] = H*B0 - H*B1 (three MMAs instead of two MMAs and adds).
         float acc[4][2][4];
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            mma_bf16_16816(acc[c][0], afrag, raw[c].x, raw[c].y);
-            mma_bf16_16816(acc[c][1], afrag, raw[c].z, raw[c].w);
+            if (kRot) {
+                float m0[4];
+                mma_bf16_16816(m0, afrag, raw[c].x, raw[c].y, zero4);
+                mma_bf16_16816(acc[c][0], afrag, raw[c].z, raw[c].w, m0);
+                mma_bf16_16816(acc[c][1], afrag_neg, raw[c].z, raw[c].w, m0);
+            } else {
+                mma_bf16_16816(acc[c][0], afrag, raw[c].x, raw[c].y, zero4);
+                mma_bf16_16816(acc[c][1], afrag, raw[c].z, raw[c].w, zero4);
+            }
         }
         // the next group's loads fly while this one is transformed
         if (group + (int)gridDim.x < num_groups) load_span(raw, group + gridDim.x);
 
-        // ---- stage B: bits 2, 8, 9 on packed pairs (the pair is bit 5), then bit 5 itself
+        // ---- stage B: bits 8, 9 on packed pairs (the pair is bit 5), then bit 5 itself
         uint64_t P[4][2][2];
 #pragma unroll
         for (int c = 0; c < 4; ++c)
@@ -174,12 +193,6 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
             for (int p = 0; p < 2; ++p)
 #pragma unroll
                 for (int h = 0; h < 2; ++h) P[c][p][h] = f2_pack(acc[c][p][2 * h], acc[c][p][2 * h + 1]);
-        if (kRot) {
-#pragma unroll
-            for (int c = 0; c < 4; ++c)
-#pragma unroll
-                for (int h = 0; h < 2; ++h) f2_butterfly(P[c][0][h], P[c][1][h]);
-        }
         if (LOG2B > 8) {
 #pragma unroll
             for (int c = 0; c < 4; c += 2)
@@ -246,56 +259,61 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
                     for (int h = 0; h < 2; ++h) f2_butterfly(W[j][i0][h], W[j + 2][i0][h]);
         }
 
-        // val[j][e]: channel (lane >> 3) * 256 + j * 64 + (lane & 7) * 8 + e of the span,
-        // e = i0 + 2 * bit1 + 4 * h
-        float val[4][8];
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-#pragma unroll
-            for (int i0 = 0; i0 < 2; ++i0)
-#pragma unroll
-                for (int h = 0; h < 2; ++h) f2_unpack(W[j][i0][h], val[j][i0 + 4 * h], val[j][i0 + 4 * h + 2]);
-
+        // W[j][i0][h] = channels e and e + 2 of word j, e = i0 + 4 * h; the word covers channels
+        // (lane >> 3) * 256 + j * 64 + (lane & 7) * 8 + 0..7 of the span
         // ---- per-token absmax (of the un-normalised transform)
         float amax = 0.f;
 #pragma unroll
         for (int j = 0; j < 4; ++j)
 #pragma unroll
-            for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(val[j][e]));
+            for (int i0 = 0; i0 < 2; ++i0)
 #pragma unroll
-        for (int m = 16; m > 0; m >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, m));
+                for (int h = 0; h < 2; ++h) {
+                    float lo, hi;
+                    f2_unpack(W[j][i0][h], lo, hi);
+                    amax = fmaxf(amax, fmaxf(fabsf(lo), fabsf(hi)));
+                }
+        // non-negative floats order like their bit patterns: one REDUX instead of five shuffles
+        amax = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(amax)));
         if (lane == 0) s_max[buf][warp] = amax;
         __syncthreads();
-        if (spans > 1) {
-            amax = 0.f;
-            for (int s = 0; s < spans; ++s) amax = fmaxf(amax, s_max[buf][tl * spans + s]);
-        }
+        if (spans > 1)
+            amax = __uint_as_float(__reduce_max_sync(
+                0xFFFFFFFFu, lane < spans ? __float_as_uint(s_max[buf][tl * spans + lane]) : 0u));
         // the previous iteration's token: all its code sums are in shared memory by now
-        if (sp == 0 && lane == 0 && prev_token >= 0) {
-            int tsum = 0;
-            for (int s = 0; s < spans; ++s) tsum += s_sum[buf ^ 1u][tl * spans + s];
-            scales[prev_token] = (prev_amax * rs) / qmax;  // s_i = (absmax / sqrt(B)) / qmax
-            sums[prev_token] = tsum;
+        if (sp == 0 && prev_token >= 0) {
+            const int tsum = __reduce_add_sync(0xFFFFFFFFu, lane < spans ? s_sum[buf ^ 1u][tl * spans + lane] : 0);
+            if (lane == 0) {
+                scales[prev_token] = (prev_amax * rs) / qmax;  // s_i = (absmax / sqrt(B)) / qmax
+                sums[prev_token] = tsum;
+            }
         }
         const float inv = amax > 0.f ? qmax / amax : 0.f;
+        const uint64_t inv2 = f2_pack(inv, inv), magic2 = f2_pack(kMagic, kMagic);
 
         // ---- quantize, sum, pack, store
-        uint8_t* crow = codes + (tok_ok ? token : 0) * row_bytes;
+        uint8_t* crow = codes + token * row_bytes;
         int lsum = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t b[8];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                if (kRot) {
-                    b[e] = __float_as_uint(fmaf(val[j][e], inv, kMagic));
-                } else {
-                    // Without a rotation x~ is a bf16 value, x~ * qmax is exact and exact half-way
-                    // quotients are common: take the correctly rounded quotient so that they survive.
-                    const float quo = amax > 0.f ? __fdiv_rn(val[j][e] * qmax, amax) : 0.f;
-                    b[e] = __float_as_uint(quo + kMagic);
+            for (int i0 = 0; i0 < 2; ++i0)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    float lo, hi;
+                    if (kRot) {
+                        f2_unpack(f2_fma(W[j][i0][h], inv2, magic2), lo, hi);
+                    } else {
+                        // Without a rotation x~ is a bf16 value, x~ * qmax is exact and exact half-way
+                        // quotients are common: take the correctly rounded quotient so that they survive.
+                        f2_unpack(W[j][i0][h], lo, hi);
+                        lo = (amax > 0.f ? __fdiv_rn(lo * qmax, amax) : 0.f) + kMagic;
+                        hi = (amax > 0.f ? __fdiv_rn(hi * qmax, amax) : 0.f) + kMagic;
+                    }
+                    b[i0 + 4 * h] = __float_as_uint(lo);
+                    b[i0 + 4 * h + 2] = __float_as_uint(hi);
                 }
-            }
             // low bytes (= the codes as int8) of the even and of the odd channels
             const uint32_t E = __byte_perm(__byte_perm(b[0], b[2], 0x0040), __byte_perm(b[4], b[6], 0x0040), 0x5410);
             const uint32_t O = __byte_perm(__byte_perm(b[1], b[3], 0x0040), __byte_perm(b[5], b[7], 0x0040), 0x5410);
@@ -303,7 +321,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
             lsum = __dp4a((int)O, 0x01010101, lsum);
             const uint32_t lo = (E & 0x0F0F0F0Fu) | ((O << 4) & 0xF0F0F0F0u);
             const int e0 = st_e0 + j * 64;
-            const bool ok = tok_ok && (FULL || (st_ok >> j & 1u));
+            const bool ok = FULL || (st_ok >> j & 1u);
             if (ok) *reinterpret_cast<uint32_t*>(crow + (e0 >> 1)) = lo;
             if (BITS == 6) {
                 // bits 5:4 of 16 consecutive channels share one word of the high plane; the two
@@ -314,19 +332,19 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
                 if (ok && ((j ^ lane) & 1) == 0) *reinterpret_cast<uint32_t*>(crow + (K >> 1) + ((e0 >> 4) << 2)) = hi;
             }
         }
-#pragma unroll
-        for (int m = 16; m > 0; m >>= 1) lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, m);
+        lsum = __reduce_add_sync(0xFFFFFFFFu, lsum);
         if (lane == 0) s_sum[buf][warp] = lsum;
-        prev_token = tok_ok ? token : -1;
+        prev_token = token;
         prev_amax = amax;
     }
     __syncthreads();
-    if (sp == 0 && lane == 0 && prev_token >= 0) {
+    if (sp == 0 && prev_token >= 0) {
         const uint32_t buf = (it & 1u) ^ 1u;  // the last iteration's slots
-        int tsum = 0;
-        for (int s = 0; s < spans; ++s) tsum += s_sum[buf][tl * spans + s];
-        scales[prev_token] = (prev_amax * rs) / qmax;
-        sums[prev_token] = tsum;
+        const int tsum = __reduce_add_sync(0xFFFFFFFFu, lane < spans ? s_sum[buf][tl * spans + lane] : 0);
+        if (lane == 0) {
+            scales[prev_token] = (prev_amax * rs) / qmax;
+            sums[prev_token] = tsum;
+        }
     }
 }
 
