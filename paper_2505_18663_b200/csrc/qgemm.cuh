@@ -2,59 +2,76 @@
 //
 //   acc_in = sum_k c_ik (u_nk - z_n),   y_in = bf16(acc_in * s_i * Delta_n + bias_n)
 //
-// Persistent, warp-specialised sm_100a kernel, one CTA per SM, output tile 128 tokens x 256
-// channels, K consumed in blocks of 128 codes:
+// Persistent, warp-specialised sm_100a kernel for CTA PAIRS (cluster of two, one CTA per SM).
+// A pair owns an output tile of 256 tokens x 192 channels and issues tcgen05.mma with
+// cta_group::2: each CTA holds 128 token rows of the activation operand and 96 of the 192 weight
+// rows, so each CTA unpacks only half of the weight tile.  K is consumed in blocks of 128 codes.
+// The limiter of this kernel is shared-memory bandwidth (TMA writes, the unpack warps' reads and
+// writes, the tensor core's operand reads), which is why
+//   * the widened ACTIVATION operand never touches shared memory: the unpack warps write it to
+//     tensor memory with tcgen05.st and the MMA takes A from there;
+//   * the pair splits the weight tile.
 //
-//   warp 0      TMA producer: packed 4/6-bit activation rows and packed 4-bit weight rows
-//               -> shared memory ring (kPackedStages deep), completion on mbarriers.
-//   warps 6-13  widen the codes to int8 in shared memory, straight into the 128-byte-swizzled
-//               K-major layout tcgen05.mma reads.  A 4-bit two's-complement nibble masked into
-//               the HIGH half of a byte is the int8 value 16*code, a 6-bit code shifted to the
-//               top of a byte is 4*code; the factor (256 or 64 per product) is an exact shift
-//               of the int32 accumulator in the epilogue.  Weights are stored as (u - 8); the
-//               rest of the zero point, -(z_n - 8) * sum_k c_ik, is a rank-1 integer correction
-//               in the epilogue, so the mainloop never subtracts per-row constants.
-//   warp 1      one thread issues tcgen05.mma kind::i8 (128x256x32 per instruction) into one of
-//               two 256-column int32 accumulators in tensor memory; tcgen05.commit frees the
-//               widened stage and publishes the finished accumulator.
-//   warps 2-5   epilogue: tcgen05.ld, shift, zero-point correction, scale, bias, optional
-//               tanh-GELU, one bf16 rounding, 16-byte stores.  Runs concurrently with the next
-//               tile's mainloop thanks to the second accumulator.
+// Roles per CTA (14 warps):
+//   warp 0      TMA producer: packed 4/6-bit activation rows (this CTA's 128 tokens) and packed
+//               4-bit weight rows (this CTA's 96 channels) -> shared-memory ring.
+//   warps 6-9   widen activation codes to int8 and store them to tensor memory (one thread per
+//               token row; warp w may touch tensor-memory lanes 32*(w%4)..+31).
+//   warps 10-13 widen weight codes to int8 into the 128-byte-swizzled K-major layout in shared memory.
+//               A 4-bit two's-complement nibble masked into the HIGH half of a byte is the int8
+//               value 16*code, a 6-bit code shifted to the top of a byte is 4*code; the factor
+//               (256 or 64 per product) is an exact shift of the int32 accumulator in the
+//               epilogue.  Weights are stored as (u - 8); the rest of the zero point,
+//               -(z_n - 8) * sum_k c_ik, is a rank-1 integer correction in the epilogue.
+//   warp 1      (leader CTA only) one thread issues tcgen05.mma.cta_group::2.kind::i8, 256x192x32
+//               per instruction, into one of two 192-column int32 accumulators per CTA;
+//               tcgen05.commit signals "stage free" / "accumulator full" to both CTAs.
+//   warps 2-5   epilogue of this CTA's 128 rows: tcgen05.ld, shift, zero-point correction, scale,
+//               bias, optional tanh-GELU, one bf16 rounding, TMA stores.  Overlaps the next
+//               tile's mainloop through the second accumulator.
 //
-// Every wait is bounded (see mbar_wait); a role that gives up raises a shared abort flag and
-// all roles walk to the common exit, where tensor memory is released.
+// Tensor memory (512 columns per CTA): [0,192) and [192,384) accumulators, [384,512) four
+// activation stages of 32 columns (128 int8 per row).
+//
+// Every wait is bounded (see mbar_wait); a role that gives up raises its CTA's abort flag and
+// all roles walk to the common exit, where the pair synchronises and tensor memory is released.
 #pragma once
 
 #include "dvdq_common.cuh"
 
 namespace dvdq {
 
-constexpr int kBM = 128, kBN = 256, kBK = 128;
-constexpr int kWideStages = 2;
-constexpr int kUnpackWarps = 8, kEpilogueWarps = 4;
-constexpr int kFirstEpilogueWarp = 2, kFirstUnpackWarp = 6;
-constexpr int kGemmThreads = (2 + kEpilogueWarps + kUnpackWarps) * 32;
+constexpr int kBM = 128;            // token rows per CTA (the pair's tile has 2 * kBM)
+constexpr int kBN = 192;            // channels of the pair's tile
+constexpr int kBNh = kBN / 2;       // weight rows widened by each CTA
+constexpr int kBK = 128;
+constexpr int kPackedStages = 4, kWideStages = 4;
+constexpr int kAWarps = 4, kWWarps = 4, kEpilogueWarps = 4;
+constexpr int kFirstEpilogueWarp = 2, kFirstAWarp = 6, kFirstWWarp = 10;
+constexpr int kGemmThreads = (2 + kEpilogueWarps + kAWarps + kWWarps) * 32;
 constexpr int kTmemCols = 512;
+constexpr int kTmemACol = 2 * kBN;  // first column of the activation stages
+constexpr int kAColsPerStage = kBK / 4;
+static_assert(kTmemACol + kWideStages * kAColsPerStage <= kTmemCols, "tensor memory budget");
 
 template <int BITS>
 struct GemmSmem {
-    static constexpr int kPackedStages = (BITS == 4) ? 4 : 3;     // what fits beside the other buffers
-    static constexpr int kALo = kBM * kBK / 2;                    // packed low plane / A4 codes
-    static constexpr int kAHi = (BITS == 6) ? kBM * kBK / 4 : 0;  // packed high plane
-    static constexpr int kW = kBN * kBK / 2;
+    static constexpr int kWideW = kBNh * kBK;                     // int8 weight half-tile, swizzled
+    static constexpr int kWideOff = 0;                            // 1024-byte aligned tiles first
+    static constexpr int kALo = kBM * kBK / 2;                    // packed low plane / A4 codes (64-byte rows)
+    static constexpr int kAHi = (BITS == 6) ? kBM * kBK / 4 : 0;  // packed high plane (32-byte rows)
+    static constexpr int kW = kBNh * kBK / 2;
     static constexpr int kPackedStage = kALo + kAHi + kW;
-    static constexpr int kWideA = kBM * kBK, kWideW = kBN * kBK;
-    static constexpr int kWideStage = kWideA + kWideW;
-    static constexpr int kWideOff = 0;  // 1024-byte aligned tiles first
-    static constexpr int kPackedOff = kWideOff + kWideStages * kWideStage;
+    static constexpr int kPackedOff = kWideOff + kWideStages * kWideW;
     static constexpr int kStageOutOff = kPackedOff + kPackedStages * kPackedStage;  // 1024-byte aligned
     static constexpr int kStageOutPerWarp = 2 * 32 * 64;  // two buffers of 32 rows x 32 bf16
     static constexpr int kConstOff = kStageOutOff + kEpilogueWarps * kStageOutPerWarp;
-    static constexpr int kConstPerWarp = 3 * kBN * 4;  // delta, zero-point rest, bias for 256 channels
+    static constexpr int kConstPerWarp = 3 * kBN * 4;  // delta, zero-point rest, bias
     static constexpr int kBarOff = kConstOff + kEpilogueWarps * kConstPerWarp;
-    static constexpr int kNumBars = 2 * kPackedStages + 2 * kWideStages + 4;
+    static constexpr int kNumBars = 2 * kPackedStages + 2 * kWideStages + 5;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kTotal = kMiscOff + 16 + 1024;  // + slack for manual 1024-byte alignment
+    static_assert(kWideW % 1024 == 0 && kPackedStage % 1024 == 0, "swizzled tiles need 1024-byte alignment");
 };
 
 __device__ __forceinline__ float gelu_tanh_f32(float y) {
@@ -63,7 +80,7 @@ __device__ __forceinline__ float gelu_tanh_f32(float y) {
 }
 
 template <int BITS, bool RAW>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmAhi,
              const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmY,
              const float* __restrict__ scales,
@@ -71,39 +88,45 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
              const __nv_bfloat16* __restrict__ bias, __nv_bfloat16* __restrict__ Y, int64_t ldy,
              int32_t* __restrict__ acc_out, int64_t ldacc, int M, int N, int K, int act) {
     using S = GemmSmem<BITS>;
-    constexpr int kPackedStages = S::kPackedStages;
     extern __shared__ uint8_t smem_raw[];
+    // identical in both CTAs of the pair: the dynamic shared window starts at the same offset
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_n = (N + kBN - 1) / kBN, num_m = (M + kBM - 1) / kBM;
+    const uint32_t rank = cluster_ctarank();       // 0 = leader of the pair
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int num_n = (N + kBN - 1) / kBN, num_m = (M + 2 * kBM - 1) / (2 * kBM);
     const int num_tiles = num_m * num_n;
     const int KB = (K + kBK - 1) / kBK;
 
     const uint32_t bar0 = sbase + S::kBarOff;
     auto pk_full = [&](int s) { return bar0 + 8u * s; };
     auto pk_empty = [&](int s) { return bar0 + 8u * (kPackedStages + s); };
-    auto wd_full = [&](int s) { return bar0 + 8u * (2 * kPackedStages + s); };
-    auto wd_empty = [&](int s) { return bar0 + 8u * (2 * kPackedStages + kWideStages + s); };
-    auto acc_full = [&](int s) { return bar0 + 8u * (2 * kPackedStages + 2 * kWideStages + s); };
-    auto acc_empty = [&](int s) { return bar0 + 8u * (2 * kPackedStages + 2 * kWideStages + 2 + s); };
+    auto wd_full = [&](int s) { return bar0 + 8u * (2 * kPackedStages + s); };                  // leader's copy is used
+    auto wd_empty = [&](int s) { return bar0 + 8u * (2 * kPackedStages + kWideStages + s); };   // one per CTA
+    auto acc_full = [&](int s) { return bar0 + 8u * (2 * kPackedStages + 2 * kWideStages + s); };      // one per CTA
+    auto acc_empty = [&](int s) { return bar0 + 8u * (2 * kPackedStages + 2 * kWideStages + 2 + s); }; // leader's copy
+    const uint32_t drain_bar = bar0 + 8u * (2 * kPackedStages + 2 * kWideStages + 4);
     volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + S::kMiscOff);  // [0] tmem base, [1] abort
     volatile uint32_t* abort_flag = misc + 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kPackedStages; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), kUnpackWarps); }
-        for (int s = 0; s < kWideStages; ++s) { mbar_init(wd_full(s), kUnpackWarps); mbar_init(wd_empty(s), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), kEpilogueWarps); }
+        for (int s = 0; s < kPackedStages; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), kAWarps + kWWarps); }
+        for (int s = 0; s < kWideStages; ++s) { mbar_init(wd_full(s), 2 * (kAWarps + kWWarps)); mbar_init(wd_empty(s), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * kEpilogueWarps); }
+        mbar_init(drain_bar, 1);
         misc[1] = 0u;
         fence_mbar_init();
     }
     if (warp == 1) {
+        // each CTA allocates all of its own tensor memory, so both allocations start at column 0
         tmem_alloc(sbase + S::kMiscOff, kTmemCols);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();  // the peer's barriers are initialised before anyone arrives on them
     tc_fence_after();
     const uint32_t tmem_base = misc[0];
 
@@ -115,8 +138,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             tma_prefetch_desc(&tmW);
             uint32_t st = 0, ph = 0, issued = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
-                const int m0 = (tile / num_n) * kBM, n0 = (tile % num_n) * kBN;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
+                const int n0 = (tile % num_n) * kBN + (int)rank * kBNh;
                 for (int kb = 0; kb < KB; ++kb) {
                     if (!mbar_wait(pk_empty(st), ph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
                     const uint32_t dst = sbase + S::kPackedOff + st * S::kPackedStage;
@@ -140,12 +164,12 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         }
         __syncwarp();
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_s8s8s32(kBM, kBN);
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (rank == 0 && lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_s8s8s32(2 * kBM, kBN);
             uint32_t st = 0, ph = 0, lt = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x, ++lt) {
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++lt) {
                 const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
                 if (!mbar_wait(acc_empty(a), aph ^ 1u, abort_flag, kWaitAccEmpty)) { ok = false; break; }
                 tc_fence_after();
@@ -153,20 +177,22 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 for (int kb = 0; kb < KB; ++kb) {
                     if (!mbar_wait(wd_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t wa = sbase + S::kWideOff + st * S::kWideStage;
-                    const uint64_t adesc = umma_desc_sw128_kmajor(wa);
-                    const uint64_t bdesc = umma_desc_sw128_kmajor(wa + S::kWideA);
+                    const uint32_t a_tmem = tmem_base + kTmemACol + st * kAColsPerStage;
+                    const uint64_t bdesc = umma_desc_sw128_kmajor(sbase + S::kWideOff + st * S::kWideW);
 #pragma unroll
-                    for (int k = 0; k < kBK / 32; ++k)  // +32 bytes along K = +2 in the 16-byte address field
-                        tc_mma_i8_ss(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                    tc_commit(wd_empty(st));
+                    for (int k = 0; k < kBK / 32; ++k)  // +32 int8 along K = +8 columns of A, +2 in B's 16-byte address field
+                        tc_mma_i8_ts_pair(d_tmem, a_tmem + 8u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    tc_commit_pair(wd_empty(st), 3);
                     if (++st == kWideStages) { st = 0; ph ^= 1u; }
                 }
-                if (ok) tc_commit(acc_full(a));
+                if (ok) tc_commit_pair(acc_full(a), 3);
             }
+            // nothing issued by this thread may still be running when the pair leaves
+            tc_commit_pair(drain_bar, 1);
+            mbar_wait(drain_bar, 0u, abort_flag, kWaitDrain);
         }
         __syncwarp();
-    } else if (warp < kFirstUnpackWarp) {
+    } else if (warp < kFirstAWarp) {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;  // tensor-memory lane quarter this warp may read
         const int ew = warp - kFirstEpilogueWarp;
@@ -178,9 +204,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         constexpr int kShift = (BITS == 4) ? 8 : 6;
         if (!RAW && lane == 0) tma_prefetch_desc(&tmY);
         uint32_t lt = 0, nstore = 0;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++lt) {
+        for (int tile = pair; tile < num_tiles; tile += num_pairs, ++lt) {
             const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
-            const int m0 = (tile / num_n) * kBM, n0 = (tile % num_n) * kBN;
+            const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM, n0 = (tile % num_n) * kBN;
             __syncwarp();
             for (int c = lane; c < kBN; c += 32) {
                 const int n = n0 + c;
@@ -263,53 +289,79 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty(a));
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty(a), 0));
         }
         if (!RAW && lane == 0) tma_store_wait_all();
         __syncwarp();
-    } else {
-        // ------------------------------------------------------------ widen 4/6-bit codes to int8
-        const int u = threadIdx.x - kFirstUnpackWarp * 32;  // 0..255
+    } else if (warp < kFirstWWarp) {
+        // ------------------------------------------------------------ widen activation codes -> tensor memory
+        const int q = warp & 3;
+        const int row = q * 32 + lane;                     // row of this CTA's tile = tensor-memory lane
+        const uint32_t sw_lo = (uint32_t)(row >> 1) & 3u;  // 64-byte-swizzled TMA tile: chunk ^= (row / 2) % 4
+        const uint32_t sw_hi = (uint32_t)(row >> 2) & 1u;  // 32-byte-swizzled TMA tile: chunk ^= (row / 4) % 2
+        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         uint32_t pst = 0, pph = 0, wst = 0, wph = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < num_tiles; tile += gridDim.x) {
+        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
             for (int kb = 0; kb < KB; ++kb) {
                 if (!mbar_wait(pk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
                 if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
                 tc_fence_after();
                 const uint8_t* pk = smem + S::kPackedOff + pst * S::kPackedStage;
-                uint8_t* wdA = smem + S::kWideOff + wst * S::kWideStage;
-                uint8_t* wdW = wdA + S::kWideA;
-                // activation tile: 128 rows x 4 chunks of 32 codes
+                const uint8_t* prow = pk + row * (kBK / 2);
+                uint32_t r[32];  // r[2i] / r[2i+1]: even / odd codes of packed word i, the K order the weights use too
+                uint32_t h[8];
+                if (BITS == 6) {
+                    const uint8_t* hrow = pk + S::kALo + row * (kBK / 4);
 #pragma unroll
-                for (int it = 0; it < (kBM * 4) / 256; ++it) {
-                    const int qi = it * 256 + u, row = qi >> 2, ck = qi & 3;
-                    const uint4 p = *reinterpret_cast<const uint4*>(pk + row * (kBK / 2) + ck * 16);
+                    for (int c = 0; c < 2; ++c) {
+                        const uint4 p = *reinterpret_cast<const uint4*>(hrow + (((uint32_t)c ^ sw_hi) << 4));
+                        h[4 * c] = p.x; h[4 * c + 1] = p.y; h[4 * c + 2] = p.z; h[4 * c + 3] = p.w;
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint4 p = *reinterpret_cast<const uint4*>(prow + (((uint32_t)c ^ sw_lo) << 4));
                     const uint32_t w[4] = {p.x, p.y, p.z, p.w};
-                    uint32_t e[4], o[4];
-                    if (BITS == 4) {
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) { e[j] = (w[j] << 4) & 0xF0F0F0F0u; o[j] = w[j] & 0xF0F0F0F0u; }
-                    } else {
-                        const uint2 hp = *reinterpret_cast<const uint2*>(pk + S::kALo + row * (kBK / 4) + ck * 8);
-                        const uint32_t h[2] = {hp.x, hp.y};
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t hh = h[j >> 1];
-                            const int a2 = 2 * (j & 1);
-                            e[j] = ((w[j] << 2) & 0x3C3C3C3Cu) | ((hh << (6 - 2 * a2)) & 0xC0C0C0C0u);
-                            o[j] = ((w[j] >> 2) & 0x3C3C3C3Cu) | ((hh << (4 - 2 * a2)) & 0xC0C0C0C0u);
+                    for (int j = 0; j < 4; ++j) {
+                        const int i = 4 * c + j;
+                        if (BITS == 4) {
+                            r[2 * i] = (w[j] << 4) & 0xF0F0F0F0u;
+                            r[2 * i + 1] = w[j] & 0xF0F0F0F0u;
+                        } else {
+                            const uint32_t hh = h[i >> 1];
+                            const int a2 = 2 * (i & 1);
+                            r[2 * i] = ((w[j] << 2) & 0x3C3C3C3Cu) | ((hh << (6 - 2 * a2)) & 0xC0C0C0C0u);
+                            r[2 * i + 1] = ((w[j] >> 2) & 0x3C3C3C3Cu) | ((hh << (4 - 2 * a2)) & 0xC0C0C0C0u);
                         }
                     }
-                    uint8_t* drow = wdA + (row >> 3) * 1024 + (row & 7) * 128;
-                    *reinterpret_cast<uint4*>(drow + (((2 * ck) ^ (row & 7)) << 4)) = make_uint4(e[0], o[0], e[1], o[1]);
-                    *reinterpret_cast<uint4*>(drow + (((2 * ck + 1) ^ (row & 7)) << 4)) = make_uint4(e[2], o[2], e[3], o[3]);
                 }
-                // weight tile: 256 rows x 4 chunks of 32 nibbles, stored as (u - 8)
-                const uint8_t* pw = pk + S::kALo + S::kAHi;
+                tmem_st_32x32(tmem_base + kTmemACol + wst * kAColsPerStage + lane_addr, r);
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) { mbar_arrive_cluster(map_to_cta(wd_full(wst), 0)); mbar_arrive(pk_empty(pst)); }
+                if (++pst == kPackedStages) { pst = 0; pph ^= 1u; }
+                if (++wst == kWideStages) { wst = 0; wph ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ widen weight codes -> shared memory
+        const int u = threadIdx.x - kFirstWWarp * 32;  // 0..127
+        uint32_t pst = 0, pph = 0, wst = 0, wph = 0;
+        bool ok = true;
+        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!mbar_wait(pk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                tc_fence_after();
+                const uint8_t* pw = smem + S::kPackedOff + pst * S::kPackedStage + S::kALo + S::kAHi;
+                uint8_t* wdW = smem + S::kWideOff + wst * S::kWideW;
+                // 96 rows x 4 chunks of 32 nibbles, stored as (u - 8)
 #pragma unroll
-                for (int it = 0; it < (kBN * 4) / 256; ++it) {
-                    const int qi = it * 256 + u, row = qi >> 2, ck = qi & 3;
+                for (int it = 0; it < (kBNh * 4) / (kWWarps * 32); ++it) {
+                    const int qi = it * (kWWarps * 32) + u, row = qi >> 2, ck = qi & 3;
                     const uint4 p = *reinterpret_cast<const uint4*>(pw + row * (kBK / 2) + ck * 16);
                     const uint32_t w[4] = {p.x, p.y, p.z, p.w};
                     uint32_t e[4], o[4];
@@ -321,7 +373,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) { mbar_arrive(wd_full(wst)); mbar_arrive(pk_empty(pst)); }
+                if (lane == 0) { mbar_arrive_cluster(map_to_cta(wd_full(wst), 0)); mbar_arrive(pk_empty(pst)); }
                 if (++pst == kPackedStages) { pst = 0; pph ^= 1u; }
                 if (++wst == kWideStages) { wst = 0; wph ^= 1u; }
             }
@@ -330,6 +382,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();  // the peer may read this CTA's shared and tensor memory until it is done too
     tc_fence_after();
     if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
 }
@@ -352,8 +405,6 @@ inline PFN_encodeTiled get_encode_tiled() {
     return fn;
 }
 
-// Byte matrix [rows, row_len] with row pitch `pitch`, tiles of box_rows x box_bytes, no swizzle,
-// out-of-range bytes read as zero.
 // bf16 matrix [rows, cols] with row pitch ld elements, tiles of 32 x 32, 64-byte swizzle
 // (the layout the epilogue stages its output in).
 inline bool make_out_map(CUtensorMap* tm, const void* base, uint64_t cols, uint64_t rows, uint64_t ld) {
@@ -368,8 +419,10 @@ inline bool make_out_map(CUtensorMap* tm, const void* base, uint64_t cols, uint6
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Byte matrix [rows, row_len] with row pitch `pitch`, tiles of box_rows x box_bytes with the given
+// swizzle (box_bytes equals the swizzle span, or no swizzle); out-of-range bytes read as zero.
 inline bool make_byte_map(CUtensorMap* tm, const void* base, uint64_t row_len, uint64_t rows, uint64_t pitch,
-                          uint32_t box_bytes, uint32_t box_rows) {
+                          uint32_t box_bytes, uint32_t box_rows, CUtensorMapSwizzle swizzle) {
     PFN_encodeTiled enc = get_encode_tiled();
     if (!enc) return false;
     const cuuint64_t dims[2] = {row_len, rows};
@@ -377,7 +430,7 @@ inline bool make_byte_map(CUtensorMap* tm, const void* base, uint64_t row_len, u
     const cuuint32_t box[2] = {box_bytes, box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -391,14 +444,18 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
     const uint64_t pitch = (uint64_t)act_row_bytes(K, BITS);
     CUtensorMap tmA, tmAhi, tmW, tmY;
-    if (!make_byte_map(&tmA, codes, (uint64_t)K / 2, (uint64_t)M, pitch, kBK / 2, kBM)) return DVDQ_ERR_CUDA;
+    if (!make_byte_map(&tmA, codes, (uint64_t)K / 2, (uint64_t)M, pitch, kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_64B))
+        return DVDQ_ERR_CUDA;
     if (BITS == 6) {
-        if (!make_byte_map(&tmAhi, static_cast<const uint8_t*>(codes) + K / 2, (uint64_t)K / 4, (uint64_t)M, pitch, kBK / 4, kBM))
+        if (!make_byte_map(&tmAhi, static_cast<const uint8_t*>(codes) + K / 2, (uint64_t)K / 4, (uint64_t)M, pitch,
+                           kBK / 4, kBM, CU_TENSOR_MAP_SWIZZLE_32B))
             return DVDQ_ERR_CUDA;
     } else {
         tmAhi = tmA;
     }
-    if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, kBN)) return DVDQ_ERR_CUDA;
+    if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, kBNh,
+                       CU_TENSOR_MAP_SWIZZLE_NONE))
+        return DVDQ_ERR_CUDA;
 
     if (RAW) {
         tmY = tmA;  // unused
@@ -406,25 +463,34 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
         return DVDQ_ERR_CUDA;
     }
 
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0;
+    auto kern = qgemm_kernel<BITS, RAW>;
+    static int max_pairs = 0;
+    if (max_pairs == 0) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) return DVDQ_ERR_CUDA;
+        int dev = 0, sm_count = 0;
         if (cudaGetDevice(&dev) != cudaSuccess) return DVDQ_ERR_CUDA;
         if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DVDQ_ERR_CUDA;
+        // how many CTA pairs the device can keep resident at once (one CTA per SM)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(sm_count & ~1), 1, 1);
+        cfg.blockDim = dim3(kGemmThreads, 1, 1);
+        cfg.dynamicSmemBytes = S::kTotal;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) != cudaSuccess || clusters < 1) return DVDQ_ERR_CUDA;
+        max_pairs = clusters < sm_count / 2 ? clusters : sm_count / 2;
     }
-    auto kern = qgemm_kernel<BITS, RAW>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) return DVDQ_ERR_CUDA;
-        attr_set = true;
-    }
-    const int64_t tiles = ((M + kBM - 1) / kBM) * ((N + kBN - 1) / kBN);
-    const unsigned grid = (unsigned)(tiles < sm_count ? tiles : sm_count);
-    kern<<<grid, kGemmThreads, S::kTotal, st>>>(tmA, tmAhi, tmW, tmY, scales, sums,
-                                                reinterpret_cast<const float*>(blob + L.delta_offset),
-                                                reinterpret_cast<const int32_t*>(blob + L.zc_offset),
-                                                static_cast<const __nv_bfloat16*>(bias), static_cast<__nv_bfloat16*>(Y), ldy,
-                                                acc_out, ldacc, (int)M, (int)N, (int)K, act);
+    const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + kBN - 1) / kBN);
+    const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
+    kern<<<2 * pairs, kGemmThreads, S::kTotal, st>>>(tmA, tmAhi, tmW, tmY, scales, sums,
+                                                     reinterpret_cast<const float*>(blob + L.delta_offset),
+                                                     reinterpret_cast<const int32_t*>(blob + L.zc_offset),
+                                                     static_cast<const __nv_bfloat16*>(bias), static_cast<__nv_bfloat16*>(Y), ldy,
+                                                     acc_out, ldacc, (int)M, (int)N, (int)K, act);
     return cuda_status(cudaGetLastError());
 }
 
