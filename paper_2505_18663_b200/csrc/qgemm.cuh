@@ -196,11 +196,10 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;  // tensor-memory lane quarter this warp may read
         const int ew = warp - kFirstEpilogueWarp;
-        float* c_delta = reinterpret_cast<float*>(smem + S::kConstOff + ew * S::kConstPerWarp);
-        float* c_zc = c_delta + kBN;    // (z_n - 8) as a float: exact, |.| <= 8
-        float* c_bias = c_zc + kBN;
+        const uint32_t c_delta = sbase + S::kConstOff + ew * S::kConstPerWarp;  // shared addresses of float[kBN] each
+        const uint32_t c_zc = c_delta + kBN * 4;    // (z_n - 8) as a float: exact, |.| <= 8
+        const uint32_t c_bias = c_zc + kBN * 4;
         const uint32_t stg0 = sbase + S::kStageOutOff + ew * S::kStageOutPerWarp;
-        uint8_t* stg_ptr = smem + S::kStageOutOff + ew * S::kStageOutPerWarp;
         constexpr int kShift = (BITS == 4) ? 8 : 6;
         if (!RAW && lane == 0) tma_prefetch_desc(&tmY);
         uint32_t lt = 0, nstore = 0;
@@ -211,9 +210,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             for (int c = lane; c < kBN; c += 32) {
                 const int n = n0 + c;
                 const bool okn = n < N;
-                c_delta[c] = okn ? delta[n] : 0.f;
-                c_zc[c] = okn ? (float)zc[n] : 0.f;
-                c_bias[c] = (okn && bias != nullptr) ? __bfloat162float(bias[n]) : 0.f;
+                sts32f(c_delta + 4 * c, okn ? delta[n] : 0.f);
+                sts32f(c_zc + 4 * c, okn ? (float)zc[n] : 0.f);
+                sts32f(c_bias + 4 * c, (okn && bias != nullptr) ? __bfloat162float(bias[n]) : 0.f);
             }
             __syncwarp();
             if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) break;
@@ -233,26 +232,24 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     int32_t* dst = acc_out + (int64_t)row * ldacc + nb;
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) {
+                        const float4 zq = lds128f(c_zc + 4 * (c * 32 + j));
                         int4 o;
-                        o.x = ((int32_t)r[j] >> kShift) - __float2int_rn(c_zc[c * 32 + j]) * S_i;
-                        o.y = ((int32_t)r[j + 1] >> kShift) - __float2int_rn(c_zc[c * 32 + j + 1]) * S_i;
-                        o.z = ((int32_t)r[j + 2] >> kShift) - __float2int_rn(c_zc[c * 32 + j + 2]) * S_i;
-                        o.w = ((int32_t)r[j + 3] >> kShift) - __float2int_rn(c_zc[c * 32 + j + 3]) * S_i;
+                        o.x = ((int32_t)r[j] >> kShift) - __float2int_rn(zq.x) * S_i;
+                        o.y = ((int32_t)r[j + 1] >> kShift) - __float2int_rn(zq.y) * S_i;
+                        o.z = ((int32_t)r[j + 2] >> kShift) - __float2int_rn(zq.z) * S_i;
+                        o.w = ((int32_t)r[j + 3] >> kShift) - __float2int_rn(zq.w) * S_i;
                         if (row_ok && nb + j < N) *reinterpret_cast<int4*>(dst + j) = o;
                     }
                 } else {
                     // The staging buffer used two chunks ago must have been read by its TMA store.
                     if (lane == 0) tma_store_wait_read<1>();
                     __syncwarp();
-                    uint8_t* buf = stg_ptr + (nstore & 1u) * (32 * 64);
+                    const uint32_t buf = stg0 + (nstore & 1u) * (32 * 64);
 #pragma unroll
                     for (int j = 0; j < 32; j += 8) {
-                        const float4 d0 = *reinterpret_cast<const float4*>(c_delta + c * 32 + j);
-                        const float4 d1 = *reinterpret_cast<const float4*>(c_delta + c * 32 + j + 4);
-                        const float4 z0 = *reinterpret_cast<const float4*>(c_zc + c * 32 + j);
-                        const float4 z1 = *reinterpret_cast<const float4*>(c_zc + c * 32 + j + 4);
-                        const float4 b0 = *reinterpret_cast<const float4*>(c_bias + c * 32 + j);
-                        const float4 b1 = *reinterpret_cast<const float4*>(c_bias + c * 32 + j + 4);
+                        const float4 d0 = lds128f(c_delta + 4 * (c * 32 + j)), d1 = lds128f(c_delta + 4 * (c * 32 + j + 4));
+                        const float4 z0 = lds128f(c_zc + 4 * (c * 32 + j)), z1 = lds128f(c_zc + 4 * (c * 32 + j + 4));
+                        const float4 b0 = lds128f(c_bias + 4 * (c * 32 + j)), b1 = lds128f(c_bias + 4 * (c * 32 + j + 4));
                         const float dl[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
                         const float zz[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
                         const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
@@ -276,7 +273,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                         // 64-byte rows, 16-byte chunk index XORed with (row >> 1) & 3: the layout a
                         // 64B-swizzled TMA store reads, and conflict-free for this per-row write.
                         const int ch = (j >> 3) ^ ((lane >> 1) & 3);
-                        *reinterpret_cast<uint4*>(buf + lane * 64 + ch * 16) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        sts128(buf + lane * 64 + ch * 16, pk[0], pk[1], pk[2], pk[3]);
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
@@ -307,21 +304,21 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 if (!mbar_wait(pk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
                 if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
                 tc_fence_after();
-                const uint8_t* pk = smem + S::kPackedOff + pst * S::kPackedStage;
-                const uint8_t* prow = pk + row * (kBK / 2);
+                const uint32_t pk = sbase + S::kPackedOff + pst * S::kPackedStage;
+                const uint32_t prow = pk + row * (kBK / 2);
                 uint32_t r[32];  // r[2i] / r[2i+1]: even / odd codes of packed word i, the K order the weights use too
                 uint32_t h[8];
                 if (BITS == 6) {
-                    const uint8_t* hrow = pk + S::kALo + row * (kBK / 4);
+                    const uint32_t hrow = pk + S::kALo + row * (kBK / 4);
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
-                        const uint4 p = *reinterpret_cast<const uint4*>(hrow + (((uint32_t)c ^ sw_hi) << 4));
+                        const uint4 p = lds128(hrow + (((uint32_t)c ^ sw_hi) << 4));
                         h[4 * c] = p.x; h[4 * c + 1] = p.y; h[4 * c + 2] = p.z; h[4 * c + 3] = p.w;
                     }
                 }
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const uint4 p = *reinterpret_cast<const uint4*>(prow + (((uint32_t)c ^ sw_lo) << 4));
+                    const uint4 p = lds128(prow + (((uint32_t)c ^ sw_lo) << 4));
                     const uint32_t w[4] = {p.x, p.y, p.z, p.w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -356,20 +353,20 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 if (!mbar_wait(pk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
                 if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
                 tc_fence_after();
-                const uint8_t* pw = smem + S::kPackedOff + pst * S::kPackedStage + S::kALo + S::kAHi;
-                uint8_t* wdW = smem + S::kWideOff + wst * S::kWideW;
+                const uint32_t pw = sbase + S::kPackedOff + pst * S::kPackedStage + S::kALo + S::kAHi;
+                const uint32_t wdW = sbase + S::kWideOff + wst * S::kWideW;
                 // 96 rows x 4 chunks of 32 nibbles, stored as (u - 8)
 #pragma unroll
                 for (int it = 0; it < (kBNh * 4) / (kWWarps * 32); ++it) {
                     const int qi = it * (kWWarps * 32) + u, row = qi >> 2, ck = qi & 3;
-                    const uint4 p = *reinterpret_cast<const uint4*>(pw + row * (kBK / 2) + ck * 16);
+                    const uint4 p = lds128(pw + row * (kBK / 2) + ck * 16);
                     const uint32_t w[4] = {p.x, p.y, p.z, p.w};
                     uint32_t e[4], o[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j) { e[j] = (w[j] << 4) & 0xF0F0F0F0u; o[j] = w[j] & 0xF0F0F0F0u; }
-                    uint8_t* drow = wdW + (row >> 3) * 1024 + (row & 7) * 128;
-                    *reinterpret_cast<uint4*>(drow + (((2 * ck) ^ (row & 7)) << 4)) = make_uint4(e[0], o[0], e[1], o[1]);
-                    *reinterpret_cast<uint4*>(drow + (((2 * ck + 1) ^ (row & 7)) << 4)) = make_uint4(e[2], o[2], e[3], o[3]);
+                    const uint32_t drow = wdW + (row >> 3) * 1024 + (row & 7) * 128;
+                    sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[0], o[0], e[1], o[1]);
+                    sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[2], o[2], e[3], o[3]);
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
