@@ -146,6 +146,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// mbar_wait by a fully converged warp with one answer for all lanes (a wait that gives up in some
+// lanes only must not split the warp before an elect.sync / __syncwarp).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t wait_id) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, wait_id);
+    return __all_sync(0xFFFFFFFFu, ok);
+}
+
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {
@@ -172,6 +179,18 @@ __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk
 template <int N>
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// True in exactly one lane of a fully converged warp.  Unlike `lane == 0`, the compiler knows the
+// enclosing control flow is warp-uniform, so descriptors and addresses stay in uniform registers.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "elect.sync _|p, 0xFFFFFFFF;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
 
 // ---- thread-block clusters (CTA pairs)
 __device__ __forceinline__ uint32_t cluster_ctarank() {

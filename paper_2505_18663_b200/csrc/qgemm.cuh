@@ -165,30 +165,36 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (rank == 0 && lane == 0) {
+        // The whole warp walks the loop (warp-uniform control flow); one elected lane issues.
+        if (rank == 0) {
             constexpr uint32_t idesc = umma_idesc_s8s8s32(2 * kBM, kBN);
             uint32_t st = 0, ph = 0, lt = 0;
             bool ok = true;
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++lt) {
                 const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
-                if (!mbar_wait(acc_empty(a), aph ^ 1u, abort_flag, kWaitAccEmpty)) { ok = false; break; }
+                if (!mbar_wait_warp(acc_empty(a), aph ^ 1u, abort_flag, kWaitAccEmpty)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + a * kBN;
                 for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_wait(wd_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
+                    if (!mbar_wait_warp(wd_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_tmem = tmem_base + kTmemACol + st * kAColsPerStage;
                     const uint64_t bdesc = umma_desc_sw128_kmajor(sbase + S::kWideOff + st * S::kWideW);
+                    if (elect_one()) {
 #pragma unroll
-                    for (int k = 0; k < kBK / 32; ++k)  // +32 int8 along K = +8 columns of A, +2 in B's 16-byte address field
-                        tc_mma_i8_ts_pair(d_tmem, a_tmem + 8u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                    tc_commit_pair(wd_empty(st), 3);
+                        for (int k = 0; k < kBK / 32; ++k)  // +32 int8 along K = +8 columns of A, +2 in B's 16-byte address field
+                            tc_mma_i8_ts_pair(d_tmem, a_tmem + 8u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        tc_commit_pair(wd_empty(st), 3);
+                    }
+                    __syncwarp();
                     if (++st == kWideStages) { st = 0; ph ^= 1u; }
                 }
-                if (ok) tc_commit_pair(acc_full(a), 3);
+                if (ok && elect_one()) tc_commit_pair(acc_full(a), 3);
+                __syncwarp();
             }
-            // nothing issued by this thread may still be running when the pair leaves
-            tc_commit_pair(drain_bar, 1);
+            // nothing issued by this warp may still be running when the pair leaves
+            if (elect_one()) tc_commit_pair(drain_bar, 1);
+            __syncwarp();
             mbar_wait(drain_bar, 0u, abort_flag, kWaitDrain);
         }
         __syncwarp();
