@@ -12,12 +12,12 @@
 //     tensor memory with tcgen05.st and the MMA takes A from there;
 //   * the pair splits the weight tile.
 //
-// Roles per CTA (14 warps):
+// Roles per CTA (22 warps; the unpack warps come in two groups that take alternate k-blocks):
 //   warp 0      TMA producer: packed 4/6-bit activation rows (this CTA's 128 tokens) and packed
 //               4-bit weight rows (this CTA's 96 channels) -> shared-memory ring.
-//   warps 6-9   widen activation codes to int8 and store them to tensor memory (one thread per
+//   warps 6-13  widen activation codes to int8 and store them to tensor memory (one thread per
 //               token row; warp w may touch tensor-memory lanes 32*(w%4)..+31).
-//   warps 10-13 widen weight codes to int8 into the 128-byte-swizzled K-major layout in shared memory.
+//   warps 14-21 widen weight codes to int8 into the 128-byte-swizzled K-major layout in shared memory.
 //               A 4-bit two's-complement nibble masked into the HIGH half of a byte is the int8
 //               value 16*code, a 6-bit code shifted to the top of a byte is 4*code; the factor
 //               (256 or 64 per product) is an exact shift of the int32 accumulator in the
@@ -46,8 +46,10 @@ constexpr int kBN = 192;            // channels of the pair's tile
 constexpr int kBNh = kBN / 2;       // weight rows widened by each CTA
 constexpr int kBK = 128;
 constexpr int kPackedStages = 4, kWideStages = 4;
-constexpr int kAWarps = 4, kWWarps = 4, kEpilogueWarps = 4;
-constexpr int kFirstEpilogueWarp = 2, kFirstAWarp = 6, kFirstWWarp = 10;
+constexpr int kUnpackGroups = 2;   // unpack warps come in groups that take alternate k-blocks
+constexpr int kAWarps = 4 * kUnpackGroups, kWWarps = 4 * kUnpackGroups, kEpilogueWarps = 4;
+constexpr int kFirstEpilogueWarp = 2, kFirstAWarp = 6, kFirstWWarp = kFirstAWarp + kAWarps;
+constexpr int kStageArrivals = (kAWarps + kWWarps) / kUnpackGroups;  // unpack warps working on one k-block, per CTA
 constexpr int kGemmThreads = (2 + kEpilogueWarps + kAWarps + kWWarps) * 32;
 constexpr int kTmemCols = 512;
 constexpr int kTmemACol = 2 * kBN;  // first column of the activation stages
@@ -112,8 +114,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     volatile uint32_t* abort_flag = misc + 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kPackedStages; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), kAWarps + kWWarps); }
-        for (int s = 0; s < kWideStages; ++s) { mbar_init(wd_full(s), 2 * (kAWarps + kWWarps)); mbar_init(wd_empty(s), 1); }
+        for (int s = 0; s < kPackedStages; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), kStageArrivals); }
+        for (int s = 0; s < kWideStages; ++s) { mbar_init(wd_full(s), 2 * kStageArrivals); mbar_init(wd_empty(s), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * kEpilogueWarps); }
         mbar_init(drain_bar, 1);
         misc[1] = 0u;
@@ -303,10 +305,15 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const uint32_t sw_lo = (uint32_t)(row >> 1) & 3u;  // 64-byte-swizzled TMA tile: chunk ^= (row / 2) % 4
         const uint32_t sw_hi = (uint32_t)(row >> 2) & 1u;  // 32-byte-swizzled TMA tile: chunk ^= (row / 4) % 2
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-        uint32_t pst = 0, pph = 0, wst = 0, wph = 0;
+        const uint32_t grp = (uint32_t)(warp - kFirstAWarp) >> 2;
+        uint32_t j = 0;  // k-blocks seen so far; this warp takes those with j % kUnpackGroups == grp
         bool ok = true;
         for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
             for (int kb = 0; kb < KB; ++kb) {
+                const uint32_t jj = j++;
+                if (jj % kUnpackGroups != grp) continue;
+                const uint32_t pst = jj % kPackedStages, pph = (jj / kPackedStages) & 1u;
+                const uint32_t wst = jj % kWideStages, wph = (jj / kWideStages) & 1u;
                 if (!mbar_wait(pk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
                 if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
                 tc_fence_after();
@@ -345,17 +352,20 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive_cluster(map_to_cta(wd_full(wst), 0)); mbar_arrive(pk_empty(pst)); }
-                if (++pst == kPackedStages) { pst = 0; pph ^= 1u; }
-                if (++wst == kWideStages) { wst = 0; wph ^= 1u; }
             }
         }
     } else {
         // ------------------------------------------------------------ widen weight codes -> shared memory
-        const int u = threadIdx.x - kFirstWWarp * 32;  // 0..127
-        uint32_t pst = 0, pph = 0, wst = 0, wph = 0;
+        const int u = (threadIdx.x - kFirstWWarp * 32) & 127;  // thread of its group of four warps
+        const uint32_t grp = (uint32_t)(warp - kFirstWWarp) >> 2;
+        uint32_t j = 0;
         bool ok = true;
         for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
             for (int kb = 0; kb < KB; ++kb) {
+                const uint32_t jj = j++;
+                if (jj % kUnpackGroups != grp) continue;
+                const uint32_t pst = jj % kPackedStages, pph = (jj / kPackedStages) & 1u;
+                const uint32_t wst = jj % kWideStages, wph = (jj / kWideStages) & 1u;
                 if (!mbar_wait(pk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
                 if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
                 tc_fence_after();
@@ -363,8 +373,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 const uint32_t wdW = sbase + S::kWideOff + wst * S::kWideW;
                 // 96 rows x 4 chunks of 32 nibbles, stored as (u - 8)
 #pragma unroll
-                for (int it = 0; it < (kBNh * 4) / (kWWarps * 32); ++it) {
-                    const int qi = it * (kWWarps * 32) + u, row = qi >> 2, ck = qi & 3;
+                for (int it = 0; it < (kBNh * 4) / 128; ++it) {
+                    const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
                     const uint4 p = lds128(pw + row * (kBK / 2) + ck * 16);
                     const uint32_t w[4] = {p.x, p.y, p.z, p.w};
                     uint32_t e[4], o[4];
@@ -377,8 +387,6 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) { mbar_arrive_cluster(map_to_cta(wd_full(wst), 0)); mbar_arrive(pk_empty(pst)); }
-                if (++pst == kPackedStages) { pst = 0; pph ^= 1u; }
-                if (++wst == kWideStages) { wst = 0; wph ^= 1u; }
             }
         }
     }
