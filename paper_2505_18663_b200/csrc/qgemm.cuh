@@ -44,8 +44,10 @@ namespace dvdq {
 constexpr int kBM = 128;            // token rows per CTA (the pair's tile has 2 * kBM)
 constexpr int kBN = 192;            // channels of the pair's tile
 constexpr int kBNh = kBN / 2;       // weight rows widened by each CTA
-constexpr int kBK = 128;
+constexpr int kBK = 128;            // codes per k-block (one unpack + four MMA instructions)
+constexpr int kPK = 2 * kBK;        // codes per TMA load of activation rows: 128-byte rows (A4), the width TMA moves at full rate
 constexpr int kPackedStages = 4, kWideStages = 4;
+constexpr int kWPackedStages = 6;   // ring of packed weight half-tiles (one k-block each)
 constexpr int kUnpackGroups = 2;   // unpack warps come in groups that take alternate k-blocks
 constexpr int kAWarps = 4 * kUnpackGroups, kWWarps = 4 * kUnpackGroups, kEpilogueWarps = 4;
 constexpr int kFirstEpilogueWarp = 2, kFirstAWarp = 6, kFirstWWarp = kFirstAWarp + kAWarps;
@@ -60,20 +62,22 @@ template <int BITS>
 struct GemmSmem {
     static constexpr int kWideW = kBNh * kBK;                     // int8 weight half-tile, swizzled
     static constexpr int kWideOff = 0;                            // 1024-byte aligned tiles first
-    static constexpr int kALo = kBM * kBK / 2;                    // packed low plane / A4 codes (64-byte rows)
-    static constexpr int kAHi = (BITS == 6) ? kBM * kBK / 4 : 0;  // packed high plane (32-byte rows)
-    static constexpr int kW = kBNh * kBK / 2;
-    static constexpr int kPackedStage = kALo + kAHi + kW;
+    static constexpr int kALo = kBM * kPK / 2;                    // packed low plane / A4 codes (128-byte rows)
+    static constexpr int kAHi = (BITS == 6) ? kBM * kPK / 4 : 0;  // packed high plane (64-byte rows)
+    static constexpr int kPackedStage = kALo + kAHi;              // activation codes of two k-blocks
     static constexpr int kPackedOff = kWideOff + kWideStages * kWideW;
     static constexpr int kStageOutOff = kPackedOff + kPackedStages * kPackedStage;  // 1024-byte aligned
-    static constexpr int kStageOutPerWarp = 2 * 32 * 64;  // two buffers of 32 rows x 32 bf16
-    static constexpr int kConstOff = kStageOutOff + kEpilogueWarps * kStageOutPerWarp;
+    static constexpr int kStageOutPerWarp = 2 * 32 * 128;  // two buffers of 32 rows x 64 bf16
+    static constexpr int kWPackedOff = kStageOutOff + kEpilogueWarps * kStageOutPerWarp;
+    static constexpr int kWPacked = kBNh * kBK / 2;              // packed weight half-tile of one k-block (64-byte rows)
+    static constexpr int kConstOff = kWPackedOff + kWPackedStages * kWPacked;
     static constexpr int kConstPerWarp = 3 * kBN * 4;  // delta, zero-point rest, bias
     static constexpr int kBarOff = kConstOff + kEpilogueWarps * kConstPerWarp;
-    static constexpr int kNumBars = 2 * kPackedStages + 2 * kWideStages + 5;
+    static constexpr int kNumBars = 2 * kPackedStages + 2 * kWideStages + 5 + 2 * kWPackedStages;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kTotal = kMiscOff + 16 + 1024;  // + slack for manual 1024-byte alignment
     static_assert(kWideW % 1024 == 0 && kPackedStage % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+    static_assert(kTotal <= 232448, "more than the 227 KB of shared memory a CTA can have");
 };
 
 __device__ __forceinline__ float gelu_tanh_f32(float y) {
@@ -100,7 +104,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
     const int num_n = (N + kBN - 1) / kBN, num_m = (M + 2 * kBM - 1) / (2 * kBM);
     const int num_tiles = num_m * num_n;
-    const int KB = (K + kBK - 1) / kBK;
+    const int KB2 = (K + kPK - 1) / kPK;  // activation loads per tile; a k-block past K reads zeros
+    const int KB = 2 * KB2;
 
     const uint32_t bar0 = sbase + S::kBarOff;
     auto pk_full = [&](int s) { return bar0 + 8u * s; };
@@ -110,14 +115,17 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     auto acc_full = [&](int s) { return bar0 + 8u * (2 * kPackedStages + 2 * kWideStages + s); };      // one per CTA
     auto acc_empty = [&](int s) { return bar0 + 8u * (2 * kPackedStages + 2 * kWideStages + 2 + s); }; // leader's copy
     const uint32_t drain_bar = bar0 + 8u * (2 * kPackedStages + 2 * kWideStages + 4);
+    auto wp_full = [&](int s) { return drain_bar + 8u * (1 + s); };
+    auto wp_empty = [&](int s) { return drain_bar + 8u * (1 + kWPackedStages + s); };
     volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + S::kMiscOff);  // [0] tmem base, [1] abort
     volatile uint32_t* abort_flag = misc + 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kPackedStages; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), kStageArrivals); }
+        for (int s = 0; s < kPackedStages; ++s) { mbar_init(pk_full(s), 1); mbar_init(pk_empty(s), kAWarps); }
         for (int s = 0; s < kWideStages; ++s) { mbar_init(wd_full(s), 2 * kStageArrivals); mbar_init(wd_empty(s), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * kEpilogueWarps); }
         mbar_init(drain_bar, 1);
+        for (int s = 0; s < kWPackedStages; ++s) { mbar_init(wp_full(s), 1); mbar_init(wp_empty(s), kWWarps / kUnpackGroups); }
         misc[1] = 0u;
         fence_mbar_init();
     }
@@ -138,20 +146,26 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             tma_prefetch_desc(&tmA);
             if (BITS == 6) tma_prefetch_desc(&tmAhi);
             tma_prefetch_desc(&tmW);
-            uint32_t st = 0, ph = 0, issued = 0;
+            uint32_t st = 0, ph = 0, issued = 0, wst = 0, wph = 0, wissued = 0;
             bool ok = true;
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
                 const int n0 = (tile % num_n) * kBN + (int)rank * kBNh;
-                for (int kb = 0; kb < KB; ++kb) {
+                for (int sb = 0; ok && sb < KB2; ++sb) {
                     if (!mbar_wait(pk_empty(st), ph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
                     const uint32_t dst = sbase + S::kPackedOff + st * S::kPackedStage;
                     mbar_arrive_expect_tx(pk_full(st), S::kPackedStage);
-                    tma_load_2d(dst, &tmA, pk_full(st), kb * (kBK / 2), m0);
-                    if (BITS == 6) tma_load_2d(dst + S::kALo, &tmAhi, pk_full(st), kb * (kBK / 4), m0);
-                    tma_load_2d(dst + S::kALo + S::kAHi, &tmW, pk_full(st), kb * (kBK / 2), n0);
+                    tma_load_2d(dst, &tmA, pk_full(st), sb * (kPK / 2), m0);
+                    if (BITS == 6) tma_load_2d(dst + S::kALo, &tmAhi, pk_full(st), sb * (kPK / 4), m0);
                     ++issued;
                     if (++st == kPackedStages) { st = 0; ph ^= 1u; }
+                    for (int h = 0; h < 2; ++h) {  // the weight rows of the two k-blocks this load covers
+                        if (!mbar_wait(wp_empty(wst), wph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
+                        mbar_arrive_expect_tx(wp_full(wst), S::kWPacked);
+                        tma_load_2d(sbase + S::kWPackedOff + wst * S::kWPacked, &tmW, wp_full(wst), (2 * sb + h) * (kBK / 2), n0);
+                        ++wissued;
+                        if (++wst == kWPackedStages) { wst = 0; wph ^= 1u; }
+                    }
                 }
             }
             if (!ok) {
@@ -161,6 +175,12 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     const uint32_t s = (st + kPackedStages - 1 - i) % kPackedStages;
                     const uint32_t p = (s < st) ? ph : (ph ^ 1u);
                     for (int it = 0; it < (1 << 16) && !mbar_try_wait(pk_full(s), p); ++it) {}
+                }
+                const uint32_t w_out = wissued < (uint32_t)kWPackedStages ? wissued : (uint32_t)kWPackedStages;
+                for (uint32_t i = 0; i < w_out; ++i) {
+                    const uint32_t s = (wst + kWPackedStages - 1 - i) % kWPackedStages;
+                    const uint32_t p = (s < wst) ? wph : (wph ^ 1u);
+                    for (int it = 0; it < (1 << 16) && !mbar_try_wait(wp_full(s), p); ++it) {}
                 }
             }
         }
@@ -249,10 +269,14 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                         if (row_ok && nb + j < N) *reinterpret_cast<int4*>(dst + j) = o;
                     }
                 } else {
-                    // The staging buffer used two chunks ago must have been read by its TMA store.
-                    if (lane == 0) tma_store_wait_read<1>();
-                    __syncwarp();
-                    const uint32_t buf = stg0 + (nstore & 1u) * (32 * 64);
+                    // Two chunks of 32 columns fill one staging buffer of 32 rows x 128 bytes, which
+                    // leaves as ONE TMA store (128-byte rows are what TMA moves at full rate).  The
+                    // buffer used two stores ago must have been read by its store.
+                    if ((c & 1) == 0) {
+                        if (lane == 0) tma_store_wait_read<1>();
+                        __syncwarp();
+                    }
+                    const uint32_t buf = stg0 + (nstore & 1u) * (32 * 128);
 #pragma unroll
                     for (int j = 0; j < 32; j += 8) {
                         const float4 d0 = lds128f(c_delta + 4 * (c * 32 + j)), d1 = lds128f(c_delta + 4 * (c * 32 + j + 4));
@@ -278,18 +302,20 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                             __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * t], v[2 * t + 1]);
                             pk[t] = *reinterpret_cast<uint32_t*>(&b2);
                         }
-                        // 64-byte rows, 16-byte chunk index XORed with (row >> 1) & 3: the layout a
-                        // 64B-swizzled TMA store reads, and conflict-free for this per-row write.
-                        const int ch = (j >> 3) ^ ((lane >> 1) & 3);
-                        sts128(buf + lane * 64 + ch * 16, pk[0], pk[1], pk[2], pk[3]);
+                        // 128-byte rows, 16-byte chunk index XORed with row % 8: the layout a
+                        // 128B-swizzled TMA store reads, and conflict-free for this per-row write.
+                        const int ch = (4 * (c & 1) + (j >> 3)) ^ (lane & 7);
+                        sts128(buf + lane * 128 + ch * 16, pk[0], pk[1], pk[2], pk[3]);
                     }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0 && nb < N && m0 + q * 32 < M) {
-                        tma_store_2d(&tmY, stg0 + (nstore & 1u) * (32 * 64), nb, m0 + q * 32);
-                        tma_store_commit();
+                    if (c & 1) {
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0 && nb - 32 < N && m0 + q * 32 < M) {
+                            tma_store_2d(&tmY, buf, nb - 32, m0 + q * 32);
+                            tma_store_commit();
+                        }
+                        ++nstore;
                     }
-                    ++nstore;
                 }
             }
             tc_fence_before();
@@ -301,49 +327,51 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     } else if (warp < kFirstWWarp) {
         // ------------------------------------------------------------ widen activation codes -> tensor memory
         const int q = warp & 3;
-        const int row = q * 32 + lane;                     // row of this CTA's tile = tensor-memory lane
-        const uint32_t sw_lo = (uint32_t)(row >> 1) & 3u;  // 64-byte-swizzled TMA tile: chunk ^= (row / 2) % 4
-        const uint32_t sw_hi = (uint32_t)(row >> 2) & 1u;  // 32-byte-swizzled TMA tile: chunk ^= (row / 4) % 2
-        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const uint32_t grp = (uint32_t)(warp - kFirstAWarp) >> 2;
+        const int row = q * 32 + lane;                     // row of this CTA's tile = tensor-memory lane
+        // One packed stage holds two k-blocks; group g unpacks the g-th half of every row.
+        const uint32_t sw_lo = (uint32_t)row & 7u;         // 128-byte-swizzled TMA tile: chunk ^= row % 8
+        const uint32_t sw_hi = (uint32_t)(row >> 1) & 3u;  // 64-byte-swizzled TMA tile: chunk ^= (row / 2) % 4
+        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         uint32_t j = 0;  // k-blocks seen so far; this warp takes those with j % kUnpackGroups == grp
         bool ok = true;
         for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
             for (int kb = 0; kb < KB; ++kb) {
                 const uint32_t jj = j++;
                 if (jj % kUnpackGroups != grp) continue;
-                const uint32_t pst = jj % kPackedStages, pph = (jj / kPackedStages) & 1u;
+                const uint32_t sb = jj / kUnpackGroups;
+                const uint32_t pst = sb % kPackedStages, pph = (sb / kPackedStages) & 1u;
                 const uint32_t wst = jj % kWideStages, wph = (jj / kWideStages) & 1u;
                 if (!mbar_wait(pk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
                 if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t pk = sbase + S::kPackedOff + pst * S::kPackedStage;
-                const uint32_t prow = pk + row * (kBK / 2);
+                const uint32_t prow = pk + row * (kPK / 2);
                 uint32_t r[32];  // r[2i] / r[2i+1]: even / odd codes of packed word i, the K order the weights use too
                 uint32_t h[8];
                 if (BITS == 6) {
-                    const uint32_t hrow = pk + S::kALo + row * (kBK / 4);
+                    const uint32_t hrow = pk + S::kALo + row * (kPK / 4);
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
-                        const uint4 p = lds128(hrow + (((uint32_t)c ^ sw_hi) << 4));
+                        const uint4 p = lds128(hrow + (((2u * grp + (uint32_t)c) ^ sw_hi) << 4));
                         h[4 * c] = p.x; h[4 * c + 1] = p.y; h[4 * c + 2] = p.z; h[4 * c + 3] = p.w;
                     }
                 }
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const uint4 p = lds128(prow + (((uint32_t)c ^ sw_lo) << 4));
+                    const uint4 p = lds128(prow + (((4u * grp + (uint32_t)c) ^ sw_lo) << 4));
                     const uint32_t w[4] = {p.x, p.y, p.z, p.w};
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int i = 4 * c + j;
+                    for (int jw = 0; jw < 4; ++jw) {
+                        const int i = 4 * c + jw;
                         if (BITS == 4) {
-                            r[2 * i] = (w[j] << 4) & 0xF0F0F0F0u;
-                            r[2 * i + 1] = w[j] & 0xF0F0F0F0u;
+                            r[2 * i] = (w[jw] << 4) & 0xF0F0F0F0u;
+                            r[2 * i + 1] = w[jw] & 0xF0F0F0F0u;
                         } else {
                             const uint32_t hh = h[i >> 1];
                             const int a2 = 2 * (i & 1);
-                            r[2 * i] = ((w[j] << 2) & 0x3C3C3C3Cu) | ((hh << (6 - 2 * a2)) & 0xC0C0C0C0u);
-                            r[2 * i + 1] = ((w[j] >> 2) & 0x3C3C3C3Cu) | ((hh << (4 - 2 * a2)) & 0xC0C0C0C0u);
+                            r[2 * i] = ((w[jw] << 2) & 0x3C3C3C3Cu) | ((hh << (6 - 2 * a2)) & 0xC0C0C0C0u);
+                            r[2 * i + 1] = ((w[jw] >> 2) & 0x3C3C3C3Cu) | ((hh << (4 - 2 * a2)) & 0xC0C0C0C0u);
                         }
                     }
                 }
@@ -356,37 +384,37 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         }
     } else {
         // ------------------------------------------------------------ widen weight codes -> shared memory
-        const int u = (threadIdx.x - kFirstWWarp * 32) & 127;  // thread of its group of four warps
         const uint32_t grp = (uint32_t)(warp - kFirstWWarp) >> 2;
+        const int u = (threadIdx.x - kFirstWWarp * 32) & 127;  // thread of its group of four warps
         uint32_t j = 0;
         bool ok = true;
         for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
             for (int kb = 0; kb < KB; ++kb) {
-                const uint32_t jj = j++;
-                if (jj % kUnpackGroups != grp) continue;
-                const uint32_t pst = jj % kPackedStages, pph = (jj / kPackedStages) & 1u;
-                const uint32_t wst = jj % kWideStages, wph = (jj / kWideStages) & 1u;
-                if (!mbar_wait(pk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t pw = sbase + S::kPackedOff + pst * S::kPackedStage + S::kALo + S::kAHi;
-                const uint32_t wdW = sbase + S::kWideOff + wst * S::kWideW;
-                // 96 rows x 4 chunks of 32 nibbles, stored as (u - 8)
+            const uint32_t jj = j++;
+            if (jj % kUnpackGroups != grp) continue;
+            const uint32_t pst = jj % kWPackedStages, pph = (jj / kWPackedStages) & 1u;
+            const uint32_t wst = jj % kWideStages, wph = (jj / kWideStages) & 1u;
+            if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+            if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+            tc_fence_after();
+            const uint32_t pw = sbase + S::kWPackedOff + pst * S::kWPacked;
+            const uint32_t wdW = sbase + S::kWideOff + wst * S::kWideW;
+            // 96 rows x 4 chunks of 32 nibbles, stored as (u - 8)
 #pragma unroll
-                for (int it = 0; it < (kBNh * 4) / 128; ++it) {
-                    const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
-                    const uint4 p = lds128(pw + row * (kBK / 2) + ck * 16);
-                    const uint32_t w[4] = {p.x, p.y, p.z, p.w};
-                    uint32_t e[4], o[4];
+            for (int it = 0; it < (kBNh * 4) / 128; ++it) {
+                const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                const uint4 p = lds128(pw + row * (kBK / 2) + ck * 16);
+                const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+                uint32_t e[4], o[4];
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) { e[j] = (w[j] << 4) & 0xF0F0F0F0u; o[j] = w[j] & 0xF0F0F0F0u; }
-                    const uint32_t drow = wdW + (row >> 3) * 1024 + (row & 7) * 128;
-                    sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[0], o[0], e[1], o[1]);
-                    sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[2], o[2], e[3], o[3]);
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) { mbar_arrive_cluster(map_to_cta(wd_full(wst), 0)); mbar_arrive(pk_empty(pst)); }
+                for (int jw = 0; jw < 4; ++jw) { e[jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[jw] = w[jw] & 0xF0F0F0F0u; }
+                const uint32_t drow = wdW + (row >> 3) * 1024 + (row & 7) * 128;
+                sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[0], o[0], e[1], o[1]);
+                sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[2], o[2], e[3], o[3]);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) { mbar_arrive_cluster(map_to_cta(wd_full(wst), 0)); mbar_arrive(wp_empty(pst)); }
             }
         }
     }
@@ -416,17 +444,17 @@ inline PFN_encodeTiled get_encode_tiled() {
     return fn;
 }
 
-// bf16 matrix [rows, cols] with row pitch ld elements, tiles of 32 x 32, 64-byte swizzle
-// (the layout the epilogue stages its output in).
+// bf16 matrix [rows, cols] with row pitch ld elements, tiles of 32 rows x 64 columns, 128-byte
+// swizzle (the layout the epilogue stages its output in).
 inline bool make_out_map(CUtensorMap* tm, const void* base, uint64_t cols, uint64_t rows, uint64_t ld) {
     PFN_encodeTiled enc = get_encode_tiled();
     if (!enc) return false;
     const cuuint64_t dims[2] = {cols, rows};
     const cuuint64_t strides[1] = {ld * 2};
-    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t box[2] = {64, 32};
     const cuuint32_t estr[2] = {1, 1};
     return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -455,19 +483,19 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
     const uint64_t pitch = (uint64_t)act_row_bytes(K, BITS);
     CUtensorMap tmA, tmAhi, tmW, tmY;
-    if (!make_byte_map(&tmA, codes, (uint64_t)K / 2, (uint64_t)M, pitch, kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_64B))
+    if (!make_byte_map(&tmA, codes, (uint64_t)K / 2, (uint64_t)M, pitch, kPK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_128B))
         return DVDQ_ERR_CUDA;
     if (BITS == 6) {
         if (!make_byte_map(&tmAhi, static_cast<const uint8_t*>(codes) + K / 2, (uint64_t)K / 4, (uint64_t)M, pitch,
-                           kBK / 4, kBM, CU_TENSOR_MAP_SWIZZLE_32B))
+                           kPK / 4, kBM, CU_TENSOR_MAP_SWIZZLE_64B))
             return DVDQ_ERR_CUDA;
     } else {
         tmAhi = tmA;
     }
+
     if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, kBNh,
                        CU_TENSOR_MAP_SWIZZLE_NONE))
         return DVDQ_ERR_CUDA;
-
     if (RAW) {
         tmY = tmA;  // unused
     } else if (!make_out_map(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)) {
