@@ -343,8 +343,6 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 const uint32_t pst = sb % kPackedStages, pph = (sb / kPackedStages) & 1u;
                 const uint32_t wst = jj % kWideStages, wph = (jj / kWideStages) & 1u;
                 if (!mbar_wait(pk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-                tc_fence_after();
                 const uint32_t pk = sbase + S::kPackedOff + pst * S::kPackedStage;
                 const uint32_t prow = pk + row * (kPK / 2);
                 uint32_t r[32];  // r[2i] / r[2i+1]: even / odd codes of packed word i, the K order the weights use too
@@ -375,11 +373,16 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                         }
                     }
                 }
+                // the codes are widened in registers before the stage of tensor memory is known to be free
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pk_empty(pst));
+                if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                tc_fence_after();
                 tmem_st_32x32(tmem_base + kTmemACol + wst * kAColsPerStage + lane_addr, r);
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) { mbar_arrive_cluster(map_to_cta(wd_full(wst), 0)); mbar_arrive(pk_empty(pst)); }
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(wd_full(wst), 0));
             }
         }
     } else {
@@ -395,26 +398,34 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const uint32_t pst = jj % kWPackedStages, pph = (jj / kWPackedStages) & 1u;
             const uint32_t wst = jj % kWideStages, wph = (jj / kWideStages) & 1u;
             if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-            if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-            tc_fence_after();
             const uint32_t pw = sbase + S::kWPackedOff + pst * S::kWPacked;
             const uint32_t wdW = sbase + S::kWideOff + wst * S::kWideW;
-            // 96 rows x 4 chunks of 32 nibbles, stored as (u - 8)
+            // 96 rows x 4 chunks of 32 nibbles, stored as (u - 8); widened in registers before the
+            // wide stage is known to be free
+            constexpr int kPieces = (kBNh * 4) / 128;
+            uint32_t e[kPieces][4], o[kPieces][4];
 #pragma unroll
-            for (int it = 0; it < (kBNh * 4) / 128; ++it) {
+            for (int it = 0; it < kPieces; ++it) {
                 const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
                 const uint4 p = lds128(pw + row * (kBK / 2) + ck * 16);
                 const uint32_t w[4] = {p.x, p.y, p.z, p.w};
-                uint32_t e[4], o[4];
 #pragma unroll
-                for (int jw = 0; jw < 4; ++jw) { e[jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[jw] = w[jw] & 0xF0F0F0F0u; }
+                for (int jw = 0; jw < 4; ++jw) { e[it][jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[it][jw] = w[jw] & 0xF0F0F0F0u; }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(wp_empty(pst));  // the packed rows are in registers
+            if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int it = 0; it < kPieces; ++it) {
+                const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
                 const uint32_t drow = wdW + (row >> 3) * 1024 + (row & 7) * 128;
-                sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[0], o[0], e[1], o[1]);
-                sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[2], o[2], e[3], o[3]);
+                sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[it][0], o[it][0], e[it][1], o[it][1]);
+                sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[it][2], o[it][2], e[it][3], o[it][3]);
             }
             fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) { mbar_arrive_cluster(map_to_cta(wd_full(wst), 0)); mbar_arrive(wp_empty(pst)); }
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(wd_full(wst), 0));
             }
         }
     }
