@@ -276,7 +276,8 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
         // non-negative floats order like their bit patterns: one REDUX instead of five shuffles
         amax = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(amax)));
         if (lane == 0) s_max[buf][warp] = amax;
-        __syncthreads();
+        // only the warps of this token meet: named barrier 1 + tl, spans * 32 threads
+        if (spans > 1) asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
         if (spans > 1)
             amax = __uint_as_float(__reduce_max_sync(
                 0xFFFFFFFFu, lane < spans ? __float_as_uint(s_max[buf][tl * spans + lane]) : 0u));
@@ -337,7 +338,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
         prev_token = token;
         prev_amax = amax;
     }
-    __syncthreads();
+    if (spans > 1) asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
     if (sp == 0 && prev_token >= 0) {
         const uint32_t buf = (it & 1u) ^ 1u;  // the last iteration's slots
         const int tsum = __reduce_add_sync(0xFFFFFFFFu, lane < spans ? s_sum[buf][tl * spans + lane] : 0);
@@ -353,7 +354,7 @@ static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t
                                     int32_t* sums, cudaStream_t st) {
     const int spans = (int)((K + kRqSpan - 1) / kRqSpan);
     if (spans > kRqMaxWarps) return DVDQ_ERR_SHAPE;
-    int tpc = 12 / spans;
+    int tpc = 12 / spans;  // at most 12 tokens per CTA: named barriers 1..12
     if (tpc < 1) tpc = 1;
     const int warps = spans * tpc;
     const int threads = warps * 32;
