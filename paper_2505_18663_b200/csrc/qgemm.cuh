@@ -250,6 +250,8 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const float s_i = (!RAW && row_ok) ? scales[row] : 0.f;
             const int32_t S_i = row_ok ? sums[row] : 0;
             const float S_f = (float)S_i;  // |sum of codes| <= K * 32 < 2^24: exact
+            const float s_k = s_i * (1.0f / (float)(1 << kShift)), nS_k = -S_f * (float)(1 << kShift);
+            const uint64_t s2 = f2_pack(s_k, s_k), negS2 = f2_pack(nS_k, nS_k);
 #pragma unroll 1
             for (int c = 0; c < kBN / 32; ++c) {
                 uint32_t r[32];
@@ -286,15 +288,19 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                         const float zz[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
                         const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
                         float v[8];
+                        // The raw accumulator is (256 or 64) x the true one: at most 22 significant
+                        // bits, so its conversion is exact and the factor moves into the per-row
+                        // constants: y = (raw - zz * S * 2^k) * (s * 2^-k * delta) + bias, on fp32 pairs.
 #pragma unroll
-                        for (int t = 0; t < 8; ++t) {
-                            // int -> float without the conversion pipe: |acc >> shift| <= K*32*8 <= 2^22
-                            const int32_t sh = (int32_t)r[j + t] >> kShift;
-                            float f = __int_as_float(sh + 0x4B400000) - 12582912.0f;
-                            f = fmaf(-zz[t], S_f, f);                 // rest of the zero point, exact
-                            float y = fmaf(f, s_i * dl[t], bb[t]);
-                            if (act == 1) y = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(y)));
-                            v[t] = y;
+                        for (int t = 0; t < 8; t += 2) {
+                            const uint64_t raw2 = f2_pack((float)(int32_t)r[j + t], (float)(int32_t)r[j + t + 1]);
+                            const uint64_t acc2 = f2_fma(f2_pack(zz[t], zz[t + 1]), negS2, raw2);   // exact
+                            const uint64_t y2 = f2_fma(acc2, f2_mul(f2_pack(dl[t], dl[t + 1]), s2), f2_pack(bb[t], bb[t + 1]));
+                            f2_unpack(y2, v[t], v[t + 1]);
+                        }
+                        if (act == 1) {
+#pragma unroll
+                            for (int t = 0; t < 8; ++t) v[t] = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(v[t])));
                         }
                         uint32_t pk[4];
 #pragma unroll
