@@ -38,7 +38,7 @@ typedef enum {
     DVDQ_OK = 0,
     DVDQ_ERR_NULL = 1,           /* a required pointer is NULL */
     DVDQ_ERR_SHAPE = 2,          /* M, N, K or a leading dimension is not supported */
-    DVDQ_ERR_BITS = 3,           /* activation bit width is not 4 or 6 */
+    DVDQ_ERR_BITS = 3,           /* activation bit width is not 4, 6 or 8 */
     DVDQ_ERR_ROT_BLOCK = 4,      /* rotation block invalid, or activations and weights disagree on it */
     DVDQ_ERR_ALIGN = 5,          /* a pointer or pitch misses its alignment requirement */
     DVDQ_ERR_WORKSPACE = 6,      /* workspace too small */
@@ -46,7 +46,7 @@ typedef enum {
     DVDQ_ERR_ARCH = 8,           /* current device is not sm_100 */
     DVDQ_ERR_CUDA = 9,           /* a CUDA runtime or driver call failed */
     DVDQ_ERR_DEVICE_TIMEOUT = 10,/* a kernel gave up on a bounded device-side wait */
-    DVDQ_ERR_UNSUPPORTED = 11    /* a reserved option (scale_group != 0, bits == 8) */
+    DVDQ_ERR_UNSUPPORTED = 11    /* a reserved option (scale_group != 0, unknown activation function) */
 } dvdq_status;
 
 /* Human-readable name of a status code (static storage, never NULL). */
@@ -54,7 +54,8 @@ const char* dvdq_status_string(dvdq_status s);
 
 /*
  * The activation quantizer of Eq. 10, X^ = Q(X H Lambda^-1):
- *   bits        b, the code width: 4 (codes in [-8,7]) or 6 (codes in [-32,31]).
+ *   bits        b, the code width: 4 (codes in [-8,7]), 6 (codes in [-32,31]) or 8 (codes in
+ *               [-128,127]; the b_high = 8 of Sec. 3.3's bit-width switching, i.e. the W4A8 steps).
  *               The quantizer is symmetric with qmax = 2^(b-1) - 1.
  *   rot_block   B, the order of the Hadamard blocks of the rotation
  *               R = I_{K/B} (x) H_B / sqrt(B); a power of two in [64, 1024] that

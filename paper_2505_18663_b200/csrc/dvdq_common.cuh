@@ -52,7 +52,8 @@ __host__ __device__ inline BlobLayout blob_layout(int64_t N, int64_t K) {
 // each code, followed by a high plane of K/4 bytes with bits 5:4.  In the high plane one
 // 32-bit word covers 16 consecutive positions p = 16m + 8a + i (a in {0,1}, i in 0..7):
 // the 2-bit field sits at bit 2*(4*(i>>1) + 2*a + (i&1)).  That order makes the GEMM's
-// widening of 16 codes into four int8 words a shift and a mask per word.
+// widening of 16 codes into four int8 words a shift and a mask per word.  A8 = K bytes: int8 codes,
+// each group of 8 channels as its four even channels followed by its four odd ones.
 __host__ __device__ inline int64_t act_row_bytes(int64_t K, int bits) { return K * bits / 8; }
 __host__ __device__ inline int hi_field_shift(int a, int i) { return 2 * (4 * (i >> 1) + 2 * a + (i & 1)); }
 

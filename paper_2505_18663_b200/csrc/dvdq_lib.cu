@@ -37,8 +37,7 @@ static dvdq_status validate_k(int64_t K) {
 
 dvdq_status validate_act_quant(const dvdq_act_quant* q, int64_t K) {
     if (!q) return DVDQ_ERR_NULL;
-    if (q->bits == 8) return DVDQ_ERR_UNSUPPORTED;
-    if (q->bits != 4 && q->bits != 6) return DVDQ_ERR_BITS;
+    if (q->bits != 4 && q->bits != 6 && q->bits != 8) return DVDQ_ERR_BITS;
     if (q->scale_group != 0) return DVDQ_ERR_UNSUPPORTED;
     if (q->rot_block != 0) {
         if (!is_pow2(q->rot_block) || q->rot_block < 64 || q->rot_block > 1024) return DVDQ_ERR_ROT_BLOCK;
@@ -80,7 +79,7 @@ const char* dvdq_status_string(dvdq_status s) {
         case DVDQ_OK: return "ok";
         case DVDQ_ERR_NULL: return "required pointer is NULL";
         case DVDQ_ERR_SHAPE: return "unsupported shape or leading dimension";
-        case DVDQ_ERR_BITS: return "activation bit width must be 4 or 6";
+        case DVDQ_ERR_BITS: return "activation bit width must be 4, 6 or 8";
         case DVDQ_ERR_ROT_BLOCK: return "rotation block invalid or inconsistent between activations and weights";
         case DVDQ_ERR_ALIGN: return "pointer or pitch not aligned as required";
         case DVDQ_ERR_WORKSPACE: return "workspace too small";
@@ -96,7 +95,7 @@ const char* dvdq_status_string(dvdq_status s) {
 int32_t dvdq_version(void) { return kLibVersion; }
 
 size_t dvdq_act_codes_bytes(int64_t M, int64_t K, int32_t bits) {
-    if (M < 0 || validate_k(K) != DVDQ_OK || (bits != 4 && bits != 6)) return 0;
+    if (M < 0 || validate_k(K) != DVDQ_OK || (bits != 4 && bits != 6 && bits != 8)) return 0;
     return (size_t)(M * act_row_bytes(K, bits));
 }
 
@@ -245,7 +244,8 @@ dvdq_status dvdq_pack_act_codes(const int8_t* codes_nat, int64_t M, int64_t K, c
     cudaStream_t st = (cudaStream_t)stream;
     const unsigned g = grid_for(M * (K / 16), 256);
     if (q->bits == 4) pack_act_codes_kernel<4><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
-    else pack_act_codes_kernel<6><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
+    else if (q->bits == 6) pack_act_codes_kernel<6><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
+    else pack_act_codes_kernel<8><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
     code_sums_kernel<<<(unsigned)((M * 32 + 255) / 256), 256, 0, st>>>(codes_nat, M, K, code_sums_out);
     return cuda_status(cudaGetLastError());
 }
@@ -261,7 +261,8 @@ dvdq_status dvdq_unpack_act_codes(const void* codes, int64_t M, int64_t K, const
     if ((s = check_device_arch()) != DVDQ_OK) return s;
     const unsigned g = grid_for(M * (K / 16), 256);
     if (q->bits == 4) unpack_act_codes_kernel<4><<<g, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint8_t*>(codes), M, K, codes_nat);
-    else unpack_act_codes_kernel<6><<<g, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint8_t*>(codes), M, K, codes_nat);
+    else if (q->bits == 6) unpack_act_codes_kernel<6><<<g, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint8_t*>(codes), M, K, codes_nat);
+    else unpack_act_codes_kernel<8><<<g, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint8_t*>(codes), M, K, codes_nat);
     return cuda_status(cudaGetLastError());
 }
 

@@ -58,6 +58,11 @@ __global__ void pack_act_codes_kernel(const int8_t* __restrict__ nat, int64_t M,
         const int64_t i = t / groups, m = t - i * groups;
         const int8_t* src = nat + i * K + m * 16;
         uint8_t* row = packed + i * row_bytes;
+        if (BITS == 8) {  // per 8 channels: the four even channels, then the four odd ones
+            for (int a = 0; a < 2; ++a)
+                for (int j = 0; j < 8; ++j) row[m * 16 + 8 * a + 4 * (j & 1) + (j >> 1)] = (uint8_t)src[8 * a + j];
+            continue;
+        }
         uint32_t lo[2] = {0u, 0u}, hi = 0u;
         for (int a = 0; a < 2; ++a)
             for (int j = 0; j < 8; ++j) {
@@ -78,6 +83,11 @@ __global__ void unpack_act_codes_kernel(const uint8_t* __restrict__ packed, int6
     for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
         const int64_t i = t / groups, m = t - i * groups;
         const uint8_t* row = packed + i * row_bytes;
+        if (BITS == 8) {
+            for (int a = 0; a < 2; ++a)
+                for (int j = 0; j < 8; ++j) nat[i * K + m * 16 + 8 * a + j] = (int8_t)row[m * 16 + 8 * a + 4 * (j & 1) + (j >> 1)];
+            continue;
+        }
         const uint32_t lo[2] = {reinterpret_cast<const uint32_t*>(row)[2 * m], reinterpret_cast<const uint32_t*>(row)[2 * m + 1]};
         const uint32_t hi = (BITS == 6) ? reinterpret_cast<const uint32_t*>(row + K / 2)[m] : 0u;
         for (int a = 0; a < 2; ++a)

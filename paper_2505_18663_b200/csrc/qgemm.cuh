@@ -62,11 +62,12 @@ template <int BITS>
 struct GemmSmem {
     static constexpr int kWideW = kBNh * kBK;                     // int8 weight half-tile, swizzled
     static constexpr int kWideOff = 0;                            // 1024-byte aligned tiles first
-    static constexpr int kALo = kBM * kPK / 2;                    // packed low plane / A4 codes (128-byte rows)
+    static constexpr int kALo = (BITS == 8) ? kBM * kPK : kBM * kPK / 2;  // A4 codes / A6 low plane (128-byte rows); A8: two tiles of 128-byte rows, one per k-block
+    static constexpr int kPStages = (BITS == 8) ? 3 : kPackedStages;  // what fits
     static constexpr int kAHi = (BITS == 6) ? kBM * kPK / 4 : 0;  // packed high plane (64-byte rows)
     static constexpr int kPackedStage = kALo + kAHi;              // activation codes of two k-blocks
     static constexpr int kPackedOff = kWideOff + kWideStages * kWideW;
-    static constexpr int kStageOutOff = kPackedOff + kPackedStages * kPackedStage;  // 1024-byte aligned
+    static constexpr int kStageOutOff = kPackedOff + kPStages * kPackedStage;  // 1024-byte aligned
     static constexpr int kStageOutPerWarp = 2 * 32 * 128;  // two buffers of 32 rows x 64 bf16
     static constexpr int kWPackedOff = kStageOutOff + kEpilogueWarps * kStageOutPerWarp;
     static constexpr int kWPacked = kBNh * kBK / 2;              // packed weight half-tile of one k-block (64-byte rows)
@@ -155,10 +156,15 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     if (!mbar_wait(pk_empty(st), ph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
                     const uint32_t dst = sbase + S::kPackedOff + st * S::kPackedStage;
                     mbar_arrive_expect_tx(pk_full(st), S::kPackedStage);
-                    tma_load_2d(dst, &tmA, pk_full(st), sb * (kPK / 2), m0);
+                    if (BITS == 8) {
+                        tma_load_2d(dst, &tmA, pk_full(st), sb * kPK, m0);
+                        tma_load_2d(dst + S::kALo / 2, &tmA, pk_full(st), sb * kPK + kBK, m0);
+                    } else {
+                        tma_load_2d(dst, &tmA, pk_full(st), sb * (kPK / 2), m0);
+                    }
                     if (BITS == 6) tma_load_2d(dst + S::kALo, &tmAhi, pk_full(st), sb * (kPK / 4), m0);
                     ++issued;
-                    if (++st == kPackedStages) { st = 0; ph ^= 1u; }
+                    if (++st == S::kPStages) { st = 0; ph ^= 1u; }
                     for (int h = 0; h < 2; ++h) {  // the weight rows of the two k-blocks this load covers
                         if (!mbar_wait(wp_empty(wst), wph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
                         mbar_arrive_expect_tx(wp_full(wst), S::kWPacked);
@@ -170,9 +176,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             }
             if (!ok) {
                 // Giving up: let copies already in flight land before the CTA exits (bounded).
-                const uint32_t n_out = issued < (uint32_t)kPackedStages ? issued : (uint32_t)kPackedStages;
+                const uint32_t n_out = issued < (uint32_t)S::kPStages ? issued : (uint32_t)S::kPStages;
                 for (uint32_t i = 0; i < n_out; ++i) {
-                    const uint32_t s = (st + kPackedStages - 1 - i) % kPackedStages;
+                    const uint32_t s = (st + S::kPStages - 1 - i) % S::kPStages;
                     const uint32_t p = (s < st) ? ph : (ph ^ 1u);
                     for (int it = 0; it < (1 << 16) && !mbar_try_wait(pk_full(s), p); ++it) {}
                 }
@@ -228,7 +234,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const uint32_t c_zc = c_delta + kBN * 4;    // (z_n - 8) as a float: exact, |.| <= 8
         const uint32_t c_bias = c_zc + kBN * 4;
         const uint32_t stg0 = sbase + S::kStageOutOff + ew * S::kStageOutPerWarp;
-        constexpr int kShift = (BITS == 4) ? 8 : 6;
+        constexpr int kShift = (BITS == 4) ? 8 : (BITS == 6) ? 6 : 4;  // log2 of (A factor 16 / 4 / 1) x (W factor 16)
         if (!RAW && lane == 0) tma_prefetch_desc(&tmY);
         uint32_t lt = 0, nstore = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++lt) {
@@ -346,7 +352,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 const uint32_t jj = j++;
                 if (jj % kUnpackGroups != grp) continue;
                 const uint32_t sb = jj / kUnpackGroups;
-                const uint32_t pst = sb % kPackedStages, pph = (sb / kPackedStages) & 1u;
+                const uint32_t pst = sb % S::kPStages, pph = (sb / S::kPStages) & 1u;
                 const uint32_t wst = jj % kWideStages, wph = (jj / kWideStages) & 1u;
                 if (!mbar_wait(pk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
                 const uint32_t pk = sbase + S::kPackedOff + pst * S::kPackedStage;
@@ -361,8 +367,17 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                         h[4 * c] = p.x; h[4 * c + 1] = p.y; h[4 * c + 2] = p.z; h[4 * c + 3] = p.w;
                     }
                 }
+                if (BITS == 8) {
+                    // int8 codes, already in the even/odd order of the weight operand: no widening
+                    const uint32_t prow8 = pk + grp * (S::kALo / 2) + row * kBK;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                    for (int c = 0; c < 8; ++c) {
+                        const uint4 p = lds128(prow8 + (((uint32_t)c ^ sw_lo) << 4));
+                        r[4 * c] = p.x; r[4 * c + 1] = p.y; r[4 * c + 2] = p.z; r[4 * c + 3] = p.w;
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < (BITS == 8 ? 0 : 4); ++c) {
                     const uint4 p = lds128(prow + (((4u * grp + (uint32_t)c) ^ sw_lo) << 4));
                     const uint32_t w[4] = {p.x, p.y, p.z, p.w};
 #pragma unroll
@@ -500,7 +515,7 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
     const uint64_t pitch = (uint64_t)act_row_bytes(K, BITS);
     CUtensorMap tmA, tmAhi, tmW, tmY;
-    if (!make_byte_map(&tmA, codes, (uint64_t)K / 2, (uint64_t)M, pitch, kPK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_128B))
+    if (!make_byte_map(&tmA, codes, (uint64_t)(BITS == 8 ? K : K / 2), (uint64_t)M, pitch, kPK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_128B))
         return DVDQ_ERR_CUDA;
     if (BITS == 6) {
         if (!make_byte_map(&tmAhi, static_cast<const uint8_t*>(codes) + K / 2, (uint64_t)K / 4, (uint64_t)M, pitch,
@@ -558,6 +573,9 @@ inline dvdq_status launch_qgemm(const void* codes, const float* scales, const in
     if (q.bits == 4)
         return raw ? launch_qgemm_t<4, true>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
                    : launch_qgemm_t<4, false>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
+    if (q.bits == 8)
+        return raw ? launch_qgemm_t<8, true>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
+                   : launch_qgemm_t<8, false>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
     return raw ? launch_qgemm_t<6, true>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
                : launch_qgemm_t<6, false>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
 }

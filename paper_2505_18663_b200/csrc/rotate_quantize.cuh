@@ -290,9 +290,15 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
             const uint32_t O = __byte_perm(__byte_perm(b[1], b[3], 0x0040), __byte_perm(b[5], b[7], 0x0040), 0x5410);
             lsum = __dp4a((int)E, 0x01010101, lsum);
             lsum = __dp4a((int)O, 0x01010101, lsum);
-            const uint32_t lo = (E & 0x0F0F0F0Fu) | ((O << 4) & 0xF0F0F0F0u);
             const int e0 = st_e0 + j * 64;
             const bool ok = FULL || (st_ok >> j & 1u);
+            if (BITS == 8) {
+                // 8-bit codes: each group of 8 channels is stored as the word of its even channels
+                // followed by the word of its odd channels, the order the GEMM consumes
+                if (ok) *reinterpret_cast<uint2*>(crow + e0) = make_uint2(E, O);
+                continue;
+            }
+            const uint32_t lo = (E & 0x0F0F0F0Fu) | ((O << 4) & 0xF0F0F0F0u);
             if (ok) *reinterpret_cast<uint32_t*>(crow + (e0 >> 1)) = lo;
             if (BITS == 6) {
                 // bits 5:4 of 16 consecutive channels share one word of the high plane; the two
@@ -383,7 +389,8 @@ inline dvdq_status launch_rotate_quantize(const void* X, int64_t M, int64_t K, i
                                           void* codes, float* scales, int32_t* sums, cudaStream_t st) {
     if (M == 0) return DVDQ_OK;
     if (q.bits == 4) return launch_rq_bits<4>(X, M, K, ldx, q.rot_block, codes, scales, sums, st);
-    return launch_rq_bits<6>(X, M, K, ldx, q.rot_block, codes, scales, sums, st);
+    if (q.bits == 6) return launch_rq_bits<6>(X, M, K, ldx, q.rot_block, codes, scales, sums, st);
+    return launch_rq_bits<8>(X, M, K, ldx, q.rot_block, codes, scales, sums, st);
 }
 
 }  // namespace dvdq

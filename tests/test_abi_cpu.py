@@ -63,7 +63,8 @@ def test_validation_happens_before_any_cuda_call():
     one = C.c_void_p(256)   # never dereferenced: validation fails first
     assert lib.dvdq_rotate_quantize(one, 4, 256, 256, None, one, one, one, None) == B.ERR_NULL
     assert lib.dvdq_rotate_quantize(one, 4, 256, 256, C.byref(q), one, one, one, None) == B.ERR_BITS
-    assert lib.dvdq_rotate_quantize(one, 4, 256, 256, C.byref(B.ActQuant(8, 256, 0)), one, one, one, None) == B.ERR_UNSUPPORTED
+    assert lib.dvdq_rotate_quantize(one, 4, 256, 256, C.byref(B.ActQuant(16, 256, 0)), one, one, one, None) == B.ERR_BITS
+    assert B.dvdq_act_codes_bytes(3, 256, 8) == 3 * 256 and B.dvdq_act_codes_bytes(3, 256, 6) == 3 * 192
     assert lib.dvdq_rotate_quantize(one, 4, 250, 256, C.byref(B.ActQuant(4, 0, 0)), one, one, one, None) == B.ERR_SHAPE
     assert lib.dvdq_rotate_quantize(one, 4, 256, 128, C.byref(B.ActQuant(4, 256, 0)), one, one, one, None) == B.ERR_SHAPE
     assert lib.dvdq_rotate_quantize(one, 4, 256, 256, C.byref(B.ActQuant(4, 96, 0)), one, one, one, None) == B.ERR_ROT_BLOCK

@@ -48,7 +48,7 @@ def synth_w(N, K, seed):
 
 # ------------------------------------------------------------------ formats
 
-@pytest.mark.parametrize("bits", [4, 6])
+@pytest.mark.parametrize("bits", [4, 6, 8])
 def test_activation_code_pack_unpack_roundtrip(bits):
     M, K = 37, 448
     lim = 2 ** (bits - 1)
@@ -88,7 +88,7 @@ RQ_CASES = [
 ]
 
 
-@pytest.mark.parametrize("bits", [4, 6])
+@pytest.mark.parametrize("bits", [4, 6, 8])
 @pytest.mark.parametrize("M,K,Bk", RQ_CASES)
 def test_rotate_quantize_matches_oracle(M, K, Bk, bits):
     x = synth_x(M, K, seed=M + K + bits)
@@ -170,6 +170,9 @@ GEMM_CASES = [
     (300, 512, 1536, 512, 6, "symmetric"),
     (257, 776, 3072, 1024, 4, "minmax"),
     (129, 256, 8960, 256, 6, "minmax"),
+    # 8-bit activations (the b_high steps of the bit-width switching): M and N tails, K not a multiple of 256
+    (300, 520, 1536, 512, 8, "minmax"),
+    (257, 192, 3200, 128, 8, "symmetric"),
 ]
 
 
@@ -195,22 +198,24 @@ def test_int32_accumulators_are_bit_exact_on_oracle_codes(M, N, K, Bk, bits, mod
     assert np.array_equal(acc.cpu().numpy(), acc_or)
 
 
-def test_int32_accumulators_at_code_extremes():
-    # every product at its largest magnitude: |acc| = K * 32 * 15
+@pytest.mark.parametrize("bits", [6, 8])
+def test_int32_accumulators_at_code_extremes(bits):
+    # every product at its largest magnitude: |acc| = K * 2^(bits-1) * 15
     M, N, K = 128, 256, 4096
-    codes = np.full((M, K), -32, dtype=np.int32)
-    codes[1::2] = 31
+    lim = 2 ** (bits - 1)
+    codes = np.full((M, K), -lim, dtype=np.int32)
+    codes[1::2] = lim - 1
     u = np.zeros((N, K), dtype=np.uint8)
     u[::2] = 15
     z = np.zeros(N, dtype=np.int32)
     z[1::2] = 15
     d = np.ones(N, dtype=np.float32)
     acc_or = orc.int_gemm(codes, u, z)
-    assert np.abs(acc_or).max() == 32 * 15 * K
+    assert np.abs(acc_or).max() == lim * 15 * K
     w, blob = gpu_pack_weights(u, d, z, 1024)
-    packed, sums = gpu_pack_codes(codes, 6, 1024)
+    packed, sums = gpu_pack_codes(codes, bits, 1024)
     acc = torch.zeros(M, N, dtype=torch.int32, device=DEV)
-    B.dvdq_qgemm_int32(packed, sums, M, act_quant(6, 1024), w, acc)
+    B.dvdq_qgemm_int32(packed, sums, M, act_quant(bits, 1024), w, acc)
     assert_device_ok()
     assert np.array_equal(acc.cpu().numpy(), acc_or)
 
@@ -218,7 +223,7 @@ def test_int32_accumulators_at_code_extremes():
 # ------------------------------------------------------------------ dequantizing epilogue
 
 @pytest.mark.parametrize("act", [0, 1])
-@pytest.mark.parametrize("M,N,K,Bk,bits,mode", [GEMM_CASES[1], GEMM_CASES[3], GEMM_CASES[4]])
+@pytest.mark.parametrize("M,N,K,Bk,bits,mode", [GEMM_CASES[1], GEMM_CASES[3], GEMM_CASES[4], GEMM_CASES[6]])
 def test_bf16_output_on_oracle_codes_and_scales(M, N, K, Bk, bits, mode, act):
     x, u, d, z, codes, s64, s32, xt = oracle_layer(M, N, K, Bk, bits, mode, seed=3 * M + N)
     bias = (torch.randn(N, generator=torch.Generator().manual_seed(N)) * 0.05).to(torch.bfloat16)
@@ -252,7 +257,7 @@ def run_qlinear(x_dev, w, bits, Bk, bias_dev, act, N):
     return Y, nat.cpu().numpy()
 
 
-@pytest.mark.parametrize("M,N,K,Bk,bits,mode", [GEMM_CASES[0], GEMM_CASES[3], GEMM_CASES[4]])
+@pytest.mark.parametrize("M,N,K,Bk,bits,mode", [GEMM_CASES[0], GEMM_CASES[3], GEMM_CASES[4], GEMM_CASES[6], GEMM_CASES[7]])
 def test_qlinear_matches_oracle_end_to_end(M, N, K, Bk, bits, mode):
     x, u, d, z, codes, s64, s32, xt = oracle_layer(M, N, K, Bk, bits, mode, seed=7 * M + N)
     out = {"codes": codes, "xt": xt, "scale64": s64, "scale32": s32,
