@@ -370,12 +370,16 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling runs)")
+    ap.add_argument("--bits", type=int, default=0, help="override the activation bit width of every layer (4, 6 or 8)")
     args = ap.parse_args()
     from paper_2505_18663_b200 import workloads as W
     wl = W.WORKLOADS[args.workload]
     if args.tokens > 0:
         import dataclasses
         wl = dataclasses.replace(wl, M=args.tokens)
+    if args.bits > 0:
+        import dataclasses
+        wl = dataclasses.replace(wl, layers=tuple(dataclasses.replace(l, bits=args.bits) for l in wl.layers))
     if args.impl == "reference":
         run_reference(args, wl)
     else:
