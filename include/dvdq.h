@@ -174,6 +174,39 @@ dvdq_status dvdq_qlinear_static(const void* X_bf16, int64_t M, int64_t ldx, cons
                                 const dvdq_weights* w /* host */, const void* bias_bf16, int32_t act,
                                 void* Y_bf16, int64_t ldy, void* cuda_stream);
 
+/* ---- delta-Guided Bit Switching: Sec. 3.3, Eq. "B_{t_i}" ----------------------------------
+ *
+ * The activation bit width of the whole model is chosen per denoising step from the
+ * accumulated relative L1 change of the model output F:
+ *     L1(F, t) = || F_t - F_{t-1} ||_1 / || F_{t-1} ||_1,
+ *     B_{t_i}  = b_low  while  sum_{t = t_p}^{t_{i-1}} L1(F, t) <  delta,
+ *                b_high once   sum                              >= delta  (and the sum restarts at 0).
+ * Reading where the paper is silent: before the first output exists the sum is empty (= 0), so
+ * the first step runs at b_low unless delta == 0; delta == 0 gives b_high on every step.
+ *
+ * dvdq_gbs_l1_terms  one pass over F_t and F_{t-1} (bf16, n elements each, 16-byte aligned):
+ *                    terms_out[0] = || F_t - F_{t-1} ||_1, terms_out[1] = || F_{t-1} ||_1 as
+ *                    fp64 on the DEVICE (two doubles, 8-byte aligned; zeroed by the call).
+ * The state and the three functions below live on the HOST; the caller copies the two terms
+ * back once per step and feeds them to dvdq_gbs_observe. */
+typedef struct {
+    double  delta;        /* threshold on the accumulated relative change */
+    int32_t b_low;        /* bit width of redundant steps: 4, 6 or 8 */
+    int32_t b_high;       /* bit width of critical steps, >= b_low */
+    double  accumulated;  /* sum of L1(F, t) since the last reset */
+    int64_t steps;        /* decisions taken so far */
+    int64_t high_steps;   /* of which b_high */
+} dvdq_gbs_state;
+
+dvdq_status dvdq_gbs_l1_terms(const void* F_t_bf16, const void* F_prev_bf16, int64_t n,
+                              double* terms_out /* device, [2] */, void* cuda_stream);
+dvdq_status dvdq_gbs_init(dvdq_gbs_state* g /* host */, double delta, int32_t b_low, int32_t b_high);
+/* Bit width for the step about to run; resets the sum when it answers b_high.  0 if g is NULL. */
+int32_t dvdq_gbs_next_bits(dvdq_gbs_state* g /* host */);
+/* Adds L1(F, t) = l1_change / l1_prev of the step that just finished.  An all-zero F_{t-1}
+ * counts as relative change 1 if F_t differs from it, else 0. */
+dvdq_status dvdq_gbs_observe(dvdq_gbs_state* g /* host */, double l1_change, double l1_prev);
+
 /* ---- test / debug entry points (so that no caller depends on the packed layouts) ---- */
 
 /* The raw accumulators of dvdq_qgemm: acc_out [M, N] int32, row pitch ldacc elements. */

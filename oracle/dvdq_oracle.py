@@ -206,3 +206,34 @@ def qlinear(x_bf16, u, delta32, z, B: int, bits: int, bias_bf16=None, act: int =
     acc = int_gemm(codes, u, z)
     y = epilogue(acc, s32, delta32, bias_bf16, act)
     return {"xt": xt, "codes": codes, "scale64": s64, "scale32": s32, "acc": acc, "y": y}
+
+
+# ---------------------------------------------------------------- delta-guided bit switching (Sec. 3.3)
+
+def gbs_l1_terms(F_t_bf16: np.ndarray, F_prev_bf16: np.ndarray):
+    """(||F_t - F_{t-1}||_1, ||F_{t-1}||_1) in fp64 from raw bf16 bits: the two norms of
+    L1(F, t) = ||F_t - F_{t-1}||_1 / ||F_{t-1}||_1  (Sec. 3.3)."""
+    a = bf16_array_to_double(F_t_bf16).ravel()
+    b = bf16_array_to_double(F_prev_bf16).ravel()
+    assert a.shape == b.shape
+    return float(np.abs(a - b).sum()), float(np.abs(b).sum())
+
+
+def gbs_schedule(l1_values, delta: float, b_low: int, b_high: int):
+    """Bit width of every step of a run, given L1(F, t) of each finished step, by the rule of
+    Sec. 3.3: step i runs at b_low while the changes summed since the last reset stay below
+    delta; once the sum reaches delta the step runs at b_high and the sum restarts from zero.
+    l1_values[i] is the change measured after step i; the decision for step i only sees the
+    values of earlier steps (the sum is empty, i.e. 0, before the first step).  Returns one
+    entry per step, len(l1_values) + 1 decisions for len(l1_values) observed changes."""
+    bits = []
+    acc = 0.0
+    for i in range(len(l1_values) + 1):
+        if acc >= delta:
+            bits.append(b_high)
+            acc = 0.0
+        else:
+            bits.append(b_low)
+        if i < len(l1_values):
+            acc += float(l1_values[i])
+    return bits

@@ -24,6 +24,7 @@ EXPORTS = [
     "dvdq_qlinear_workspace_bytes", "dvdq_rotate_quantize", "dvdq_pack_weights", "dvdq_qgemm",
     "dvdq_qlinear", "dvdq_qlinear_static", "dvdq_qgemm_int32", "dvdq_pack_act_codes", "dvdq_unpack_act_codes",
     "dvdq_unpack_weights", "dvdq_last_device_status",
+    "dvdq_gbs_l1_terms", "dvdq_gbs_init", "dvdq_gbs_next_bits", "dvdq_gbs_observe",
 ]
 
 
@@ -43,6 +44,12 @@ class Weights(C.Structure):
     _fields_ = [("magic", C.c_uint32), ("version", C.c_uint32), ("N", C.c_int64), ("K", C.c_int64),
                 ("rot_block", C.c_int32), ("k_layout", C.c_int32), ("blob", C.c_void_p),
                 ("blob_bytes", C.c_uint64)]
+
+
+class GbsState(C.Structure):
+    """dvdq_gbs_state: host-side state of the delta-guided bit switching (Sec. 3.3)."""
+    _fields_ = [("delta", C.c_double), ("b_low", C.c_int32), ("b_high", C.c_int32), ("accumulated", C.c_double),
+                ("steps", C.c_int64), ("high_steps", C.c_int64)]
 
 
 _lib = None
@@ -83,6 +90,10 @@ def load():
         "dvdq_unpack_act_codes": (C.c_int, [p, i64, i64, aq, p, p]),
         "dvdq_unpack_weights": (C.c_int, [wp, p, p, p, p]),
         "dvdq_last_device_status": (C.c_int, [C.POINTER(C.c_uint32)]),
+        "dvdq_gbs_l1_terms": (C.c_int, [p, p, i64, p, p]),
+        "dvdq_gbs_init": (C.c_int, [C.POINTER(GbsState), C.c_double, i32, i32]),
+        "dvdq_gbs_next_bits": (i32, [C.POINTER(GbsState)]),
+        "dvdq_gbs_observe": (C.c_int, [C.POINTER(GbsState), C.c_double, C.c_double]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -235,6 +246,30 @@ def dvdq_unpack_weights(w: Weights, Wq: torch.Tensor, delta: torch.Tensor, zero:
         raise TypeError("Wq must be contiguous")
     _check(load().dvdq_unpack_weights(C.byref(w), _ptr(Wq, torch.uint8, "Wq"), _ptr(delta, torch.float32, "delta"),
                                       _ptr(zero, torch.int32, "zero"), _stream(stream)), "dvdq_unpack_weights")
+
+
+def dvdq_gbs_l1_terms(F_t: torch.Tensor, F_prev: torch.Tensor, terms: torch.Tensor, stream=None) -> None:
+    """terms (float64[2], device) <- (||F_t - F_prev||_1, ||F_prev||_1) of two bf16 tensors of equal size."""
+    if F_t.numel() != F_prev.numel() or not F_t.is_contiguous() or not F_prev.is_contiguous():
+        raise TypeError("F_t and F_prev must be contiguous and of equal size")
+    if terms.dtype != torch.float64 or terms.numel() < 2:
+        raise TypeError("terms must hold two float64 values")
+    _check(load().dvdq_gbs_l1_terms(_ptr(F_t, torch.bfloat16, "F_t"), _ptr(F_prev, torch.bfloat16, "F_prev"), F_t.numel(),
+                                    _ptr(terms, torch.float64, "terms"), _stream(stream)), "dvdq_gbs_l1_terms")
+
+
+def dvdq_gbs_init(delta: float, b_low: int, b_high: int) -> GbsState:
+    g = GbsState()
+    _check(load().dvdq_gbs_init(C.byref(g), float(delta), b_low, b_high), "dvdq_gbs_init")
+    return g
+
+
+def dvdq_gbs_next_bits(g: GbsState) -> int:
+    return int(load().dvdq_gbs_next_bits(C.byref(g)))
+
+
+def dvdq_gbs_observe(g: GbsState, l1_change: float, l1_prev: float) -> None:
+    _check(load().dvdq_gbs_observe(C.byref(g), float(l1_change), float(l1_prev)), "dvdq_gbs_observe")
 
 
 def dvdq_last_device_status():

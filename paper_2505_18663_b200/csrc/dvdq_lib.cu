@@ -3,6 +3,7 @@
 // unit, so that the device status word is a single symbol.
 #include "dvdq_common.cuh"
 
+#include "gbs.cuh"
 #include "pack.cuh"
 #include "qgemm.cuh"
 #include "rotate_quantize.cuh"
@@ -274,6 +275,61 @@ dvdq_status dvdq_unpack_weights(const dvdq_weights* w, uint8_t* Wq, float* delta
     unpack_weights_kernel<<<grid_for(w->N * (w->K / 2), 256), 256, 0, (cudaStream_t)stream>>>(
         static_cast<const uint8_t*>(w->blob), w->N, w->K, Wq, delta, zero);
     return cuda_status(cudaGetLastError());
+}
+
+// ---- delta-Guided Bit Switching (Sec. 3.3) ---------------------------------------------
+
+dvdq_status dvdq_gbs_l1_terms(const void* F_t, const void* F_prev, int64_t n, double* terms_out, void* stream) {
+    if (n < 0) return DVDQ_ERR_SHAPE;
+    if (!terms_out) return DVDQ_ERR_NULL;
+    if (!aligned(terms_out, 8)) return DVDQ_ERR_ALIGN;
+    if (n > 0 && (!F_t || !F_prev)) return DVDQ_ERR_NULL;
+    if (n > 0 && (!aligned(F_t, 16) || !aligned(F_prev, 16))) return DVDQ_ERR_ALIGN;
+    dvdq_status s = check_device_arch();
+    if (s != DVDQ_OK) return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(terms_out, 0, 2 * sizeof(double), st) != cudaSuccess) return DVDQ_ERR_CUDA;
+    if (n == 0) return DVDQ_OK;
+    int64_t blocks = (n / 8 + 255) / 256;
+    if (blocks < 1) blocks = 1;
+    if (blocks > 148 * 8) blocks = 148 * 8;
+    gbs_l1_terms_kernel<<<(unsigned)blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(F_t),
+                                                          static_cast<const __nv_bfloat16*>(F_prev), n, terms_out);
+    return cuda_status(cudaGetLastError());
+}
+
+dvdq_status dvdq_gbs_init(dvdq_gbs_state* g, double delta, int32_t b_low, int32_t b_high) {
+    if (!g) return DVDQ_ERR_NULL;
+    if (!(delta >= 0.0)) return DVDQ_ERR_SHAPE;  // also rejects NaN
+    const bool ok_low = b_low == 4 || b_low == 6 || b_low == 8, ok_high = b_high == 4 || b_high == 6 || b_high == 8;
+    if (!ok_low || !ok_high || b_low > b_high) return DVDQ_ERR_BITS;
+    g->delta = delta;
+    g->b_low = b_low;
+    g->b_high = b_high;
+    g->accumulated = 0.0;
+    g->steps = 0;
+    g->high_steps = 0;
+    return DVDQ_OK;
+}
+
+int32_t dvdq_gbs_next_bits(dvdq_gbs_state* g) {
+    if (!g) return 0;
+    g->steps += 1;
+    if (g->accumulated >= g->delta) {  // enough feature change has piled up: one step at b_high, counter back to zero
+        g->accumulated = 0.0;
+        g->high_steps += 1;
+        return g->b_high;
+    }
+    return g->b_low;
+}
+
+dvdq_status dvdq_gbs_observe(dvdq_gbs_state* g, double l1_change, double l1_prev) {
+    if (!g) return DVDQ_ERR_NULL;
+    if (!(l1_change >= 0.0) || !(l1_prev >= 0.0)) return DVDQ_ERR_SHAPE;
+    // an all-zero previous output gives no ratio: count it as no change (0/0) or as a full change (x/0)
+    const double rel = l1_prev > 0.0 ? l1_change / l1_prev : (l1_change > 0.0 ? 1.0 : 0.0);
+    g->accumulated += rel;
+    return DVDQ_OK;
 }
 
 dvdq_status dvdq_last_device_status(uint32_t* detail) {
