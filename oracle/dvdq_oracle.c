@@ -196,6 +196,113 @@ void oracle_weight_quantize_symmetric(const double* wt, int64_t N, int64_t K,
     }
 }
 
+/* ---------------------------------------------------------------- Bounded-init Grid Refinement (Alg. 1, Sec. 3.1) */
+
+/* Quant of Sec. 3.1 for one row with a given grid (Delta, z); returns the squared error
+ * || w - Delta (W_q - z) ||^2 and, if the pointers are not NULL, the three row sums the
+ * refinement formulas need:  <W_q - z, w>,  <W_q - z, W_q - z>,  sum of W_q. */
+static double bgr_row_quantize(const double* w, int64_t K, double levels, double d, double z,
+                               uint8_t* u_or_null, double* s_qw, double* s_qq, double* s_q) {
+    double e2 = 0.0, qw = 0.0, qq = 0.0, sq = 0.0;
+    for (int64_t k = 0; k < K; ++k) {
+        double c = nearbyint(w[k] / d) + z;
+        if (c < 0.0) c = 0.0;
+        if (c > levels) c = levels;
+        double q = c - z;
+        double r = w[k] - d * q;
+        e2 += r * r; qw += q * w[k]; qq += q * q; sq += c;
+        if (u_or_null) u_or_null[k] = (uint8_t)c;
+    }
+    if (s_qw) *s_qw = qw;
+    if (s_qq) *s_qq = qq;
+    if (s_q) *s_q = sq;
+    return e2;
+}
+
+/* Alg. 1 for every row (output channel) on its own: the objective of Sec. 3.1,
+ * || W - Delta (W_q - z) ||_F with one (Delta, z) per row, separates over rows.
+ *
+ *   for i = 1, 2, ... (shrink steps, delta_l = delta_u = (max - min) / n_steps):
+ *       clip the row to [min + i delta_l, max - i delta_u]; MinMax grid of the clipped row
+ *       (Delta(0), z(0)); quantize the UNclipped row on it; then repeat
+ *           Delta' = <W_q - z, w> / <W_q - z, W_q - z>                  (least squares, z and W_q fixed)
+ *           z'     = clamp(round(mean(W_q) - mean(w) / Delta'), 0, 2^b - 1)  (relax, then round)
+ *           W_q'   = clamp(round(w / Delta') + z', 0, 2^b - 1)
+ *       until the error stops falling by at least eps; keep the best grid seen.
+ *
+ * Readings where Alg. 1 cannot be taken literally:
+ *   - it uses one letter for the number of rows and for the number of shrink steps: n_steps here;
+ *   - its bounds cross once 2 i >= n_steps, so i stops before that;
+ *   - its stopping test, E(j-1) - E(j-2) < eps, holds at once for any falling error: the loop
+ *     here stops when the improvement E(j-1) - E(j) drops below eps (or after max_iter rounds);
+ *   - the text says z is rounded after the relaxation, the formula omits the rounding: rounded here;
+ *   - the candidate of a shrink step is its lowest-error iterate, and a z(0) outside [0, 2^b - 1]
+ *     is pulled into that range (the code format has no other zero points).
+ * bits is a parameter so that a 2-bit example can be worked by hand; the method uses b = 4.
+ * Outputs: u [N,K] codes, delta [N] (double), zero [N], err [N] = final row error (not squared). */
+void oracle_bgr_quantize(const double* wt, int64_t N, int64_t K, int bits, int n_steps, double eps, int max_iter,
+                         uint8_t* u, double* delta, int32_t* zero, double* err) {
+    const double levels = (double)((1 << bits) - 1);
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+        const double* w = wt + n * K;
+        double lo = w[0], hi = w[0], mean = 0.0;
+        for (int64_t k = 0; k < K; ++k) { if (w[k] < lo) lo = w[k]; if (w[k] > hi) hi = w[k]; mean += w[k]; }
+        mean /= (double)K;
+        double best_e2 = INFINITY, best_d = 1.0, best_z = 0.0;
+        const double step = (hi - lo) / (double)n_steps;
+        for (int i = 1; 2 * i < n_steps && hi > lo; ++i) {
+            const double lo_c = lo + i * step, hi_c = hi - i * step;   /* min and max of the clipped row */
+            double d = (hi_c - lo_c) / levels;
+            double z = -nearbyint(lo_c / d);
+            if (z < 0.0) z = 0.0;
+            if (z > levels) z = levels;
+            double qw, qq, sq;
+            double e2 = bgr_row_quantize(w, K, levels, d, z, NULL, &qw, &qq, &sq);
+            if (e2 < best_e2) { best_e2 = e2; best_d = d; best_z = z; }
+            for (int j = 1; j <= max_iter; ++j) {
+                if (!(qq > 0.0) || !(qw > 0.0)) break;      /* no usable least-squares step */
+                const double d1 = qw / qq;
+                double z1 = nearbyint(sq / (double)K - mean / d1);
+                if (z1 < 0.0) z1 = 0.0;
+                if (z1 > levels) z1 = levels;
+                const double e2_1 = bgr_row_quantize(w, K, levels, d1, z1, NULL, &qw, &qq, &sq);
+                const double improvement = sqrt(e2) - sqrt(e2_1);
+                d = d1; z = z1; e2 = e2_1;
+                if (e2 < best_e2) { best_e2 = e2; best_d = d; best_z = z; }
+                if (improvement < eps) break;
+            }
+        }
+        if (!(best_e2 < INFINITY)) {                            /* constant row, or n_steps < 3 */
+            best_d = (fabs(hi) > 0.0) ? fabs(hi) : 1.0;
+            best_z = 0.0;
+            if (hi > lo) { best_d = (hi - lo) / levels; best_z = -nearbyint(lo / best_d); if (best_z < 0.0) best_z = 0.0; if (best_z > levels) best_z = levels; }
+            best_e2 = bgr_row_quantize(w, K, levels, best_d, best_z, NULL, NULL, NULL, NULL);
+        }
+        best_e2 = bgr_row_quantize(w, K, levels, best_d, best_z, u + n * K, NULL, NULL, NULL);
+        delta[n] = best_d;
+        zero[n] = (int32_t)best_z;
+        err[n] = sqrt(best_e2);
+    }
+}
+
+/* The error of the plain MinMax grid of Sec. 3.1 for every row, for comparisons with the above. */
+void oracle_minmax_row_error(const double* wt, int64_t N, int64_t K, int bits, double* err) {
+    const double levels = (double)((1 << bits) - 1);
+#pragma omp parallel for schedule(static)
+    for (int64_t n = 0; n < N; ++n) {
+        const double* w = wt + n * K;
+        double lo = w[0], hi = w[0];
+        for (int64_t k = 1; k < K; ++k) { if (w[k] < lo) lo = w[k]; if (w[k] > hi) hi = w[k]; }
+        double d = (hi - lo) / levels;
+        if (!(d > 0.0)) { err[n] = 0.0; continue; }
+        double z = -nearbyint(lo / d);
+        if (z < 0.0) z = 0.0;
+        if (z > levels) z = levels;
+        err[n] = sqrt(bgr_row_quantize(w, K, levels, d, z, NULL, NULL, NULL, NULL));
+    }
+}
+
 /* ---------------------------------------------------------------- integer GEMM */
 
 /* acc_in = sum_k c_ik * (u_nk - z_n)   (the integer core of Y = X^ Lambda W^^T, Eq. 10).

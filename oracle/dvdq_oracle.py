@@ -55,6 +55,10 @@ def _load():
             lib.oracle_weight_quantize_minmax.argtypes = [p, i64, i64, p, p, p]
             lib.oracle_weight_quantize_symmetric.restype = None
             lib.oracle_weight_quantize_symmetric.argtypes = [p, i64, i64, p, p, p]
+            lib.oracle_bgr_quantize.restype = None
+            lib.oracle_bgr_quantize.argtypes = [p, i64, i64, C.c_int, C.c_int, C.c_double, C.c_int, p, p, p, p]
+            lib.oracle_minmax_row_error.restype = None
+            lib.oracle_minmax_row_error.argtypes = [p, i64, i64, C.c_int, p]
             lib.oracle_int_gemm.restype = i64
             lib.oracle_int_gemm.argtypes = [p, p, p, i64, i64, i64, p]
             lib.oracle_gelu_tanh.restype = C.c_double
@@ -154,6 +158,28 @@ def weight_quantize(wt: np.ndarray, mode: str = "symmetric"):
           "minmax": _load().oracle_weight_quantize_minmax}[mode]
     fn(_ptr(wt), N, K, _ptr(u), _ptr(d), _ptr(z))
     return u, d, z
+
+
+def bgr_quantize(wt: np.ndarray, bits: int = 4, n_steps: int = 100, eps: float = 1e-5, max_iter: int = 50):
+    """Bounded-init Grid Refinement (Alg. 1) per output channel ->
+    (u uint8 [N,K], delta fp64 [N], z int32 [N], err fp64 [N] = || w - Delta (u - z) ||_2 per row)."""
+    wt = _c(wt, np.float64)
+    N, K = wt.shape
+    u = np.empty((N, K), dtype=np.uint8)
+    d = np.empty(N, dtype=np.float64)
+    z = np.empty(N, dtype=np.int32)
+    e = np.empty(N, dtype=np.float64)
+    _load().oracle_bgr_quantize(_ptr(wt), N, K, bits, n_steps, float(eps), max_iter, _ptr(u), _ptr(d), _ptr(z), _ptr(e))
+    return u, d, z, e
+
+
+def minmax_row_error(wt: np.ndarray, bits: int = 4) -> np.ndarray:
+    """|| w - Delta (W_q - z) ||_2 per row for the plain MinMax grid of Sec. 3.1."""
+    wt = _c(wt, np.float64)
+    N, K = wt.shape
+    e = np.empty(N, dtype=np.float64)
+    _load().oracle_minmax_row_error(_ptr(wt), N, K, bits, _ptr(e))
+    return e
 
 
 def int_gemm(codes: np.ndarray, u: np.ndarray, z: np.ndarray) -> np.ndarray:
