@@ -125,6 +125,28 @@ dvdq_status dvdq_pack_weights(const uint8_t* Wq, const float* delta, const int32
                               int64_t N, int64_t K, int32_t rot_block,
                               void* blob_out, dvdq_weights* out /* host */, void* cuda_stream);
 
+/* ---- (0') offline weight quantizer: Bounded-init Grid Refinement, Alg. 1 / Sec. 3.1 ---------
+ *
+ * For every output channel (row) on its own -- the objective || W - Delta (W_q - z) ||_F with
+ * one (Delta, z) per row separates over rows -- and for every shrink step i = 1, 2, ... with
+ * delta_l = delta_u = (max - min) / n_steps:
+ *     clip the row to [min + i delta_l, max - i delta_u]; MinMax grid of the clipped row;
+ *     quantize the unclipped row on it; then repeat
+ *         Delta' = <W_q - z, w> / <W_q - z, W_q - z>,
+ *         z'     = clamp(round(mean(W_q) - mean(w) / Delta'), 0, 15),
+ *         W_q'   = clamp(round(w / Delta') + z', 0, 15)
+ *     until the row error improves by less than eps (or max_iter rounds); the best grid seen wins.
+ * (Alg. 1 as printed reuses one letter for rows and shrink steps, lets its bounds cross, and
+ * stops on a test that is true at once; the statement above is the reading built here.)
+ *
+ *   W_rot      [N, K] fp32, row-major, dense: the weights ALREADY rotated (W~ = W R)
+ *   n_steps    shrink steps across the row's range (the paper's n; e.g. 100); eps >= 0; max_iter >= 0
+ *   Wq_out     [N, K] uint8 codes 0..15, delta_out [N] fp32, zero_out [N] int32 0..15:
+ *              exactly the inputs of dvdq_pack_weights
+ * All arithmetic is fp64 (round half to even).  K % 64 == 0, K <= 16384. */
+dvdq_status dvdq_bgr_quantize(const float* W_rot, int64_t N, int64_t K, int32_t n_steps, double eps, int32_t max_iter,
+                              uint8_t* Wq_out, float* delta_out, int32_t* zero_out, void* cuda_stream);
+
 /* ---- (2) low-bit GEMM + dequantizing epilogue: Eq. 10, Y = X^ Lambda W^^T ----------
  *
  *   acc_in = sum_k c_ik (u_nk - z_n)      exact int32 (tensor cores, int8 operands)

@@ -24,7 +24,7 @@ EXPORTS = [
     "dvdq_qlinear_workspace_bytes", "dvdq_rotate_quantize", "dvdq_pack_weights", "dvdq_qgemm",
     "dvdq_qlinear", "dvdq_qlinear_static", "dvdq_qgemm_int32", "dvdq_pack_act_codes", "dvdq_unpack_act_codes",
     "dvdq_unpack_weights", "dvdq_last_device_status",
-    "dvdq_gbs_l1_terms", "dvdq_gbs_init", "dvdq_gbs_next_bits", "dvdq_gbs_observe",
+    "dvdq_bgr_quantize", "dvdq_gbs_l1_terms", "dvdq_gbs_init", "dvdq_gbs_next_bits", "dvdq_gbs_observe",
 ]
 
 
@@ -90,6 +90,7 @@ def load():
         "dvdq_unpack_act_codes": (C.c_int, [p, i64, i64, aq, p, p]),
         "dvdq_unpack_weights": (C.c_int, [wp, p, p, p, p]),
         "dvdq_last_device_status": (C.c_int, [C.POINTER(C.c_uint32)]),
+        "dvdq_bgr_quantize": (C.c_int, [p, i64, i64, i32, C.c_double, i32, p, p, p, p]),
         "dvdq_gbs_l1_terms": (C.c_int, [p, p, i64, p, p]),
         "dvdq_gbs_init": (C.c_int, [C.POINTER(GbsState), C.c_double, i32, i32]),
         "dvdq_gbs_next_bits": (i32, [C.POINTER(GbsState)]),
@@ -246,6 +247,17 @@ def dvdq_unpack_weights(w: Weights, Wq: torch.Tensor, delta: torch.Tensor, zero:
         raise TypeError("Wq must be contiguous")
     _check(load().dvdq_unpack_weights(C.byref(w), _ptr(Wq, torch.uint8, "Wq"), _ptr(delta, torch.float32, "delta"),
                                       _ptr(zero, torch.int32, "zero"), _stream(stream)), "dvdq_unpack_weights")
+
+
+def dvdq_bgr_quantize(W_rot: torch.Tensor, n_steps: int, eps: float, max_iter: int, Wq: torch.Tensor,
+                      delta: torch.Tensor, zero: torch.Tensor, stream=None) -> None:
+    """Bounded-init Grid Refinement of rotated fp32 weights [N, K] -> (Wq uint8, delta fp32, zero int32)."""
+    if W_rot.dim() != 2 or not W_rot.is_contiguous() or not Wq.is_contiguous():
+        raise TypeError("W_rot and Wq must be dense [N, K]")
+    N, K = W_rot.shape
+    _check(load().dvdq_bgr_quantize(_ptr(W_rot, torch.float32, "W_rot"), N, K, n_steps, float(eps), max_iter,
+                                    _ptr(Wq, torch.uint8, "Wq"), _ptr(delta, torch.float32, "delta"),
+                                    _ptr(zero, torch.int32, "zero"), _stream(stream)), "dvdq_bgr_quantize")
 
 
 def dvdq_gbs_l1_terms(F_t: torch.Tensor, F_prev: torch.Tensor, terms: torch.Tensor, stream=None) -> None:

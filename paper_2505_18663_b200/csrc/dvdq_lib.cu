@@ -3,6 +3,7 @@
 // unit, so that the device status word is a single symbol.
 #include "dvdq_common.cuh"
 
+#include "bgr.cuh"
 #include "gbs.cuh"
 #include "pack.cuh"
 #include "qgemm.cuh"
@@ -274,6 +275,28 @@ dvdq_status dvdq_unpack_weights(const dvdq_weights* w, uint8_t* Wq, float* delta
     if ((s = check_device_arch()) != DVDQ_OK) return s;
     unpack_weights_kernel<<<grid_for(w->N * (w->K / 2), 256), 256, 0, (cudaStream_t)stream>>>(
         static_cast<const uint8_t*>(w->blob), w->N, w->K, Wq, delta, zero);
+    return cuda_status(cudaGetLastError());
+}
+
+// ---- Bounded-init Grid Refinement (Alg. 1) ------------------------------------------------
+
+dvdq_status dvdq_bgr_quantize(const float* W_rot, int64_t N, int64_t K, int32_t n_steps, double eps, int32_t max_iter,
+                              uint8_t* Wq_out, float* delta_out, int32_t* zero_out, void* stream) {
+    if (N < 0 || N > 0x7FFFFFFFll || validate_k(K) != DVDQ_OK || n_steps < 1 || max_iter < 0 || !(eps >= 0.0)) return DVDQ_ERR_SHAPE;
+    if (N == 0) return DVDQ_OK;
+    if (!W_rot || !Wq_out || !delta_out || !zero_out) return DVDQ_ERR_NULL;
+    if (!aligned(W_rot, 4) || !aligned(delta_out, 4) || !aligned(zero_out, 4)) return DVDQ_ERR_ALIGN;
+    dvdq_status s = check_device_arch();
+    if (s != DVDQ_OK) return s;
+    const size_t smem = (size_t)K * sizeof(float);
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(bgr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 16384 * (int)sizeof(float)) != cudaSuccess)
+            return DVDQ_ERR_CUDA;
+        attr_set = true;
+    }
+    bgr_kernel<<<(unsigned)N, kBgrThreads, smem, (cudaStream_t)stream>>>(W_rot, (int)K, n_steps, eps, max_iter, Wq_out,
+                                                                         delta_out, zero_out);
     return cuda_status(cudaGetLastError());
 }
 
