@@ -57,7 +57,7 @@ __device__ __forceinline__ uint32_t stage_a_entry(int m, int s) {
 // iteration i are finalised after the barrier of iteration i + 1 from double-buffered slots.
 template <int LOG2B, int BITS, bool FULL>
 __global__ void __maxnreg__(80)  // two CTAs of 12 warps per SM
-rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
+rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
           uint8_t* __restrict__ codes, float* __restrict__ scales, int32_t* __restrict__ sums,
           int spans, int tokens_per_cta, int num_groups) {
     extern __shared__ float4 s_turn[];  // 256 float4 per warp
@@ -106,13 +106,17 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
         wr[1] = (b34 + 4) * 8 + (low ^ 4);
     }
     const int rd = lane * 8 + (lane & 7);
-    const int64_t row_bytes = act_row_bytes(K, BITS);
+    const int row_bytes = (int)act_row_bytes(K, BITS);
+    // byte offsets of the lane's first output word (+ 32 j, or + 64 j for 8-bit codes) and of its
+    // first high-plane word (+ 16 j): everything else in the loop is one 32 x 32 -> 64 bit multiply-add
+    const int st_b0 = BITS == 8 ? st_e0 : st_e0 >> 1;
+    const int st_h0 = (K >> 1) + ((st_e0 >> 4) << 2);
     const float rs = (LOG2B & 1) ? rsqrtf((float)(1 << LOG2B)) : 1.0f / (float)(1 << (LOG2B / 2));
 
     auto load_span = [&](uint4 (&raw)[4], int group) {
-        int64_t token = (int64_t)group * tokens_per_cta + tl;
-        if (token >= M) token = M - 1;  // a clamped duplicate; its results are never stored
-        const uint4* src = reinterpret_cast<const uint4*>(X + token * ldx + ld_e0);
+        int token = group * tokens_per_cta + tl;
+        if (token >= M) token = M - 1;  // a clamped duplicate
+        const uint4* src = reinterpret_cast<const uint4*>(X + ((int64_t)token * ldx + ld_e0));
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             raw[c] = make_uint4(0u, 0u, 0u, 0u);
@@ -123,14 +127,14 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
     uint4 raw[4];
     int group = blockIdx.x;
     if (group < num_groups) load_span(raw, group);
-    int64_t prev_token = -1;
+    int prev_token = -1;
     float prev_amax = 0.f;
     uint32_t it = 0;
     for (; group < num_groups; group += gridDim.x, ++it) {
         const uint32_t buf = it & 1u;
         // A token past the end is a clamped duplicate of the last one: it computes and stores
         // the same bytes to the same places, which needs no predicate.
-        int64_t token = (int64_t)group * tokens_per_cta + tl;
+        int token = group * tokens_per_cta + tl;
         if (token >= M) token = M - 1;
 
         // ---- stage A: D = H_16 * B on index bits {0, 3, 4, 1} (k-slot bit 0 = half of a word,
@@ -263,7 +267,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
         const uint64_t inv2 = f2_pack(inv, inv), magic2 = f2_pack(kMagic, kMagic);
 
         // ---- quantize, sum, pack, store
-        uint8_t* crow = codes + token * row_bytes;
+        uint8_t* crow = codes + (int64_t)token * row_bytes;
         int lsum = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -290,23 +294,22 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int64_t M, int K, int64_t ldx,
             const uint32_t O = __byte_perm(__byte_perm(b[1], b[3], 0x0040), __byte_perm(b[5], b[7], 0x0040), 0x5410);
             lsum = __dp4a((int)E, 0x01010101, lsum);
             lsum = __dp4a((int)O, 0x01010101, lsum);
-            const int e0 = st_e0 + j * 64;
             const bool ok = FULL || (st_ok >> j & 1u);
             if (BITS == 8) {
                 // 8-bit codes: each group of 8 channels is stored as the word of its even channels
                 // followed by the word of its odd channels, the order the GEMM consumes
-                if (ok) *reinterpret_cast<uint2*>(crow + e0) = make_uint2(E, O);
+                if (ok) *reinterpret_cast<uint2*>(crow + st_b0 + 64 * j) = make_uint2(E, O);
                 continue;
             }
             const uint32_t lo = (E & 0x0F0F0F0Fu) | ((O << 4) & 0xF0F0F0F0u);
-            if (ok) *reinterpret_cast<uint32_t*>(crow + (e0 >> 1)) = lo;
+            if (ok) *reinterpret_cast<uint32_t*>(crow + st_b0 + 32 * j) = lo;
             if (BITS == 6) {
                 // bits 5:4 of 16 consecutive channels share one word of the high plane; the two
                 // halves sit in neighbouring lanes
                 uint32_t hi = ((E >> 4) & 0x03030303u) | ((O >> 2) & 0x0C0C0C0Cu);
                 hi <<= 4 * (lane & 1);
                 hi |= __shfl_xor_sync(0xFFFFFFFFu, hi, 1);
-                if (ok && ((j ^ lane) & 1) == 0) *reinterpret_cast<uint32_t*>(crow + (K >> 1) + ((e0 >> 4) << 2)) = hi;
+                if (ok && ((j ^ lane) & 1) == 0) *reinterpret_cast<uint32_t*>(crow + st_h0 + 16 * j) = hi;
             }
         }
         lsum = __reduce_add_sync(0xFFFFFFFFu, lsum);
@@ -336,7 +339,7 @@ static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t
     const int threads = warps * 32;
     const size_t smem = (size_t)warps * 256 * sizeof(float4);
     const int64_t groups = (M + tpc - 1) / tpc;
-    if (groups > 0x7FFFFFFFll) return DVDQ_ERR_SHAPE;
+    if (M > 0x7FFFFF00ll || ldx > 0x7FFFFFFFll || groups * tpc > 0x7FFFFFFFll) return DVDQ_ERR_SHAPE;
     auto kern = rq_kernel<LOG2B, BITS, FULL>;
     static bool attr_set = false;
     static int sm_count = 0;
@@ -357,7 +360,7 @@ static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t
     }
     const int64_t resident = (int64_t)sm_count * blocks_per_sm[warps];
     const unsigned grid = (unsigned)(groups < resident ? groups : resident);
-    kern<<<grid, threads, smem, st>>>((const __nv_bfloat16*)X, M, (int)K, ldx, (uint8_t*)codes, scales, sums, spans, tpc,
+    kern<<<grid, threads, smem, st>>>((const __nv_bfloat16*)X, (int)M, (int)K, (int)ldx, (uint8_t*)codes, scales, sums, spans, tpc,
                                       (int)groups);
     return cuda_status(cudaGetLastError());
 }
