@@ -51,7 +51,7 @@ constexpr int kWPackedStages = 6;   // ring of packed weight half-tiles (one k-b
 constexpr int kUnpackGroups = 2;   // unpack warps come in groups that take alternate k-blocks
 constexpr int kAWarps = 4 * kUnpackGroups, kWWarps = 4 * kUnpackGroups, kEpilogueWarps = 4;
 constexpr int kFirstEpilogueWarp = 2, kFirstAWarp = 6, kFirstWWarp = kFirstAWarp + kAWarps;
-constexpr int kStageArrivals = (kAWarps + kWWarps) / kUnpackGroups;  // unpack warps working on one k-block, per CTA
+constexpr int kStageArrivals = (kAWarps + kWWarps) / kUnpackGroups;  // unpack warps that fill one wide stage, per CTA
 constexpr int kGemmThreads = (2 + kEpilogueWarps + kAWarps + kWWarps) * 32;
 constexpr int kTmemCols = 512;
 constexpr int kTmemACol = 2 * kBN;  // first column of the activation stages
