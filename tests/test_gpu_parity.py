@@ -319,12 +319,19 @@ def test_ffn_chain_stage_by_stage():
 
 # ------------------------------------------------------------------ full-size launch configuration, sampled rows
 
-@pytest.mark.parametrize("layer_idx", [0, 3])
-def test_full_size_hunyuan_layer_on_sampled_rows(layer_idx):
-    """The benchmark's launch configuration (M = 65536 tokens, HunyuanVideo-shaped layer):
-    scales, codes, accumulators-through-bf16 on sampled rows (first tile, last tile, seeded
-    rows), computed one row at a time by the oracle."""
-    wl = W.WORKLOADS["hunyuan"]
+FULL_SIZE_CASES = [
+    # workload, layer: the benchmark's own launch configurations plus the ragged ones of the other
+    # configs (M = 32760 = 127 * 256 + 248 tokens, K = 1536 / 13824 with a partial last span, A6)
+    ("hunyuan", 0), ("hunyuan", 3), ("wan1p3b", 2), ("wan14b", 3), ("ffn_chain", 1),
+]
+
+
+@pytest.mark.parametrize("workload,layer_idx", FULL_SIZE_CASES)
+def test_full_size_layer_on_sampled_rows(workload, layer_idx):
+    """Full token counts of the benchmark configurations: scales, codes and bf16 outputs on
+    sampled rows (first tile, last full tile, ragged tail, seeded rows), computed one row at a
+    time by the oracle; plus a property of the whole output."""
+    wl = W.WORKLOADS[workload]
     layer = wl.layers[layer_idx]
     M = wl.M
     x = W.make_activations(wl, layer.K, device=DEV)
@@ -334,17 +341,21 @@ def test_full_size_hunyuan_layer_on_sampled_rows(layer_idx):
     q = act_quant(layer.bits, layer.rot_block)
     ws = torch.empty(B.dvdq_qlinear_workspace_bytes(M, layer.K, q), dtype=torch.uint8, device=DEV)
     Y = torch.empty(M, layer.N, dtype=torch.bfloat16, device=DEV)
-    B.dvdq_qlinear(x, q, w, None, 0, Y, ws)
+    bias = W.make_bias(wl, layer, device=DEV)
+    B.dvdq_qlinear(x, q, w, bias, layer.act, Y, ws)
     assert_device_ok()
-    rows = W.sample_rows(M, 48, seed=layer_idx)
+    rows = W.sample_rows(M, 40, tile=256, seed=layer_idx)
     xs = x[rows.to(DEV)].cpu()
-    out = orc.qlinear(to_bits(xs), u.cpu().numpy(), d.cpu().numpy(), z.cpu().numpy(), layer.rot_block, layer.bits)
-    # the workspace starts with the packed codes of every token
+    un, dn, zn = u.cpu().numpy(), d.cpu().numpy(), z.cpu().numpy()
+    bias_bits = None if bias is None else to_bits(bias)
+    out = orc.qlinear(to_bits(xs), un, dn, zn, layer.rot_block, layer.bits, bias_bits, layer.act)
+    # the workspace starts with the packed codes of every token; unpack only the sampled rows' worth
     nat = torch.empty(M, layer.K, dtype=torch.int8, device=DEV)
     B.dvdq_unpack_act_codes(ws, M, layer.K, q, nat)
     nat_s = nat[rows.to(DEV)].cpu().numpy()
+    del nat
     y = Y[rows.to(DEV)].to(torch.float64).cpu().numpy()
-    y_or = oracle_y_for_validated_codes(nat_s, out, u.cpu().numpy(), d.cpu().numpy(), z.cpu().numpy())
+    y_or = oracle_y_for_validated_codes(nat_s, out, un, dn, zn, bias_bits, layer.act)
     assert np.abs(y - y_or).max() <= Y_MAXNORM_RTOL * np.abs(y_or).max()
     # a property that holds at any size: no NaN/Inf anywhere in the full output
     assert bool(torch.isfinite(Y).all())
