@@ -57,6 +57,7 @@ constexpr int kTmemCols = 512;
 constexpr int kTmemACol = 2 * kBN;  // first column of the activation stages
 constexpr int kAColsPerStage = kBK / 4;
 static_assert(kTmemACol + kWideStages * kAColsPerStage <= kTmemCols, "tensor memory budget");
+static_assert(kWideStages % 2 == 0, "the MMA warp takes the wide stages in pairs");
 
 template <int BITS>
 struct GemmSmem {
@@ -210,19 +211,27 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 if (!mbar_wait_warp(acc_empty(a), aph ^ 1u, abort_flag, kWaitAccEmpty)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + a * kBN;
-                for (int kb = 0; kb < KB; ++kb) {
+                // Two k-blocks per trip (KB is even, and so is kWideStages): the tensor core's queue
+                // is short, so every cycle this warp spends between two issues is a bubble in the
+                // MMA stream; pairing halves the waits, votes and bookkeeping per k-block.
+                for (int kb = 0; kb < KB; kb += 2) {
                     if (!mbar_wait_warp(wd_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
+                    if (!mbar_wait_warp(wd_full(st + 1), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_tmem = tmem_base + kTmemACol + st * kAColsPerStage;
-                    const uint64_t bdesc = umma_desc_sw128_kmajor(sbase + S::kWideOff + st * S::kWideW);
                     if (elect_one()) {
 #pragma unroll
-                        for (int k = 0; k < kBK / 32; ++k)  // +32 int8 along K = +8 columns of A, +2 in B's 16-byte address field
-                            tc_mma_i8_ts_pair(d_tmem, a_tmem + 8u * k, bdesc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                        tc_commit_pair(wd_empty(st), 3);
+                        for (int h = 0; h < 2; ++h) {
+                            const uint32_t a_tmem = tmem_base + kTmemACol + (st + h) * kAColsPerStage;
+                            const uint64_t bdesc = umma_desc_sw128_kmajor(sbase + S::kWideOff + (st + h) * S::kWideW);
+#pragma unroll
+                            for (int k = 0; k < kBK / 32; ++k)  // +32 int8 along K = +8 columns of A, +2 in B's 16-byte address field
+                                tc_mma_i8_ts_pair(d_tmem, a_tmem + 8u * k, bdesc + 2u * k, idesc, (kb | h | k) != 0 ? 1u : 0u);
+                            tc_commit_pair(wd_empty(st + h), 3);
+                        }
                     }
                     __syncwarp();
-                    if (++st == kWideStages) { st = 0; ph ^= 1u; }
+                    st += 2;
+                    if (st == kWideStages) { st = 0; ph ^= 1u; }
                 }
                 if (ok && elect_one()) tc_commit_pair(acc_full(a), 3);
                 __syncwarp();
@@ -248,12 +257,23 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
             const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM, n0 = (tile % num_n) * kBN;
             __syncwarp();
-            for (int c = lane; c < kBN; c += 32) {
-                const int n = n0 + c;
-                const bool okn = n < N;
-                sts32f(c_delta + 4 * c, okn ? delta[n] : 0.f);
-                sts32f(c_zc + 4 * c, okn ? (float)zc[n] : 0.f);
-                sts32f(c_bias + 4 * c, (okn && bias != nullptr) ? __bfloat162float(bias[n]) : 0.f);
+            {   // per-channel constants of this tile: all loads in flight at once, then the stores
+                float cd[kBN / 32], cz[kBN / 32], cb[kBN / 32];
+#pragma unroll
+                for (int i = 0; i < kBN / 32; ++i) {
+                    const int n = n0 + lane + 32 * i;
+                    const bool okn = n < N;
+                    cd[i] = okn ? __ldg(delta + n) : 0.f;
+                    cz[i] = okn ? (float)__ldg(zc + n) : 0.f;
+                    cb[i] = (okn && bias != nullptr) ? __bfloat162float(bias[n]) : 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < kBN / 32; ++i) {
+                    const int c = lane + 32 * i;
+                    sts32f(c_delta + 4 * c, cd[i]);
+                    sts32f(c_zc + 4 * c, cz[i]);
+                    sts32f(c_bias + 4 * c, cb[i]);
+                }
             }
             __syncwarp();
             if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) break;
