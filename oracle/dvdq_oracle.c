@@ -350,6 +350,20 @@ void oracle_epilogue(const int32_t* acc, const float* scale, const float* delta,
     }
 }
 
+/* The tail of the epilogue for values already dequantized in fp64 (used by the block-wise
+ * variant, whose sum over blocks is formed before): y = bf16(v + bias) [GELU, bf16 again]. */
+void oracle_round_output(const double* v, const uint16_t* bias_or_null, int act, int64_t M, int64_t N, uint16_t* y) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t n = 0; n < N; ++n) {
+            double t = v[i * N + n];
+            if (bias_or_null) t += oracle_bf16_to_double(bias_or_null[n]);
+            uint16_t h = oracle_double_to_bf16(t);
+            if (act == 1) h = oracle_double_to_bf16(oracle_gelu_tanh(oracle_bf16_to_double(h)));
+            y[i * N + n] = h;
+        }
+}
+
 /* The exact product the method approximates, Y = X W^T in fp64 (Sec. 3.2), for the
  * invariance and convergence checks. */
 void oracle_exact_linear(const double* x, const double* w, int64_t M, int64_t N, int64_t K, double* y) {

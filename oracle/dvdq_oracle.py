@@ -65,6 +65,8 @@ def _load():
             lib.oracle_gelu_tanh.argtypes = [C.c_double]
             lib.oracle_epilogue.restype = None
             lib.oracle_epilogue.argtypes = [p, p, p, p, C.c_int, i64, i64, p]
+            lib.oracle_round_output.restype = None
+            lib.oracle_round_output.argtypes = [p, p, C.c_int, i64, i64, p]
             lib.oracle_exact_linear.restype = None
             lib.oracle_exact_linear.argtypes = [p, p, i64, i64, i64, p]
             _lib = lib
@@ -263,3 +265,46 @@ def gbs_schedule(l1_values, delta: float, b_low: int, b_high: int):
         if i < len(l1_values):
             acc += float(l1_values[i])
     return bits
+
+
+# ---------------------------------------------------------------- block-wise scales (Sec. 3.2, last paragraph)
+
+def act_quantize_grouped(xt: np.ndarray, bits: int, group: int):
+    """The block-wise variant of the auto-scaling: one absmax scale per token AND per block of
+    `group` consecutive rotated channels (the quantizer of Eq. 10 applied to every block on its
+    own).  Returns (codes int32 [M,K], scale fp64 [M,K/group], scale fp32 [M,K/group])."""
+    xt = _c(xt, np.float64)
+    M, K = xt.shape
+    assert group > 0 and K % group == 0
+    G = K // group
+    codes = np.empty((M, K), dtype=np.int32)
+    s64 = np.empty((M, G), dtype=np.float64)
+    s32 = np.empty((M, G), dtype=np.float32)
+    for g in range(G):
+        c, a, b = act_quantize(xt[:, g * group:(g + 1) * group], bits)
+        codes[:, g * group:(g + 1) * group] = c
+        s64[:, g] = a
+        s32[:, g] = b
+    return codes, s64, s32
+
+
+def qlinear_grouped(x_bf16, u, delta32, z, B: int, bits: int, group: int, bias_bf16=None, act: int = 0):
+    """The layer with block-wise activation scales:
+        y_in = bf16( Delta_n * sum_g s_ig * sum_{k in block g} c_ik (u_nk - z_n) + bias_n ),
+    every block's integer GEMM on its own, combined in fp64 (scales and Delta are their stored
+    binary32 values), then the same rounding / GELU as the per-token path."""
+    xt = rotate(x_bf16, B)
+    codes, s64, s32 = act_quantize_grouped(xt, bits, group)
+    M, K = codes.shape
+    N = u.shape[0]
+    v = np.zeros((M, N), dtype=np.float64)
+    for g in range(K // group):
+        sl = slice(g * group, (g + 1) * group)
+        acc = int_gemm(codes[:, sl], np.ascontiguousarray(u[:, sl]), z)
+        v += acc.astype(np.float64) * s32[:, g].astype(np.float64)[:, None]
+    v *= np.asarray(delta32, dtype=np.float32).astype(np.float64)[None, :]
+    v = np.ascontiguousarray(v)
+    b = None if bias_bf16 is None else _c(bias_bf16, np.uint16)
+    y = np.empty((M, N), dtype=np.uint16)
+    _load().oracle_round_output(_ptr(v), None if b is None else _ptr(b), act, M, N, _ptr(y))
+    return {"xt": xt, "codes": codes, "scale64": s64, "scale32": s32, "y": y}

@@ -308,3 +308,39 @@ def test_error_halves_per_activation_bit_and_vanishes_without_weight_error():
     # and the dequantized integer result equals the same product in plain floating point
     ref = (out["scale32"].astype(np.float64)[:, None] * out["codes"]) @ (d.astype(np.float64)[:, None] * (u.astype(np.float64) - z[:, None])).T
     assert np.abs(bf16_values(out["y"]) - ref).max() <= np.abs(ref).max() * 2.0 ** -8
+
+
+# ------------------------------------------------------------------ block-wise scales
+
+def test_grouped_quantizer_reduces_to_the_per_token_one_and_keeps_its_invariants():
+    g = torch.Generator().manual_seed(21)
+    x = torch.randn(12, 2048, generator=g)
+    x[:, 5] *= 30.0                                             # an outlier channel in the first block only
+    xb = x.to(torch.bfloat16)
+    w = (torch.randn(16, 2048, generator=g) * 0.02).to(torch.bfloat16)
+    from helpers import to_bits, bf16_values
+    u, d, z = orc.prepare_weights(to_bits(w), 1024, "minmax")
+    # one block = the whole row: identical to the per-token path, bit for bit
+    a = orc.qlinear_grouped(to_bits(xb), u, d, z, 1024, 4, 2048)
+    b = orc.qlinear(to_bits(xb), u, d, z, 1024, 4)
+    assert np.array_equal(a["codes"], b["codes"]) and np.array_equal(a["y"], b["y"])
+    # two blocks: every block has its own scale = its own absmax / qmax, error <= scale / 2 per element
+    c = orc.qlinear_grouped(to_bits(xb), u, d, z, 1024, 4, 1024)
+    xt = c["xt"]
+    for blk in range(2):
+        sl = slice(blk * 1024, (blk + 1) * 1024)
+        s = c["scale64"][:, blk]
+        assert np.allclose(s * 7, np.abs(xt[:, sl]).max(axis=1), rtol=1e-15)
+        assert (np.abs(xt[:, sl] - s[:, None] * c["codes"][:, sl]) <= s[:, None] / 2 * (1 + 1e-12)).all()
+        assert (np.abs(c["codes"][:, sl]).max(axis=1) == 7).all()
+    # the combination over blocks, retyped with numpy from the stage outputs
+    acc0 = orc.int_gemm(c["codes"][:, :1024], np.ascontiguousarray(u[:, :1024]), z).astype(np.float64)
+    acc1 = orc.int_gemm(c["codes"][:, 1024:], np.ascontiguousarray(u[:, 1024:]), z).astype(np.float64)
+    v = (acc0 * c["scale32"][:, :1].astype(np.float64) + acc1 * c["scale32"][:, 1:].astype(np.float64)) * d.astype(np.float64)[None, :]
+    ref = torch.from_numpy(v).to(torch.bfloat16).to(torch.float64).numpy()   # torch's cast: fp64 -> bf16, ties to even
+    assert np.array_equal(bf16_values(c["y"]), ref)
+    # the outlier only costs its own block its resolution: the block-wise result is closer to X W^T
+    exact = xb.to(torch.float64).numpy() @ w.to(torch.float64).numpy().T
+    err_tok = np.linalg.norm(bf16_values(b["y"]) - exact)
+    err_blk = np.linalg.norm(bf16_values(c["y"]) - exact)
+    assert err_blk < err_tok
