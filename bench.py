@@ -107,14 +107,15 @@ def layer_ops(M, layer):
     return 2.0 * M * layer.N * layer.K
 
 
-def rq_bytes(M, layer):
-    """Algorithmic HBM bytes of rotate-quantize: bf16 row in, packed codes + scale + code sum out."""
-    return M * (2.0 * layer.K + layer.K * layer.bits / 8.0 + 8.0)
+def rq_bytes(M, layer, scale_group=0):
+    """Algorithmic HBM bytes of rotate-quantize: bf16 row in, packed codes + scales + code sums out."""
+    per_token = layer.K // scale_group if scale_group else 1
+    return M * (2.0 * layer.K + layer.K * layer.bits / 8.0 + 8.0 * per_token)
 
 
 # ------------------------------------------------------------------ the CPU oracle leg
 
-def oracle_sample(wl, tokens, steps=1, warmup=0):
+def oracle_sample(wl, tokens, steps=1, warmup=0, scale_group=0):
     """Times the CPU oracle, as it stands, on `tokens` tokens of every layer of the workload
     (rotation + quantizer + integer GEMM + epilogue; weight preparation is offline and not
     timed).  Returns (seconds per step, ops per step, threads)."""
@@ -134,7 +135,10 @@ def oracle_sample(wl, tokens, steps=1, warmup=0):
 
     def one_step():
         for layer, xb, u, d, z in prepared:
-            orc.qlinear(xb, u, d, z, layer.rot_block, layer.bits, None, layer.act)
+            if scale_group:
+                orc.qlinear_grouped(xb, u, d, z, layer.rot_block, layer.bits, scale_group, None, layer.act)
+            else:
+                orc.qlinear(xb, u, d, z, layer.rot_block, layer.bits, None, layer.act)
 
     for _ in range(warmup):
         one_step()
@@ -150,7 +154,7 @@ def run_reference(args, wl):
     if rank != 0:
         return
     tokens = args.ref_tokens
-    dt, ops, threads = oracle_sample(wl, tokens, steps=args.steps, warmup=min(args.warmup, 1))
+    dt, ops, threads = oracle_sample(wl, tokens, steps=args.steps, warmup=min(args.warmup, 1), scale_group=args.scale_group)
     value = ops / dt / 1e12
     sample = f"{tokens} tokens of each of the {len(wl.layers)} layers of '{wl.name}' per step (full K and N)"
     line = {
@@ -170,6 +174,7 @@ def config_of(wl, args):
                 f"{l.K}->{l.N} A{l.bits} B{l.rot_block}" for l in wl.layers),
             "weights": "4-bit per-output-channel codes (random, Gaussian-shaped)",
             "l2_policy": "inputs larger than L2 (every layer streams >= 400 MB)",
+            "act_scales": (f"one per token and block of {args.scale_group} channels" if args.scale_group else "one per token"),
             "parallelism": f"dp{args.gpus} (token-sharded replicas, no collective)"}
 
 
@@ -207,10 +212,13 @@ def run_cuda(args, wl):
         blob = torch.empty(B.dvdq_weight_blob_bytes(layer.N, layer.K), dtype=torch.uint8, device=dev)
         w = B.dvdq_pack_weights(u, d, z, layer.rot_block, blob)
         del u
-        q = B.ActQuant(layer.bits, layer.rot_block, 0)
+        q = B.ActQuant(layer.bits, layer.rot_block, args.scale_group)
         codes = torch.empty(B.dvdq_act_codes_bytes(M, layer.K, layer.bits), dtype=torch.uint8, device=dev)
-        scales = torch.empty(M, dtype=torch.float32, device=dev)
-        sums = torch.empty(M, dtype=torch.int32, device=dev)
+        n_scales = B.dvdq_act_scales_count(M, layer.K, q)
+        if n_scales == 0:
+            raise SystemExit(f"layer {layer.K}->{layer.N}: activation quantizer options not supported")
+        scales = torch.empty(n_scales, dtype=torch.float32, device=dev)
+        sums = torch.empty(n_scales, dtype=torch.int32, device=dev)
         Y = torch.empty(M, layer.N, dtype=torch.bfloat16, device=dev)
         bias = W.make_bias(wl, layer, device=dev)
         layers.append(dict(layer=layer, w=w, blob=blob, q=q, codes=codes, scales=scales, sums=sums, Y=Y, bias=bias))
@@ -268,13 +276,13 @@ def run_cuda(args, wl):
     int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
     gemm_ops = sum(layer_ops(M, L["layer"]) for L in layers)
     gemm_tops = gemm_ops / (sum(gm_ms) * 1e-3) / 1e12
-    rq_total_bytes = sum(rq_bytes(M, L["layer"]) for L in layers)
+    rq_total_bytes = sum(rq_bytes(M, L["layer"], args.scale_group) for L in layers)
     rq_gbs = rq_total_bytes / (sum(rq_ms) * 1e-3) / 1e9
     stages = []
     for li, L in enumerate(layers):
         layer = L["layer"]
         stages.append({"layer": f"{layer.K}->{layer.N} A{layer.bits}",
-                       "rq_ms": rq_ms[li], "rq_gbs": rq_bytes(M, layer) / (rq_ms[li] * 1e-3) / 1e9,
+                       "rq_ms": rq_ms[li], "rq_gbs": rq_bytes(M, layer, args.scale_group) / (rq_ms[li] * 1e-3) / 1e9,
                        "qgemm_ms": gm_ms[li], "qgemm_tops": layer_ops(M, layer) / (gm_ms[li] * 1e-3) / 1e12})
 
     # ---- end to end through dvdq_qlinear with HOST buffers (pinned), copies inside the timed region
@@ -306,7 +314,7 @@ def run_cuda(args, wl):
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
-        dt, ops, threads = oracle_sample(wl, args.ref_tokens)
+        dt, ops, threads = oracle_sample(wl, args.ref_tokens, scale_group=args.scale_group)
         line["cpu_baseline"] = {"value": ops / dt / 1e12, "unit": "TOPS", "cores": threads, "kind": "oracle",
                                 "sample": f"{args.ref_tokens} tokens of each layer of '{wl.name}' (full K and N), {dt:.1f} s"}
     print(json.dumps(line), flush=True)
@@ -403,6 +411,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling runs)")
+    ap.add_argument("--scale-group", type=int, default=0,
+                    help="0: one activation scale per token; 1024: one per token and block of 1024 channels")
     ap.add_argument("--bits", type=int, default=0, help="override the activation bit width of every layer (4, 6 or 8)")
     args = ap.parse_args()
     from paper_2505_18663_b200 import workloads as W

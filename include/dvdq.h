@@ -46,7 +46,7 @@ typedef enum {
     DVDQ_ERR_ARCH = 8,           /* current device is not sm_100 */
     DVDQ_ERR_CUDA = 9,           /* a CUDA runtime or driver call failed */
     DVDQ_ERR_DEVICE_TIMEOUT = 10,/* a kernel gave up on a bounded device-side wait */
-    DVDQ_ERR_UNSUPPORTED = 11    /* a reserved option (scale_group != 0, unknown activation function) */
+    DVDQ_ERR_UNSUPPORTED = 11    /* an option that is not built (scale_group other than 0 or 1024, unknown activation function) */
 } dvdq_status;
 
 /* Human-readable name of a status code (static storage, never NULL). */
@@ -60,8 +60,11 @@ const char* dvdq_status_string(dvdq_status s);
  *   rot_block   B, the order of the Hadamard blocks of the rotation
  *               R = I_{K/B} (x) H_B / sqrt(B); a power of two in [64, 1024] that
  *               divides K.  0 means no rotation (R = I).
- *   scale_group granularity of Lambda: 0 = one absmax scale per token over all K
- *               channels (the only built value; others give DVDQ_ERR_UNSUPPORTED).
+ *   scale_group granularity of Lambda: 0 = one absmax scale per token over all K channels;
+ *               1024 = the block-wise variant of Sec. 3.2's last paragraph, one scale per token
+ *               and per block of 1024 consecutive rotated channels (K % 1024 == 0; every block
+ *               is quantized on its own, the GEMM rescales per block).  Other values give
+ *               DVDQ_ERR_UNSUPPORTED.
  */
 typedef struct {
     int32_t bits;
@@ -89,6 +92,8 @@ typedef struct {
 
 /* Bytes of the packed activation codes of an [M, K] tensor: M * K * bits / 8. 0 on bad input. */
 size_t dvdq_act_codes_bytes(int64_t M, int64_t K, int32_t bits);
+/* Number of scales (and of code sums) of an [M, K] tensor: M, or M * K / 1024 block-wise. 0 on bad input. */
+size_t dvdq_act_scales_count(int64_t M, int64_t K, const dvdq_act_quant* q);
 /* Bytes of the device blob that dvdq_pack_weights() writes for an [N, K] matrix. 0 on bad input. */
 size_t dvdq_weight_blob_bytes(int64_t N, int64_t K);
 /* Bytes of the workspace dvdq_qlinear() needs (codes, scales and code sums of X). 0 on bad input. */
@@ -101,8 +106,10 @@ size_t dvdq_qlinear_workspace_bytes(int64_t M, int64_t K, const dvdq_act_quant* 
  *
  *   X_bf16         [M, K] bf16, row pitch ldx elements; 16-byte aligned, ldx % 8 == 0
  *   codes_out      dvdq_act_codes_bytes(M, K, bits) bytes, 16-byte aligned (opaque layout)
- *   scales_out     [M] fp32, s_i  (0 for an all-zero token, whose codes are all 0)
- *   code_sums_out  [M] int32, sum_k c_ik (used by the GEMM for the weight zero point)
+ *   scales_out     [M] fp32, s_i  (0 for an all-zero token, whose codes are all 0);
+ *                  block-wise: [M, K/1024], one scale per token and block
+ *   code_sums_out  [M] int32, sum_k c_ik (used by the GEMM for the weight zero point);
+ *                  block-wise: [M, K/1024], the sum over each block
  * K % 64 == 0, K <= 16384.  M == 0 is a no-op.
  */
 dvdq_status dvdq_rotate_quantize(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,
@@ -151,6 +158,8 @@ dvdq_status dvdq_bgr_quantize(const float* W_rot, int64_t N, int64_t K, int32_t 
  *
  *   acc_in = sum_k c_ik (u_nk - z_n)      exact int32 (tensor cores, int8 operands)
  *   y_in   = bf16( acc_in * s_i * Delta_n + bias_n )   fp32 arithmetic, one rounding
+ *   block-wise scales: y_in = bf16( Delta_n * sum_g s_ig * acc_ing + bias_n ), acc_ing the exact
+ *   int32 sum over block g, the sum over blocks in fp32
  *   act == 1 applies tanh-GELU to the rounded value and rounds to bf16 again.
  *
  *   codes, scales, code_sums   outputs of dvdq_rotate_quantize for the same M, K, q

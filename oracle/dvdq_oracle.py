@@ -288,23 +288,31 @@ def act_quantize_grouped(xt: np.ndarray, bits: int, group: int):
     return codes, s64, s32
 
 
-def qlinear_grouped(x_bf16, u, delta32, z, B: int, bits: int, group: int, bias_bf16=None, act: int = 0):
-    """The layer with block-wise activation scales:
+def combine_grouped(codes, u, z, s32, delta32, group: int, bias_bf16=None, act: int = 0) -> np.ndarray:
+    """Given codes and block scales, the output of the layer with block-wise activation scales:
         y_in = bf16( Delta_n * sum_g s_ig * sum_{k in block g} c_ik (u_nk - z_n) + bias_n ),
     every block's integer GEMM on its own, combined in fp64 (scales and Delta are their stored
-    binary32 values), then the same rounding / GELU as the per-token path."""
-    xt = rotate(x_bf16, B)
-    codes, s64, s32 = act_quantize_grouped(xt, bits, group)
+    binary32 values), then the same rounding / GELU as the per-token path.  bf16 bits [M,N]."""
+    codes = _c(codes, np.int32)
     M, K = codes.shape
     N = u.shape[0]
     v = np.zeros((M, N), dtype=np.float64)
     for g in range(K // group):
         sl = slice(g * group, (g + 1) * group)
-        acc = int_gemm(codes[:, sl], np.ascontiguousarray(u[:, sl]), z)
+        acc = int_gemm(np.ascontiguousarray(codes[:, sl]), np.ascontiguousarray(u[:, sl]), z)
         v += acc.astype(np.float64) * s32[:, g].astype(np.float64)[:, None]
     v *= np.asarray(delta32, dtype=np.float32).astype(np.float64)[None, :]
     v = np.ascontiguousarray(v)
     b = None if bias_bf16 is None else _c(bias_bf16, np.uint16)
     y = np.empty((M, N), dtype=np.uint16)
     _load().oracle_round_output(_ptr(v), None if b is None else _ptr(b), act, M, N, _ptr(y))
+    return y
+
+
+def qlinear_grouped(x_bf16, u, delta32, z, B: int, bits: int, group: int, bias_bf16=None, act: int = 0):
+    """The layer with block-wise activation scales: rotation, the block-wise quantizer, then
+    combine_grouped."""
+    xt = rotate(x_bf16, B)
+    codes, s64, s32 = act_quantize_grouped(xt, bits, group)
+    y = combine_grouped(codes, u, z, s32, delta32, group, bias_bf16, act)
     return {"xt": xt, "codes": codes, "scale64": s64, "scale32": s32, "y": y}

@@ -20,7 +20,7 @@ OK, ERR_NULL, ERR_SHAPE, ERR_BITS, ERR_ROT_BLOCK, ERR_ALIGN, ERR_WORKSPACE, ERR_
     ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_UNSUPPORTED = range(12)
 
 EXPORTS = [
-    "dvdq_status_string", "dvdq_version", "dvdq_act_codes_bytes", "dvdq_weight_blob_bytes",
+    "dvdq_status_string", "dvdq_version", "dvdq_act_codes_bytes", "dvdq_act_scales_count", "dvdq_weight_blob_bytes",
     "dvdq_qlinear_workspace_bytes", "dvdq_rotate_quantize", "dvdq_pack_weights", "dvdq_qgemm",
     "dvdq_qlinear", "dvdq_qlinear_static", "dvdq_qgemm_int32", "dvdq_pack_act_codes", "dvdq_unpack_act_codes",
     "dvdq_unpack_weights", "dvdq_last_device_status",
@@ -78,6 +78,7 @@ def load():
         "dvdq_status_string": (C.c_char_p, [C.c_int]),
         "dvdq_version": (i32, []),
         "dvdq_act_codes_bytes": (sz, [i64, i64, i32]),
+        "dvdq_act_scales_count": (sz, [i64, i64, aq]),
         "dvdq_weight_blob_bytes": (sz, [i64, i64]),
         "dvdq_qlinear_workspace_bytes": (sz, [i64, i64, aq]),
         "dvdq_rotate_quantize": (C.c_int, [p, i64, i64, i64, aq, p, p, p, p]),
@@ -143,6 +144,10 @@ def dvdq_version() -> int:
 
 def dvdq_act_codes_bytes(M: int, K: int, bits: int) -> int:
     return int(load().dvdq_act_codes_bytes(M, K, bits))
+
+
+def dvdq_act_scales_count(M: int, K: int, q: ActQuant) -> int:
+    return int(load().dvdq_act_scales_count(M, K, C.byref(q)))
 
 
 def dvdq_weight_blob_bytes(N: int, K: int) -> int:

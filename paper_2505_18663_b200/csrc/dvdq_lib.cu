@@ -40,7 +40,10 @@ static dvdq_status validate_k(int64_t K) {
 dvdq_status validate_act_quant(const dvdq_act_quant* q, int64_t K) {
     if (!q) return DVDQ_ERR_NULL;
     if (q->bits != 4 && q->bits != 6 && q->bits != 8) return DVDQ_ERR_BITS;
-    if (q->scale_group != 0) return DVDQ_ERR_UNSUPPORTED;
+    // block-wise scales: one per token and per 1024-channel block (the unit a warp of the transform
+    // and eight k-blocks of the GEMM work on); other block sizes are not built
+    if (q->scale_group != 0 && q->scale_group != kScaleBlock) return DVDQ_ERR_UNSUPPORTED;
+    if (q->scale_group != 0 && K % kScaleBlock != 0) return DVDQ_ERR_SHAPE;
     if (q->rot_block != 0) {
         if (!is_pow2(q->rot_block) || q->rot_block < 64 || q->rot_block > 1024) return DVDQ_ERR_ROT_BLOCK;
         if (K % q->rot_block != 0) return DVDQ_ERR_ROT_BLOCK;
@@ -61,12 +64,14 @@ dvdq_status validate_weights(const dvdq_weights* w) {
 struct WorkspacePlan {
     int64_t codes_off, scales_off, sums_off, total;
 };
-static WorkspacePlan workspace_plan(int64_t M, int64_t K, int bits) {
+static int64_t scales_per_token(int64_t K, const dvdq_act_quant& q) { return q.scale_group ? K / q.scale_group : 1; }
+static WorkspacePlan workspace_plan(int64_t M, int64_t K, const dvdq_act_quant& q) {
     WorkspacePlan p;
+    const int64_t per_token = scales_per_token(K, q);
     p.codes_off = 0;
-    p.scales_off = align_up(M * act_row_bytes(K, bits), 256);
-    p.sums_off = p.scales_off + align_up(M * 4, 256);
-    p.total = p.sums_off + align_up(M * 4, 256);
+    p.scales_off = align_up(M * act_row_bytes(K, q.bits), 256);
+    p.sums_off = p.scales_off + align_up(M * per_token * 4, 256);
+    p.total = p.sums_off + align_up(M * per_token * 4, 256);
     return p;
 }
 
@@ -101,6 +106,11 @@ size_t dvdq_act_codes_bytes(int64_t M, int64_t K, int32_t bits) {
     return (size_t)(M * act_row_bytes(K, bits));
 }
 
+size_t dvdq_act_scales_count(int64_t M, int64_t K, const dvdq_act_quant* q) {
+    if (M < 0 || validate_k(K) != DVDQ_OK || validate_act_quant(q, K) != DVDQ_OK) return 0;
+    return (size_t)(M * scales_per_token(K, *q));
+}
+
 size_t dvdq_weight_blob_bytes(int64_t N, int64_t K) {
     if (N <= 0 || N % 8 != 0 || validate_k(K) != DVDQ_OK) return 0;
     return (size_t)blob_layout(N, K).total;
@@ -108,7 +118,7 @@ size_t dvdq_weight_blob_bytes(int64_t N, int64_t K) {
 
 size_t dvdq_qlinear_workspace_bytes(int64_t M, int64_t K, const dvdq_act_quant* q) {
     if (M < 0 || validate_k(K) != DVDQ_OK || validate_act_quant(q, K) != DVDQ_OK) return 0;
-    return (size_t)workspace_plan(M, K, q->bits).total;
+    return (size_t)workspace_plan(M, K, *q).total;
 }
 
 dvdq_status dvdq_rotate_quantize(const void* X, int64_t M, int64_t K, int64_t ldx, const dvdq_act_quant* q,
@@ -194,7 +204,7 @@ dvdq_status dvdq_qlinear(const void* X, int64_t M, int64_t ldx, const dvdq_act_q
     if (M == 0) return DVDQ_OK;
     if (!workspace) return DVDQ_ERR_NULL;
     if (!aligned(workspace, 256)) return DVDQ_ERR_ALIGN;
-    const WorkspacePlan p = workspace_plan(M, w->K, q->bits);
+    const WorkspacePlan p = workspace_plan(M, w->K, *q);
     if (workspace_bytes < (size_t)p.total) return DVDQ_ERR_WORKSPACE;
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     void* codes = ws + p.codes_off;
@@ -217,7 +227,7 @@ dvdq_status dvdq_qlinear_static(const void* X, int64_t M, int64_t ldx, const dvd
     if ((s = validate_act_quant(q, w->K)) != DVDQ_OK) return s;
     if (M < 0) return DVDQ_ERR_SHAPE;
     if (M == 0) return DVDQ_OK;
-    const WorkspacePlan p = workspace_plan(M, w->K, q->bits);
+    const WorkspacePlan p = workspace_plan(M, w->K, *q);
     if (p.total > (int64_t)DVDQ_STATIC_SCRATCH_BYTES) return DVDQ_ERR_WORKSPACE;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DVDQ_ERR_CUDA;
@@ -248,7 +258,8 @@ dvdq_status dvdq_pack_act_codes(const int8_t* codes_nat, int64_t M, int64_t K, c
     if (q->bits == 4) pack_act_codes_kernel<4><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
     else if (q->bits == 6) pack_act_codes_kernel<6><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
     else pack_act_codes_kernel<8><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
-    code_sums_kernel<<<(unsigned)((M * 32 + 255) / 256), 256, 0, st>>>(codes_nat, M, K, code_sums_out);
+    const int64_t block = q->scale_group ? q->scale_group : K;
+    code_sums_kernel<<<(unsigned)((M * (K / block) * 32 + 255) / 256), 256, 0, st>>>(codes_nat, M, K, block, code_sums_out);
     return cuda_status(cudaGetLastError());
 }
 

@@ -105,14 +105,19 @@ __global__ void unpack_act_codes_kernel(const uint8_t* __restrict__ packed, int6
     }
 }
 
-__global__ void code_sums_kernel(const int8_t* __restrict__ nat, int64_t M, int64_t K, int32_t* __restrict__ sums) {
+// One warp per (token, block): sum of the codes of `block` consecutive channels (block = K for
+// the per-token variant).
+__global__ void code_sums_kernel(const int8_t* __restrict__ nat, int64_t M, int64_t K, int64_t block,
+                                 int32_t* __restrict__ sums) {
     const int lane = threadIdx.x & 31;
-    const int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (row >= M) return;
+    const int64_t unit = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t per_row = K / block;
+    if (unit >= M * per_row) return;
+    const int64_t row = unit / per_row, blk = unit - row * per_row;
     int s = 0;
-    for (int64_t k = lane; k < K; k += 32) s += nat[row * K + k];
+    for (int64_t k = lane; k < block; k += 32) s += nat[row * K + blk * block + k];
     for (int m = 16; m > 0; m >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, m);
-    if (lane == 0) sums[row] = s;
+    if (lane == 0) sums[unit] = s;
 }
 
 inline unsigned grid_for(int64_t work, int threads) {

@@ -59,9 +59,11 @@ constexpr int kAColsPerStage = kBK / 4;
 static_assert(kTmemACol + kWideStages * kAColsPerStage <= kTmemCols, "tensor memory budget");
 static_assert(kWideStages % 2 == 0, "the MMA warp takes the wide stages in pairs");
 
-template <int BITS>
+// BLK: block-wise activation scales (tile of 128 channels, see the kernel).
+template <int BITS, bool BLK>
 struct GemmSmem {
-    static constexpr int kWideW = kBNh * kBK;                     // int8 weight half-tile, swizzled
+    static constexpr int BN = BLK ? 128 : kBN, BNh = BN / 2;
+    static constexpr int kWideW = BNh * kBK;                     // int8 weight half-tile, swizzled
     static constexpr int kWideOff = 0;                            // 1024-byte aligned tiles first
     static constexpr int kALo = (BITS == 8) ? kBM * kPK : kBM * kPK / 2;  // A4 codes / A6 low plane (128-byte rows); A8: two tiles of 128-byte rows, one per k-block
     static constexpr int kPStages = (BITS == 8) ? 3 : kPackedStages;  // what fits
@@ -71,9 +73,9 @@ struct GemmSmem {
     static constexpr int kStageOutOff = kPackedOff + kPStages * kPackedStage;  // 1024-byte aligned
     static constexpr int kStageOutPerWarp = 2 * 32 * 128;  // two buffers of 32 rows x 64 bf16
     static constexpr int kWPackedOff = kStageOutOff + kEpilogueWarps * kStageOutPerWarp;
-    static constexpr int kWPacked = kBNh * kBK / 2;              // packed weight half-tile of one k-block (64-byte rows)
+    static constexpr int kWPacked = BNh * kBK / 2;              // packed weight half-tile of one k-block (64-byte rows)
     static constexpr int kConstOff = kWPackedOff + kWPackedStages * kWPacked;
-    static constexpr int kConstPerWarp = 3 * kBN * 4;  // delta, zero-point rest, bias
+    static constexpr int kConstPerWarp = 3 * BN * 4;  // delta, zero-point rest, bias
     static constexpr int kBarOff = kConstOff + kEpilogueWarps * kConstPerWarp;
     static constexpr int kNumBars = 2 * kPackedStages + 2 * kWideStages + 5 + 2 * kWPackedStages;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
@@ -94,15 +96,16 @@ __device__ __forceinline__ float gelu_tanh_f32(float y) {
     return y * r;
 }
 
-template <int BITS, bool RAW>
+template <int BITS, bool RAW, bool BLK>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmAhi,
              const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmY,
              const float* __restrict__ scales,
              const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
              const __nv_bfloat16* __restrict__ bias, __nv_bfloat16* __restrict__ Y, int64_t ldy,
-             int32_t* __restrict__ acc_out, int64_t ldacc, int M, int N, int K, int act) {
-    using S = GemmSmem<BITS>;
+             int32_t* __restrict__ acc_out, int64_t ldacc, int M, int N, int K, int act, int spr) {
+    using S = GemmSmem<BITS, BLK>;
+    constexpr int BN = S::BN, BNh = S::BNh;  // channels of the pair's tile / weight rows per CTA
     extern __shared__ uint8_t smem_raw[];
     // identical in both CTAs of the pair: the dynamic shared window starts at the same offset
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -111,10 +114,13 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();       // 0 = leader of the pair
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-    const int num_n = (N + kBN - 1) / kBN, num_m = (M + 2 * kBM - 1) / (2 * kBM);
+    const int num_n = (N + BN - 1) / BN, num_m = (M + 2 * kBM - 1) / (2 * kBM);
     const int num_tiles = num_m * num_n;
     const int KB2 = (K + kPK - 1) / kPK;  // activation loads per tile; a k-block past K reads zeros
     const int KB = 2 * KB2;
+    // one accumulator per tile, or (block-wise scales) one per tile and block of 1024 codes
+    const int NG = BLK ? K / kScaleBlock : 1;
+    const int KBG = BLK ? kScaleBlock / kBK : KB;  // k-blocks per accumulator
 
     const uint32_t bar0 = sbase + S::kBarOff;
     auto pk_full = [&](int s) { return bar0 + 8u * s; };
@@ -159,7 +165,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             bool ok = true;
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
-                const int n0 = (tile % num_n) * kBN + (int)rank * kBNh;
+                const int n0 = (tile % num_n) * BN + (int)rank * BNh;
                 for (int sb = 0; ok && sb < KB2; ++sb) {
                     if (!mbar_wait(pk_empty(st), ph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
                     const uint32_t dst = sbase + S::kPackedOff + st * S::kPackedStage;
@@ -203,18 +209,19 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         // The whole warp walks the loop (warp-uniform control flow); one elected lane issues.
         if (rank == 0) {
-            constexpr uint32_t idesc = umma_idesc_s8s8s32(2 * kBM, kBN);
+            constexpr uint32_t idesc = umma_idesc_s8s8s32(2 * kBM, BN);
             uint32_t st = 0, ph = 0, lt = 0;
             bool ok = true;
-            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++lt) {
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs)
+            for (int g = 0; ok && g < NG; ++g, ++lt) {
                 const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
                 if (!mbar_wait_warp(acc_empty(a), aph ^ 1u, abort_flag, kWaitAccEmpty)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + a * kBN;
+                const uint32_t d_tmem = tmem_base + a * BN;
                 // Two k-blocks per trip (KB is even, and so is kWideStages): the tensor core's queue
                 // is short, so every cycle this warp spends between two issues is a bubble in the
                 // MMA stream; pairing halves the waits, votes and bookkeeping per k-block.
-                for (int kb = 0; kb < KB; kb += 2) {
+                for (int kb = 0; kb < KBG; kb += 2) {
                     if (!mbar_wait_warp(wd_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     if (!mbar_wait_warp(wd_full(st + 1), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     tc_fence_after();
@@ -246,21 +253,123 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;  // tensor-memory lane quarter this warp may read
         const int ew = warp - kFirstEpilogueWarp;
-        const uint32_t c_delta = sbase + S::kConstOff + ew * S::kConstPerWarp;  // shared addresses of float[kBN] each
-        const uint32_t c_zc = c_delta + kBN * 4;    // (z_n - 8) as a float: exact, |.| <= 8
-        const uint32_t c_bias = c_zc + kBN * 4;
+        const uint32_t c_delta = sbase + S::kConstOff + ew * S::kConstPerWarp;  // shared addresses of float[BN] each
+        const uint32_t c_zc = c_delta + BN * 4;    // (z_n - 8) as a float: exact, |.| <= 8
+        const uint32_t c_bias = c_zc + BN * 4;
         const uint32_t stg0 = sbase + S::kStageOutOff + ew * S::kStageOutPerWarp;
         constexpr int kShift = (BITS == 4) ? 8 : (BITS == 6) ? 6 : 4;  // log2 of (A factor 16 / 4 / 1) x (W factor 16)
         if (!RAW && lane == 0) tma_prefetch_desc(&tmY);
+        if constexpr (BLK) {
+            // Block-wise scales: every block of 1024 codes has its own int32 accumulator (the two
+            // accumulators alternate) and its own scale per token.  This warp keeps the running
+            // fp32 sum over blocks of its 32 rows in tensor-memory columns [256, 384) -- lanes only
+            // it touches -- and dequantizes after the last block:
+            //     y = Delta_n * sum_g s_ig (acc_g - (z_n - 8) S_ig) + bias_n.
+            constexpr uint32_t kFloatCol = 2 * BN;
+            uint32_t lt = 0, nstore = 0;
+            for (int tile = pair; tile < num_tiles; tile += num_pairs) {
+                const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM, n0 = (tile % num_n) * BN;
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < BN / 32; ++i) {
+                    const int c = lane + 32 * i, n = n0 + c;
+                    const bool okn = n < N;
+                    sts32f(c_delta + 4 * c, okn ? __ldg(delta + n) : 0.f);
+                    sts32f(c_zc + 4 * c, okn ? (float)__ldg(zc + n) : 0.f);
+                    sts32f(c_bias + 4 * c, (okn && bias != nullptr) ? __bfloat162float(bias[n]) : 0.f);
+                }
+                __syncwarp();
+                const int row = m0 + q * 32 + lane;
+                const bool row_ok = row < M;
+                const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+                bool ok = true;
+                for (int g = 0; g < NG; ++g, ++lt) {
+                    const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
+                    if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) { ok = false; break; }
+                    tc_fence_after();
+                    const float s_g = row_ok ? scales[(int64_t)row * NG + g] : 0.f;
+                    const float S_g = row_ok ? (float)sums[(int64_t)row * NG + g] : 0.f;
+                    const float s_k = s_g * (1.0f / (float)(1 << kShift)), nS_k = -S_g * (float)(1 << kShift);
+                    const bool last = g == NG - 1;
+#pragma unroll 1
+                    for (int hc = 0; hc < BN / 16; ++hc) {
+                        uint32_t r[16], f[16];
+                        tmem_ld_32x16(tmem_base + a * BN + hc * 16 + lane_addr, r);
+                        if (g > 0) tmem_ld_32x16(tmem_base + kFloatCol + hc * 16 + lane_addr, f);
+                        tmem_ld_wait();
+                        float v[16];
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4) {
+                            const float4 z4 = lds128f(c_zc + 4 * (hc * 16 + j));
+                            const float zz[4] = {z4.x, z4.y, z4.z, z4.w};
+#pragma unroll
+                            for (int t = 0; t < 4; ++t) {
+                                const float part = fmaf(zz[t], nS_k, (float)(int32_t)r[j + t]) * s_k;  // the fma is exact
+                                v[j + t] = g > 0 ? __uint_as_float(f[j + t]) + part : part;
+                            }
+                        }
+                        if (!last) {
+#pragma unroll
+                            for (int t = 0; t < 16; ++t) f[t] = __float_as_uint(v[t]);
+                            tmem_st_32x16(tmem_base + kFloatCol + hc * 16 + lane_addr, f);
+                            continue;
+                        }
+                        // last block: dequantize, round, stage 64 columns per TMA store
+                        if ((hc & 3) == 0) {
+                            if (lane == 0) tma_store_wait_read<1>();
+                            __syncwarp();
+                        }
+                        const uint32_t buf = stg0 + (nstore & 1u) * (32 * 128);
+#pragma unroll
+                        for (int j = 0; j < 16; j += 8) {
+                            const float4 d0 = lds128f(c_delta + 4 * (hc * 16 + j)), d1 = lds128f(c_delta + 4 * (hc * 16 + j + 4));
+                            const float4 b0 = lds128f(c_bias + 4 * (hc * 16 + j)), b1 = lds128f(c_bias + 4 * (hc * 16 + j + 4));
+                            const float dl[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+                            const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int t = 0; t < 8; t += 2) {
+                                float y0 = fmaf(v[j + t], dl[t], bb[t]), y1 = fmaf(v[j + t + 1], dl[t + 1], bb[t + 1]);
+                                if (act == 1) {
+                                    y0 = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(y0)));
+                                    y1 = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(y1)));
+                                }
+                                __nv_bfloat162 b2 = __floats2bfloat162_rn(y0, y1);
+                                pk[t >> 1] = *reinterpret_cast<uint32_t*>(&b2);
+                            }
+                            const int ch = (2 * (hc & 3) + (j >> 3)) ^ (lane & 7);
+                            sts128(buf + lane * 128 + ch * 16, pk[0], pk[1], pk[2], pk[3]);
+                        }
+                        if ((hc & 3) == 3) {
+                            fence_proxy_async_smem();
+                            __syncwarp();
+                            const int nb = n0 + (hc >> 2) * 64;
+                            if (lane == 0 && nb < N && m0 + q * 32 < M) {
+                                tma_store_2d(&tmY, buf, nb, m0 + q * 32);
+                                tma_store_commit();
+                            }
+                            ++nstore;
+                        }
+                    }
+                    if (!last) tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty(a), 0));
+                }
+                if (!ok) break;
+            }
+            if (lane == 0) tma_store_wait_all();
+            __syncwarp();
+        } else {
         uint32_t lt = 0, nstore = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++lt) {
             const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
-            const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM, n0 = (tile % num_n) * kBN;
+            const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM, n0 = (tile % num_n) * BN;
             __syncwarp();
             {   // per-channel constants of this tile: all loads in flight at once, then the stores
-                float cd[kBN / 32], cz[kBN / 32], cb[kBN / 32];
+                float cd[BN / 32], cz[BN / 32], cb[BN / 32];
 #pragma unroll
-                for (int i = 0; i < kBN / 32; ++i) {
+                for (int i = 0; i < BN / 32; ++i) {
                     const int n = n0 + lane + 32 * i;
                     const bool okn = n < N;
                     cd[i] = okn ? __ldg(delta + n) : 0.f;
@@ -268,7 +377,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     cb[i] = (okn && bias != nullptr) ? __bfloat162float(bias[n]) : 0.f;
                 }
 #pragma unroll
-                for (int i = 0; i < kBN / 32; ++i) {
+                for (int i = 0; i < BN / 32; ++i) {
                     const int c = lane + 32 * i;
                     sts32f(c_delta + 4 * c, cd[i]);
                     sts32f(c_zc + 4 * c, cz[i]);
@@ -281,14 +390,16 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             const int row = m0 + q * 32 + lane;
             const bool row_ok = row < M;
             const float s_i = (!RAW && row_ok) ? scales[row] : 0.f;
-            const int32_t S_i = row_ok ? sums[row] : 0;
+            int32_t S_i = row_ok ? sums[(int64_t)row * spr] : 0;
+            if (RAW && row_ok)
+                for (int g = 1; g < spr; ++g) S_i += sums[(int64_t)row * spr + g];  // spr == 1 unless the scales are block-wise
             const float S_f = (float)S_i;  // |sum of codes| <= K * 32 < 2^24: exact
             const float s_k = s_i * (1.0f / (float)(1 << kShift)), nS_k = -S_f * (float)(1 << kShift);
             const uint64_t s2 = f2_pack(s_k, s_k), negS2 = f2_pack(nS_k, nS_k);
 #pragma unroll 1
-            for (int c = 0; c < kBN / 32; ++c) {
+            for (int c = 0; c < BN / 32; ++c) {
                 uint32_t r[32];
-                tmem_ld_32x32(tmem_base + a * kBN + c * 32 + ((uint32_t)(q * 32) << 16), r);
+                tmem_ld_32x32(tmem_base + a * BN + c * 32 + ((uint32_t)(q * 32) << 16), r);
                 tmem_ld_wait();
                 const int nb = n0 + c * 32;
                 if (RAW) {
@@ -363,6 +474,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         }
         if (!RAW && lane == 0) tma_store_wait_all();
         __syncwarp();
+        }
     } else if (warp < kFirstWWarp) {
         // ------------------------------------------------------------ widen activation codes -> tensor memory
         const int q = warp & 3;
@@ -448,9 +560,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
             const uint32_t pw = sbase + S::kWPackedOff + pst * S::kWPacked;
             const uint32_t wdW = sbase + S::kWideOff + wst * S::kWideW;
-            // 96 rows x 4 chunks of 32 nibbles, stored as (u - 8); widened in registers before the
+            // BNh rows x 4 chunks of 32 nibbles, stored as (u - 8); widened in registers before the
             // wide stage is known to be free
-            constexpr int kPieces = (kBNh * 4) / 128;
+            constexpr int kPieces = (BNh * 4) / 128;
             uint32_t e[kPieces][4], o[kPieces][4];
 #pragma unroll
             for (int it = 0; it < kPieces; ++it) {
@@ -532,11 +644,11 @@ inline bool make_byte_map(CUtensorMap* tm, const void* base, uint64_t row_len, u
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BITS, bool RAW>
-static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const int32_t* sums, int64_t M,
+template <int BITS, bool RAW, bool BLK>
+static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                   const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
                                   int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
-    using S = GemmSmem<BITS>;
+    using S = GemmSmem<BITS, BLK>;
     const int64_t K = w.K, N = w.N;
     const BlobLayout L = blob_layout(N, K);
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
@@ -552,7 +664,7 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
         tmAhi = tmA;
     }
 
-    if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, kBNh,
+    if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, S::BNh,
                        CU_TENSOR_MAP_SWIZZLE_NONE))
         return DVDQ_ERR_CUDA;
     if (RAW) {
@@ -561,7 +673,7 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
         return DVDQ_ERR_CUDA;
     }
 
-    auto kern = qgemm_kernel<BITS, RAW>;
+    auto kern = qgemm_kernel<BITS, RAW, BLK>;
     static int max_pairs = 0;
     if (max_pairs == 0) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) return DVDQ_ERR_CUDA;
@@ -582,13 +694,13 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
         if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) != cudaSuccess || clusters < 1) return DVDQ_ERR_CUDA;
         max_pairs = clusters < sm_count / 2 ? clusters : sm_count / 2;
     }
-    const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + kBN - 1) / kBN);
+    const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + S::BN - 1) / S::BN);
     const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
     kern<<<2 * pairs, kGemmThreads, S::kTotal, st>>>(tmA, tmAhi, tmW, tmY, scales, sums,
                                                      reinterpret_cast<const float*>(blob + L.delta_offset),
                                                      reinterpret_cast<const int32_t*>(blob + L.zc_offset),
                                                      static_cast<const __nv_bfloat16*>(bias), static_cast<__nv_bfloat16*>(Y), ldy,
-                                                     acc_out, ldacc, (int)M, (int)N, (int)K, act);
+                                                     acc_out, ldacc, (int)M, (int)N, (int)K, act, spr);
     return cuda_status(cudaGetLastError());
 }
 
@@ -596,15 +708,22 @@ inline dvdq_status launch_qgemm(const void* codes, const float* scales, const in
                                 const dvdq_act_quant& q, const dvdq_weights& w, const void* bias, int act,
                                 void* Y, int64_t ldy, int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
     if (M == 0) return DVDQ_OK;
+    // The int32 output does not depend on the scales: it always runs the per-token kernel, which
+    // adds up the code sums of a token's blocks itself.
     const bool raw = acc_out != nullptr;
-    if (q.bits == 4)
-        return raw ? launch_qgemm_t<4, true>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
-                   : launch_qgemm_t<4, false>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
-    if (q.bits == 8)
-        return raw ? launch_qgemm_t<8, true>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
-                   : launch_qgemm_t<8, false>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
-    return raw ? launch_qgemm_t<6, true>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
-               : launch_qgemm_t<6, false>(codes, scales, sums, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
+    const int spr = q.scale_group != 0 ? (int)(w.K / q.scale_group) : 1;  // code sums (and scales) per token
+#define DVDQ_GEMM_CASE(B)                                                                                          \
+    if (q.bits == B) {                                                                                             \
+        if (raw) return launch_qgemm_t<B, true, false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st); \
+        if (q.scale_group != 0)                                                                                    \
+            return launch_qgemm_t<B, false, true>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);      \
+        return launch_qgemm_t<B, false, false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);         \
+    }
+    DVDQ_GEMM_CASE(4)
+    DVDQ_GEMM_CASE(6)
+    DVDQ_GEMM_CASE(8)
+#undef DVDQ_GEMM_CASE
+    return DVDQ_ERR_BITS;
 }
 
 }  // namespace dvdq

@@ -59,7 +59,7 @@ template <int LOG2B, int BITS, bool FULL>
 __global__ void __maxnreg__(80)  // two CTAs of 12 warps per SM
 rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
           uint8_t* __restrict__ codes, float* __restrict__ scales, int32_t* __restrict__ sums,
-          int spans, int tokens_per_cta, int num_groups) {
+          int spans, int tokens_per_cta, int num_groups, int blockwise) {
     extern __shared__ float4 s_turn[];  // 256 float4 per warp
     __shared__ float s_max[2][kRqMaxWarps];
     __shared__ int s_sum[2][kRqMaxWarps];
@@ -249,14 +249,18 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
                 }
         // non-negative floats order like their bit patterns: one REDUX instead of five shuffles
         amax = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(amax)));
-        if (lane == 0) s_max[buf][warp] = amax;
-        // only the warps of this token meet: named barrier 1 + tl, spans * 32 threads
-        if (spans > 1) asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
-        if (spans > 1)
-            amax = __uint_as_float(__reduce_max_sync(
-                0xFFFFFFFFu, lane < spans ? __float_as_uint(s_max[buf][tl * spans + lane]) : 0u));
+        // Block-wise scales (one per token and per 1024-channel span): the warp's own absmax is
+        // the scale's, nothing is shared between warps.  Per-token scale: the token's warps meet.
+        if (!blockwise) {
+            if (lane == 0) s_max[buf][warp] = amax;
+            // only the warps of this token meet: named barrier 1 + tl, spans * 32 threads
+            if (spans > 1) asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
+            if (spans > 1)
+                amax = __uint_as_float(__reduce_max_sync(
+                    0xFFFFFFFFu, lane < spans ? __float_as_uint(s_max[buf][tl * spans + lane]) : 0u));
+        }
         // the previous iteration's token: all its code sums are in shared memory by now
-        if (sp == 0 && prev_token >= 0) {
+        if (!blockwise && sp == 0 && prev_token >= 0) {
             const int tsum = __reduce_add_sync(0xFFFFFFFFu, lane < spans ? s_sum[buf ^ 1u][tl * spans + lane] : 0);
             if (lane == 0) {
                 scales[prev_token] = (prev_amax * rs) / qmax;  // s_i = (absmax / sqrt(B)) / qmax
@@ -313,10 +317,18 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
             }
         }
         lsum = __reduce_add_sync(0xFFFFFFFFu, lsum);
+        if (blockwise) {
+            if (lane == 0) {
+                scales[(int64_t)token * spans + sp] = (amax * rs) / qmax;
+                sums[(int64_t)token * spans + sp] = lsum;
+            }
+            continue;
+        }
         if (lane == 0) s_sum[buf][warp] = lsum;
         prev_token = token;
         prev_amax = amax;
     }
+    if (blockwise) return;
     if (spans > 1) asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
     if (sp == 0 && prev_token >= 0) {
         const uint32_t buf = (it & 1u) ^ 1u;  // the last iteration's slots
@@ -330,7 +342,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
 
 template <int LOG2B, int BITS, bool FULL>
 static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t ldx, void* codes, float* scales,
-                                    int32_t* sums, cudaStream_t st) {
+                                    int32_t* sums, int blockwise, cudaStream_t st) {
     const int spans = (int)((K + kRqSpan - 1) / kRqSpan);
     if (spans > kRqMaxWarps) return DVDQ_ERR_SHAPE;
     int tpc = 12 / spans;  // at most 12 tokens per CTA: named barriers 1..12
@@ -361,20 +373,20 @@ static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t
     const int64_t resident = (int64_t)sm_count * blocks_per_sm[warps];
     const unsigned grid = (unsigned)(groups < resident ? groups : resident);
     kern<<<grid, threads, smem, st>>>((const __nv_bfloat16*)X, (int)M, (int)K, (int)ldx, (uint8_t*)codes, scales, sums, spans, tpc,
-                                      (int)groups);
+                                      (int)groups, blockwise);
     return cuda_status(cudaGetLastError());
 }
 
 template <int BITS>
 static dvdq_status launch_rq_bits(const void* X, int64_t M, int64_t K, int64_t ldx, int rot_block, void* codes,
-                                  float* scales, int32_t* sums, cudaStream_t st) {
+                                  float* scales, int32_t* sums, int blockwise, cudaStream_t st) {
     int log2b = 0;
     while ((1 << log2b) < rot_block) ++log2b;
     const bool full = K % kRqSpan == 0;
 #define DVDQ_RQ_CASE(L)                                                                              \
     case L:                                                                                          \
-        return full ? launch_rq_kernel<L, BITS, true>(X, M, K, ldx, codes, scales, sums, st)         \
-                    : launch_rq_kernel<L, BITS, false>(X, M, K, ldx, codes, scales, sums, st);
+        return full ? launch_rq_kernel<L, BITS, true>(X, M, K, ldx, codes, scales, sums, blockwise, st)         \
+                    : launch_rq_kernel<L, BITS, false>(X, M, K, ldx, codes, scales, sums, blockwise, st);
     switch (log2b) {
         DVDQ_RQ_CASE(0)
         DVDQ_RQ_CASE(6)
@@ -391,9 +403,9 @@ static dvdq_status launch_rq_bits(const void* X, int64_t M, int64_t K, int64_t l
 inline dvdq_status launch_rotate_quantize(const void* X, int64_t M, int64_t K, int64_t ldx, const dvdq_act_quant& q,
                                           void* codes, float* scales, int32_t* sums, cudaStream_t st) {
     if (M == 0) return DVDQ_OK;
-    if (q.bits == 4) return launch_rq_bits<4>(X, M, K, ldx, q.rot_block, codes, scales, sums, st);
-    if (q.bits == 6) return launch_rq_bits<6>(X, M, K, ldx, q.rot_block, codes, scales, sums, st);
-    return launch_rq_bits<8>(X, M, K, ldx, q.rot_block, codes, scales, sums, st);
+    if (q.bits == 4) return launch_rq_bits<4>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, st);
+    if (q.bits == 6) return launch_rq_bits<6>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, st);
+    return launch_rq_bits<8>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, st);
 }
 
 }  // namespace dvdq

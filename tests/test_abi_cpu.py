@@ -44,7 +44,14 @@ def test_size_queries():
     assert ws >= 1000 * 1536 + 8000 and ws % 256 == 0
     assert B.dvdq_qlinear_workspace_bytes(1000, 3072, B.ActQuant(4, 2048, 0)) == 0   # B > 1024
     assert B.dvdq_qlinear_workspace_bytes(1000, 1536, B.ActQuant(4, 1024, 0)) == 0   # B does not divide K
-    assert B.dvdq_qlinear_workspace_bytes(1000, 3072, B.ActQuant(4, 1024, 64)) == 0  # reserved granularity
+    assert B.dvdq_qlinear_workspace_bytes(1000, 3072, B.ActQuant(4, 1024, 64)) == 0  # granularity that is not built
+    # block-wise scales: one scale and one code sum per token and block of 1024 channels
+    qb = B.ActQuant(4, 256, 1024)
+    assert B.dvdq_act_scales_count(1000, 3072, q) == 1000
+    assert B.dvdq_act_scales_count(1000, 3072, qb) == 3000
+    assert B.dvdq_act_scales_count(1000, 3200, qb) == 0                               # K is not a multiple of the block
+    assert B.dvdq_qlinear_workspace_bytes(1000, 3072, qb) >= 1000 * 1536 + 2 * 3000 * 4
+    assert B.dvdq_qlinear_workspace_bytes(1000, 3072, qb) > B.dvdq_qlinear_workspace_bytes(1000, 3072, B.ActQuant(4, 256, 0))
 
 
 def test_status_strings():
@@ -70,6 +77,8 @@ def test_validation_happens_before_any_cuda_call():
     assert lib.dvdq_rotate_quantize(one, 4, 256, 256, C.byref(B.ActQuant(4, 96, 0)), one, one, one, None) == B.ERR_ROT_BLOCK
     assert lib.dvdq_rotate_quantize(one, 4, 256, 256, C.byref(B.ActQuant(4, 512, 0)), one, one, one, None) == B.ERR_ROT_BLOCK
     assert lib.dvdq_rotate_quantize(one, 4, 256, 256, C.byref(B.ActQuant(4, 256, 1)), one, one, one, None) == B.ERR_UNSUPPORTED
+    assert lib.dvdq_rotate_quantize(one, 4, 2048, 2048, C.byref(B.ActQuant(4, 256, 512)), one, one, one, None) == B.ERR_UNSUPPORTED
+    assert lib.dvdq_rotate_quantize(one, 4, 1536, 1536, C.byref(B.ActQuant(4, 256, 1024)), one, one, one, None) == B.ERR_SHAPE
     assert lib.dvdq_rotate_quantize(None, 4, 256, 256, C.byref(B.ActQuant(4, 256, 0)), one, one, one, None) == B.ERR_NULL
     assert lib.dvdq_rotate_quantize(C.c_void_p(8), 4, 256, 256, C.byref(B.ActQuant(4, 256, 0)), one, one, one, None) == B.ERR_ALIGN
     # weight handle checks

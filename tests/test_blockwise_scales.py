@@ -1,0 +1,185 @@
+"""Block-wise activation scales (one scale per token and per block of 1024 rotated channels; the
+granularity study of Sec. 3.2): the CUDA path against the oracle's block-wise quantizer and layer."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import dvdq_oracle as orc
+from paper_2505_18663_b200 import binding as B
+
+from helpers import bf16_values, check_codes_against_oracle, gpu_pack_weights, to_bits
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+G = 1024                # the block the library builds
+SCALE_RTOL = 1e-6
+Y_MAXNORM_RTOL = 4e-3
+
+
+def assert_device_ok():
+    status, detail = B.dvdq_last_device_status()
+    assert status == B.OK, f"device status {status} ({B.status_string(status)}), wait id {detail}"
+
+
+def synth_x(M, K, seed, outliers=4, gain=20.0):
+    g = torch.Generator().manual_seed(seed)
+    x = torch.randn(M, K, generator=g)
+    # tokens differ in size and the outlier channels sit in some blocks only: the case block-wise
+    # scales are for
+    x *= torch.exp(torch.randn(M, 1, generator=g))
+    if outliers:
+        x[:, torch.randperm(K, generator=g)[:outliers]] *= gain
+    return x.to(torch.bfloat16)
+
+
+def synth_w(N, K, seed, mode):
+    g = torch.Generator().manual_seed(seed)
+    w = torch.randn(N, K, generator=g) * 0.02
+    if mode == "minmax":
+        w += 0.004 * torch.randn(N, 1, generator=g)
+    return w.to(torch.bfloat16)
+
+
+def gpu_rotate_quantize_blockwise(x_dev, bits, Bk):
+    M, K = x_dev.shape
+    q = B.ActQuant(bits, Bk, G)
+    n = B.dvdq_act_scales_count(M, K, q)
+    assert n == M * (K // G)
+    codes = torch.empty(B.dvdq_act_codes_bytes(M, K, bits), dtype=torch.uint8, device=DEV)
+    scales = torch.full((n,), -1.0, dtype=torch.float32, device=DEV)
+    sums = torch.full((n,), 123456, dtype=torch.int32, device=DEV)
+    B.dvdq_rotate_quantize(x_dev, q, codes, scales, sums)
+    nat = torch.empty(M, K, dtype=torch.int8, device=DEV)
+    B.dvdq_unpack_act_codes(codes, M, K, q, nat)
+    torch.cuda.synchronize()
+    return codes, scales.view(M, K // G), sums.view(M, K // G), nat
+
+
+def check_blockwise_codes(nat, codes_or, xt, s64):
+    for g in range(codes_or.shape[1] // G):
+        sl = slice(g * G, (g + 1) * G)
+        check_codes_against_oracle(nat[:, sl], codes_or[:, sl], xt[:, sl], s64[:, g])
+
+
+@pytest.mark.parametrize("bits", [4, 6, 8])
+@pytest.mark.parametrize("M,K,Bk", [(300, 3072, 256), (257, 2048, 1024), (65, 1024, 64), (130, 5120, 128)])
+def test_rotate_quantize_blockwise_matches_oracle(M, K, Bk, bits):
+    x = synth_x(M, K, seed=M + K + bits)
+    xt = orc.rotate(to_bits(x), Bk)
+    codes_or, s64, s32 = orc.act_quantize_grouped(xt, bits, G)
+    _, scales, sums, nat = gpu_rotate_quantize_blockwise(x.to(DEV), bits, Bk)
+    assert_device_ok()
+    s = scales.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(s - s64) <= SCALE_RTOL * s64)
+    nat = nat.cpu().numpy()
+    check_blockwise_codes(nat, codes_or, xt, s64)
+    # the sums belong to the codes that were written, block by block, exactly
+    assert np.array_equal(sums.cpu().numpy(), nat.astype(np.int64).reshape(M, K // G, G).sum(axis=2))
+
+
+def test_blockwise_equals_per_token_when_there_is_one_block():
+    M, K, bits, Bk = 200, 1024, 4, 256
+    x = synth_x(M, K, seed=5).to(DEV)
+    pc, ps, pS, pn = gpu_rotate_quantize_blockwise(x, bits, Bk)
+    q = B.ActQuant(bits, Bk, 0)
+    codes = torch.empty_like(pc)
+    scales = torch.empty(M, dtype=torch.float32, device=DEV)
+    sums = torch.empty(M, dtype=torch.int32, device=DEV)
+    B.dvdq_rotate_quantize(x, q, codes, scales, sums)
+    torch.cuda.synchronize()
+    assert torch.equal(codes, pc) and torch.equal(scales, ps.view(-1)) and torch.equal(sums, pS.view(-1))
+
+
+LAYER_CASES = [
+    # M, N, K, B, bits, weight mode: M and N tails (N tail against the 128-wide tile), 1 to 5 blocks, z != 8
+    (257, 392, 3072, 256, 4, "minmax"),
+    (300, 128, 1024, 1024, 4, "symmetric"),
+    (130, 520, 2048, 128, 6, "minmax"),
+    (513, 256, 5120, 512, 8, "minmax"),
+]
+
+
+def pack_blockwise(codes_np, bits, Bk):
+    M, K = codes_np.shape
+    q = B.ActQuant(bits, Bk, G)
+    nat = torch.from_numpy(codes_np.astype(np.int8)).to(DEV)
+    packed = torch.empty(B.dvdq_act_codes_bytes(M, K, bits), dtype=torch.uint8, device=DEV)
+    sums = torch.empty(M * (K // G), dtype=torch.int32, device=DEV)
+    B.dvdq_pack_act_codes(nat, q, packed, sums)
+    return packed, sums, q
+
+
+@pytest.mark.parametrize("act", [0, 1])
+@pytest.mark.parametrize("M,N,K,Bk,bits,mode", LAYER_CASES)
+def test_qgemm_blockwise_on_oracle_codes_and_scales(M, N, K, Bk, bits, mode, act):
+    x = synth_x(M, K, seed=3 * M + N)
+    u, d, z = orc.prepare_weights(to_bits(synth_w(N, K, M + N, mode)), Bk, mode)
+    codes, s64, s32 = orc.act_quantize_grouped(orc.rotate(to_bits(x), Bk), bits, G)
+    bias = (torch.randn(N, generator=torch.Generator().manual_seed(N)) * 0.05).to(torch.bfloat16)
+    y_or = bf16_values(orc.combine_grouped(codes, u, z, s32, d, G, to_bits(bias), act))
+    w, blob = gpu_pack_weights(u, d, z, Bk)
+    packed, sums, q = pack_blockwise(codes, bits, Bk)
+    assert np.array_equal(sums.cpu().numpy().reshape(M, K // G), codes.reshape(M, K // G, G).sum(axis=2))
+    Y = torch.zeros(M, N + 8, dtype=torch.bfloat16, device=DEV)[:, :N]
+    B.dvdq_qgemm(packed, torch.from_numpy(np.ascontiguousarray(s32)).to(DEV), sums, M, q, w, bias.to(DEV), act, Y)
+    assert_device_ok()
+    y = Y.to(torch.float64).cpu().numpy()
+    assert np.abs(y - y_or).max() <= Y_MAXNORM_RTOL * np.abs(y_or).max()
+    # same integer inputs: what differs is fp32 against fp64 in the combination of at most five
+    # block terms -- a few ulp of fp32, far below the bf16 rounding, so nearly every output is equal
+    assert np.mean(y != y_or) < 0.02
+    # the int32 output does not depend on the scales: bit-exact against the whole-K integer GEMM
+    acc = torch.zeros(M, N, dtype=torch.int32, device=DEV)
+    B.dvdq_qgemm_int32(packed, sums, M, q, w, acc)
+    assert_device_ok()
+    assert np.array_equal(acc.cpu().numpy(), orc.int_gemm(codes, u, z))
+
+
+@pytest.mark.parametrize("M,N,K,Bk,bits,mode", LAYER_CASES)
+def test_qlinear_blockwise_matches_oracle_end_to_end(M, N, K, Bk, bits, mode):
+    x = synth_x(M, K, seed=7 * M + N)
+    u, d, z = orc.prepare_weights(to_bits(synth_w(N, K, M + N + 1, mode)), Bk, mode)
+    out = orc.qlinear_grouped(to_bits(x), u, d, z, Bk, bits, G)
+    w, blob = gpu_pack_weights(u, d, z, Bk)
+    q = B.ActQuant(bits, Bk, G)
+    ws = torch.empty(B.dvdq_qlinear_workspace_bytes(M, K, q), dtype=torch.uint8, device=DEV)
+    Y = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+    B.dvdq_qlinear(x.to(DEV), q, w, None, 0, Y, ws)
+    nat = torch.empty(M, K, dtype=torch.int8, device=DEV)
+    B.dvdq_unpack_act_codes(ws, M, K, q, nat)
+    assert_device_ok()
+    nat = nat.cpu().numpy()
+    # codes first (equal, or +-1 on a rounding tie), then the rest of the layer on the validated codes
+    check_blockwise_codes(nat, out["codes"], out["xt"], out["scale64"])
+    y_or = bf16_values(orc.combine_grouped(nat.astype(np.int32), u, z, out["scale32"], d, G))
+    y = Y.to(torch.float64).cpu().numpy()
+    assert np.abs(y - y_or).max() <= Y_MAXNORM_RTOL * np.abs(y_or).max()
+    # and the static-scratch entry point takes the same option
+    if B.dvdq_qlinear_workspace_bytes(M, K, q) <= B.STATIC_SCRATCH_BYTES:
+        Y2 = torch.empty_like(Y)
+        B.dvdq_qlinear_static(x.to(DEV), q, w, None, 0, Y2)
+        assert_device_ok()
+        assert torch.equal(Y, Y2)
+
+
+def test_blockwise_scales_lower_the_quantization_error():
+    """What the option is for: with outlier channels confined to one block, the other blocks get a
+    finer grid, so the layer output is closer to the unquantized product than with one scale per token."""
+    M, N, K, Bk, bits = 256, 256, 4096, 256, 4
+    g = torch.Generator().manual_seed(11)
+    x = torch.randn(M, K, generator=g)
+    x[:, 5:9] *= 30.0                      # all outliers in the first rotation block
+    x = x.to(torch.bfloat16)
+    wb = synth_w(N, K, 12, "symmetric")
+    u, d, z = orc.prepare_weights(to_bits(wb), Bk, "symmetric")
+    w, blob = gpu_pack_weights(u, d, z, Bk)
+    exact = orc.exact_linear(bf16_values(to_bits(x)), bf16_values(to_bits(wb)))
+    errs = []
+    for group in (0, G):
+        q = B.ActQuant(bits, Bk, group)
+        ws = torch.empty(B.dvdq_qlinear_workspace_bytes(M, K, q), dtype=torch.uint8, device=DEV)
+        Y = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+        B.dvdq_qlinear(x.to(DEV), q, w, None, 0, Y, ws)
+        assert_device_ok()
+        errs.append(np.linalg.norm(Y.to(torch.float64).cpu().numpy() - exact))
+    assert errs[1] < 0.85 * errs[0], errs
