@@ -263,8 +263,9 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             // Block-wise scales: every block of 1024 codes has its own int32 accumulator (the two
             // accumulators alternate) and its own scale per token.  This warp keeps the running
             // fp32 sum over blocks of its 32 rows in tensor-memory columns [256, 384) -- lanes only
-            // it touches -- and dequantizes after the last block:
-            //     y = Delta_n * sum_g s_ig (acc_g - (z_n - 8) S_ig) + bias_n.
+            // it touches -- and dequantizes after the last block.  acc_g here is the sum over the
+            // stored codes (u - 8); the rest of the zero point is one term per row:
+            //     y = Delta_n * (sum_g s_ig acc_g - (z_n - 8) T_i) + bias_n,  T_i = sum_g s_ig S_ig.
             constexpr uint32_t kFloatCol = 2 * BN;
             uint32_t lt = 0, nstore = 0;
             for (int tile = pair; tile < num_tiles; tile += num_pairs) {
@@ -282,54 +283,49 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 const int row = m0 + q * 32 + lane;
                 const bool row_ok = row < M;
                 const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+                // the zero-point term of all blocks at once: T_i = sum_g s_ig S_ig (each S_ig is exact in fp32)
+                float T = 0.f;
+                if (row_ok)
+                    for (int g = 0; g < NG; ++g) T = fmaf(scales[(int64_t)row * NG + g], (float)sums[(int64_t)row * NG + g], T);
                 bool ok = true;
                 for (int g = 0; g < NG; ++g, ++lt) {
                     const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
+                    const float s_k = (row_ok ? scales[(int64_t)row * NG + g] : 0.f) * (1.0f / (float)(1 << kShift));
                     if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) { ok = false; break; }
                     tc_fence_after();
-                    const float s_g = row_ok ? scales[(int64_t)row * NG + g] : 0.f;
-                    const float S_g = row_ok ? (float)sums[(int64_t)row * NG + g] : 0.f;
-                    const float s_k = s_g * (1.0f / (float)(1 << kShift)), nS_k = -S_g * (float)(1 << kShift);
                     const bool last = g == NG - 1;
 #pragma unroll 1
-                    for (int hc = 0; hc < BN / 16; ++hc) {
-                        uint32_t r[16], f[16];
-                        tmem_ld_32x16(tmem_base + a * BN + hc * 16 + lane_addr, r);
-                        if (g > 0) tmem_ld_32x16(tmem_base + kFloatCol + hc * 16 + lane_addr, f);
+                    for (int hc = 0; hc < BN / 32; ++hc) {
+                        uint32_t r[32], f[32];
+                        tmem_ld_32x32(tmem_base + a * BN + hc * 32 + lane_addr, r);
+                        if (g > 0) tmem_ld_32x32(tmem_base + kFloatCol + hc * 32 + lane_addr, f);
                         tmem_ld_wait();
-                        float v[16];
 #pragma unroll
-                        for (int j = 0; j < 16; j += 4) {
-                            const float4 z4 = lds128f(c_zc + 4 * (hc * 16 + j));
-                            const float zz[4] = {z4.x, z4.y, z4.z, z4.w};
-#pragma unroll
-                            for (int t = 0; t < 4; ++t) {
-                                const float part = fmaf(zz[t], nS_k, (float)(int32_t)r[j + t]) * s_k;  // the fma is exact
-                                v[j + t] = g > 0 ? __uint_as_float(f[j + t]) + part : part;
-                            }
-                        }
+                        for (int t = 0; t < 32; ++t)  // running sum of s_ig * acc_g (the raw accumulator is 2^kShift x the true one)
+                            f[t] = __float_as_uint(fmaf((float)(int32_t)r[t], s_k, g > 0 ? __uint_as_float(f[t]) : 0.f));
                         if (!last) {
-#pragma unroll
-                            for (int t = 0; t < 16; ++t) f[t] = __float_as_uint(v[t]);
-                            tmem_st_32x16(tmem_base + kFloatCol + hc * 16 + lane_addr, f);
+                            tmem_st_32x32(tmem_base + kFloatCol + hc * 32 + lane_addr, f);
                             continue;
                         }
                         // last block: dequantize, round, stage 64 columns per TMA store
-                        if ((hc & 3) == 0) {
+                        if ((hc & 1) == 0) {
                             if (lane == 0) tma_store_wait_read<1>();
                             __syncwarp();
                         }
                         const uint32_t buf = stg0 + (nstore & 1u) * (32 * 128);
 #pragma unroll
-                        for (int j = 0; j < 16; j += 8) {
-                            const float4 d0 = lds128f(c_delta + 4 * (hc * 16 + j)), d1 = lds128f(c_delta + 4 * (hc * 16 + j + 4));
-                            const float4 b0 = lds128f(c_bias + 4 * (hc * 16 + j)), b1 = lds128f(c_bias + 4 * (hc * 16 + j + 4));
+                        for (int j = 0; j < 32; j += 8) {
+                            const float4 d0 = lds128f(c_delta + 4 * (hc * 32 + j)), d1 = lds128f(c_delta + 4 * (hc * 32 + j + 4));
+                            const float4 z0 = lds128f(c_zc + 4 * (hc * 32 + j)), z1 = lds128f(c_zc + 4 * (hc * 32 + j + 4));
+                            const float4 b0 = lds128f(c_bias + 4 * (hc * 32 + j)), b1 = lds128f(c_bias + 4 * (hc * 32 + j + 4));
                             const float dl[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+                            const float zz[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
                             const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
                             uint32_t pk[4];
 #pragma unroll
                             for (int t = 0; t < 8; t += 2) {
-                                float y0 = fmaf(v[j + t], dl[t], bb[t]), y1 = fmaf(v[j + t + 1], dl[t + 1], bb[t + 1]);
+                                float y0 = fmaf(fmaf(-zz[t], T, __uint_as_float(f[j + t])), dl[t], bb[t]);
+                                float y1 = fmaf(fmaf(-zz[t + 1], T, __uint_as_float(f[j + t + 1])), dl[t + 1], bb[t + 1]);
                                 if (act == 1) {
                                     y0 = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(y0)));
                                     y1 = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(y1)));
@@ -337,13 +333,13 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                                 __nv_bfloat162 b2 = __floats2bfloat162_rn(y0, y1);
                                 pk[t >> 1] = *reinterpret_cast<uint32_t*>(&b2);
                             }
-                            const int ch = (2 * (hc & 3) + (j >> 3)) ^ (lane & 7);
+                            const int ch = (4 * (hc & 1) + (j >> 3)) ^ (lane & 7);
                             sts128(buf + lane * 128 + ch * 16, pk[0], pk[1], pk[2], pk[3]);
                         }
-                        if ((hc & 3) == 3) {
+                        if (hc & 1) {
                             fence_proxy_async_smem();
                             __syncwarp();
-                            const int nb = n0 + (hc >> 2) * 64;
+                            const int nb = n0 + (hc >> 1) * 64;
                             if (lane == 0 && nb < N && m0 + q * 32 < M) {
                                 tma_store_2d(&tmY, buf, nb, m0 + q * 32);
                                 tma_store_commit();
@@ -351,10 +347,12 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                             ++nstore;
                         }
                     }
-                    if (!last) tmem_st_wait();
+                    // the accumulator is read: the MMA warp may have it back before this warp's
+                    // running sums have landed (nobody else touches those columns)
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty(a), 0));
+                    if (!last) tmem_st_wait();
                 }
                 if (!ok) break;
             }
