@@ -271,7 +271,7 @@ def test_qlinear_matches_oracle_end_to_end(M, N, K, Bk, bits, mode):
 
 
 def test_tiny_config_full_comparison():
-    """BASELINE config 1: 256 tokens x 256 -> 256, four outlier channels x20, W4A4, B = 256, seed 0."""
+    """The small single-layer case: 256 tokens x 256 -> 256, four outlier channels x20, W4A4, B = 256, seed 0."""
     wl = W.WORKLOADS["tiny"]
     layer = wl.layers[0]
     x = W.make_activations(wl, layer.K)
