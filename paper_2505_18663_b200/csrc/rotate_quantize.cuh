@@ -53,22 +53,33 @@ __device__ __forceinline__ uint32_t stage_a_entry(int m, int s) {
 
 // One warp-span of work per loop iteration; CTAs are persistent and walk over groups of
 // tokens_per_cta tokens.  FULL = every span is complete (K a multiple of 1024): no per-chunk
-// predicates.  Per iteration there is ONE CTA barrier (the token absmax); the code sums of
-// iteration i are finalised after the barrier of iteration i + 1 from double-buffered slots.
+// predicates.  Per iteration the warps of a token meet once (a named barrier) for the token's
+// absmax, which they combine with a shared-memory atomic max; their code sums are added up the
+// same way and written out after the next iteration's barrier.  The slots rotate over three sets:
+// a warp's whole iteration is a chain of dependent steps, so the exchange is kept as short as
+// it can be (an atomic, the barrier, one broadcast load).
 template <int LOG2B, int BITS, bool FULL>
 __global__ void __maxnreg__(80)  // two CTAs of 12 warps per SM
 rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
           uint8_t* __restrict__ codes, float* __restrict__ scales, int32_t* __restrict__ sums,
           int spans, int tokens_per_cta, int num_groups, int blockwise) {
     extern __shared__ float4 s_turn[];  // 256 float4 per warp
-    __shared__ float s_max[2][kRqMaxWarps];
-    __shared__ int s_sum[2][kRqMaxWarps];
+    __shared__ unsigned s_max[3][kRqMaxWarps];  // [slot set][token of the CTA]: bits of the token absmax
+    __shared__ int s_sum[3][kRqMaxWarps];       // sum of the token's codes
     constexpr bool kRot = LOG2B > 0;
     constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
     constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: ulp 1, so the fma rounds to an integer
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int tl = warp / spans, sp = warp - tl * spans;
     const int g = lane >> 2, t = lane & 3;
+    const bool team = !blockwise && spans > 1;  // the token's warps exchange absmax and code sums
+    if (team) {
+        if (threadIdx.x < 3 * kRqMaxWarps) {
+            (&s_max[0][0])[threadIdx.x] = 0u;
+            (&s_sum[0][0])[threadIdx.x] = 0;
+        }
+        __syncthreads();
+    }
 
     // ---- loop invariants
     // stage-A matrix fragment (H_16, or the identity without a rotation)
@@ -129,9 +140,13 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
     if (group < num_groups) load_span(raw, group);
     int prev_token = -1;
     float prev_amax = 0.f;
-    uint32_t it = 0;
-    for (; group < num_groups; group += gridDim.x, ++it) {
-        const uint32_t buf = it & 1u;
+    int cur = 0, nxt = 1, prv = 2;  // slot sets of this iteration, the next one and the previous one
+    for (; group < num_groups; group += gridDim.x) {
+        // the next iteration's slots start from zero; their last readers passed the previous barrier
+        if (team && sp == 0 && lane == 0) {
+            s_max[nxt][tl] = 0u;
+            s_sum[nxt][tl] = 0;
+        }
         // A token past the end is a clamped duplicate of the last one: it computes and stores
         // the same bytes to the same places, which needs no predicate.
         int token = group * tokens_per_cta + tl;
@@ -251,21 +266,11 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
         amax = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(amax)));
         // Block-wise scales (one per token and per 1024-channel span): the warp's own absmax is
         // the scale's, nothing is shared between warps.  Per-token scale: the token's warps meet.
-        if (!blockwise) {
-            if (lane == 0) s_max[buf][warp] = amax;
+        if (team) {
+            if (lane == 0) atomicMax(&s_max[cur][tl], __float_as_uint(amax));
             // only the warps of this token meet: named barrier 1 + tl, spans * 32 threads
-            if (spans > 1) asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
-            if (spans > 1)
-                amax = __uint_as_float(__reduce_max_sync(
-                    0xFFFFFFFFu, lane < spans ? __float_as_uint(s_max[buf][tl * spans + lane]) : 0u));
-        }
-        // the previous iteration's token: all its code sums are in shared memory by now
-        if (!blockwise && sp == 0 && prev_token >= 0) {
-            const int tsum = __reduce_add_sync(0xFFFFFFFFu, lane < spans ? s_sum[buf ^ 1u][tl * spans + lane] : 0);
-            if (lane == 0) {
-                scales[prev_token] = (prev_amax * rs) / qmax;  // s_i = (absmax / sqrt(B)) / qmax
-                sums[prev_token] = tsum;
-            }
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
+            amax = __uint_as_float(s_max[cur][tl]);
         }
         const float inv = amax > 0.f ? qmax / amax : 0.f;
         const uint64_t inv2 = f2_pack(inv, inv), magic2 = f2_pack(kMagic, kMagic);
@@ -324,19 +329,33 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
             }
             continue;
         }
-        if (lane == 0) s_sum[buf][warp] = lsum;
+        if (!team) {  // a single span per token
+            if (lane == 0) {
+                scales[token] = (amax * rs) / qmax;
+                sums[token] = lsum;
+            }
+            continue;
+        }
+        if (lane == 0) {
+            atomicAdd(&s_sum[cur][tl], lsum);
+            // the previous iteration's token: its warps added their code sums before this iteration's barrier
+            if (sp == 0 && prev_token >= 0) {
+                scales[prev_token] = (prev_amax * rs) / qmax;  // s_i = (absmax / sqrt(B)) / qmax
+                sums[prev_token] = s_sum[prv][tl];
+            }
+        }
         prev_token = token;
         prev_amax = amax;
+        const int r = prv;
+        prv = cur;
+        cur = nxt;
+        nxt = r;
     }
-    if (blockwise) return;
-    if (spans > 1) asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
-    if (sp == 0 && prev_token >= 0) {
-        const uint32_t buf = (it & 1u) ^ 1u;  // the last iteration's slots
-        const int tsum = __reduce_add_sync(0xFFFFFFFFu, lane < spans ? s_sum[buf][tl * spans + lane] : 0);
-        if (lane == 0) {
-            scales[prev_token] = (prev_amax * rs) / qmax;
-            sums[prev_token] = tsum;
-        }
+    if (!team) return;
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
+    if (sp == 0 && lane == 0 && prev_token >= 0) {
+        scales[prev_token] = (prev_amax * rs) / qmax;
+        sums[prev_token] = s_sum[prv][tl];  // the last iteration's slots
     }
 }
 
