@@ -107,10 +107,10 @@ def layer_ops(M, layer):
     return 2.0 * M * layer.N * layer.K
 
 
-def rq_bytes(M, layer, scale_group=0):
-    """Algorithmic HBM bytes of rotate-quantize: bf16 row in, packed codes + scales + code sums out."""
+def rq_bytes(M, layer, scale_group=0, container=0):
+    """Algorithmic HBM bytes of rotate-quantize: bf16 row in, codes as stored + scales + code sums out."""
     per_token = layer.K // scale_group if scale_group else 1
-    return M * (2.0 * layer.K + layer.K * layer.bits / 8.0 + 8.0 * per_token)
+    return M * (2.0 * layer.K + layer.K * (container or layer.bits) / 8.0 + 8.0 * per_token)
 
 
 # ------------------------------------------------------------------ the CPU oracle leg
@@ -174,6 +174,7 @@ def config_of(wl, args):
                 f"{l.K}->{l.N} A{l.bits} B{l.rot_block}" for l in wl.layers),
             "weights": "4-bit per-output-channel codes (random, Gaussian-shaped)",
             "l2_policy": "inputs larger than L2 (every layer streams >= 400 MB)",
+            "act_codes": ("one int8 per code" if args.container else "packed, b bits per code"),
             "act_scales": (f"one per token and block of {args.scale_group} channels" if args.scale_group else "one per token"),
             "parallelism": f"dp{args.gpus} (token-sharded replicas, no collective)"}
 
@@ -212,8 +213,8 @@ def run_cuda(args, wl):
         blob = torch.empty(B.dvdq_weight_blob_bytes(layer.N, layer.K), dtype=torch.uint8, device=dev)
         w = B.dvdq_pack_weights(u, d, z, layer.rot_block, blob)
         del u
-        q = B.ActQuant(layer.bits, layer.rot_block, args.scale_group)
-        codes = torch.empty(B.dvdq_act_codes_bytes(M, layer.K, layer.bits), dtype=torch.uint8, device=dev)
+        q = B.ActQuant(layer.bits, layer.rot_block, args.scale_group, args.container)
+        codes = torch.empty(B.dvdq_act_codes_bytes_q(M, layer.K, q), dtype=torch.uint8, device=dev)
         n_scales = B.dvdq_act_scales_count(M, layer.K, q)
         if n_scales == 0:
             raise SystemExit(f"layer {layer.K}->{layer.N}: activation quantizer options not supported")
@@ -276,13 +277,13 @@ def run_cuda(args, wl):
     int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
     gemm_ops = sum(layer_ops(M, L["layer"]) for L in layers)
     gemm_tops = gemm_ops / (sum(gm_ms) * 1e-3) / 1e12
-    rq_total_bytes = sum(rq_bytes(M, L["layer"], args.scale_group) for L in layers)
+    rq_total_bytes = sum(rq_bytes(M, L["layer"], args.scale_group, args.container) for L in layers)
     rq_gbs = rq_total_bytes / (sum(rq_ms) * 1e-3) / 1e9
     stages = []
     for li, L in enumerate(layers):
         layer = L["layer"]
         stages.append({"layer": f"{layer.K}->{layer.N} A{layer.bits}",
-                       "rq_ms": rq_ms[li], "rq_gbs": rq_bytes(M, layer, args.scale_group) / (rq_ms[li] * 1e-3) / 1e9,
+                       "rq_ms": rq_ms[li], "rq_gbs": rq_bytes(M, layer, args.scale_group, args.container) / (rq_ms[li] * 1e-3) / 1e9,
                        "qgemm_ms": gm_ms[li], "qgemm_tops": layer_ops(M, layer) / (gm_ms[li] * 1e-3) / 1e12})
 
     # ---- end to end through dvdq_qlinear with HOST buffers (pinned), copies inside the timed region
@@ -296,7 +297,7 @@ def run_cuda(args, wl):
         return
 
     # the ncu counters were taken on the default workload (hunyuan, its own bit widths, per-token scales)
-    captured = wl.name == "hunyuan" and wl.M == 65536 and args.bits == 0 and args.scale_group == 0
+    captured = wl.name == "hunyuan" and wl.M == 65536 and args.bits == 0 and args.scale_group == 0 and args.container == 0
     line = {
         "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -413,6 +414,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling runs)")
+    ap.add_argument("--container", type=int, default=0,
+                    help="0: activation codes packed (b bits each); 8: one int8 per code")
     ap.add_argument("--scale-group", type=int, default=0,
                     help="0: one activation scale per token; 1024: one per token and block of 1024 channels")
     ap.add_argument("--bits", type=int, default=0, help="override the activation bit width of every layer (4, 6 or 8)")

@@ -65,11 +65,18 @@ const char* dvdq_status_string(dvdq_status s);
  *               and per block of 1024 consecutive rotated channels (K % 1024 == 0; every block
  *               is quantized on its own, the GEMM rescales per block).  Other values give
  *               DVDQ_ERR_UNSUPPORTED.
+ *   container_bits  how the codes are kept between the transform and the GEMM (the values are
+ *               the same either way): 0 = packed, b bits per code; 8 = one int8 per code.
+ *               int8 tensor cores are the narrowest integer ones on sm_100, so packed codes
+ *               are widened inside the GEMM; codes kept in bytes go from HBM into the tensor
+ *               core's operand layout untouched, which is faster, at K instead of K*b/8 bytes
+ *               per token.  Other values give DVDQ_ERR_UNSUPPORTED.
  */
 typedef struct {
     int32_t bits;
     int32_t rot_block;
     int32_t scale_group;
+    int32_t container_bits;
 } dvdq_act_quant;
 
 /*
@@ -92,6 +99,8 @@ typedef struct {
 
 /* Bytes of the packed activation codes of an [M, K] tensor: M * K * bits / 8. 0 on bad input. */
 size_t dvdq_act_codes_bytes(int64_t M, int64_t K, int32_t bits);
+/* The same for a quantizer description: M * K * (container_bits ? container_bits : bits) / 8. */
+size_t dvdq_act_codes_bytes_q(int64_t M, int64_t K, const dvdq_act_quant* q);
 /* Number of scales (and of code sums) of an [M, K] tensor: M, or M * K / 1024 block-wise. 0 on bad input. */
 size_t dvdq_act_scales_count(int64_t M, int64_t K, const dvdq_act_quant* q);
 /* Bytes of the device blob that dvdq_pack_weights() writes for an [N, K] matrix. 0 on bad input. */
@@ -105,7 +114,7 @@ size_t dvdq_qlinear_workspace_bytes(int64_t M, int64_t K, const dvdq_act_quant* 
  * a_i = max_k |x~_ik|, s_i = a_i / qmax, c_ik = round_half_even(x~_ik / s_i).
  *
  *   X_bf16         [M, K] bf16, row pitch ldx elements; 16-byte aligned, ldx % 8 == 0
- *   codes_out      dvdq_act_codes_bytes(M, K, bits) bytes, 16-byte aligned (opaque layout)
+ *   codes_out      dvdq_act_codes_bytes_q(M, K, q) bytes, 16-byte aligned (opaque layout)
  *   scales_out     [M] fp32, s_i  (0 for an all-zero token, whose codes are all 0);
  *                  block-wise: [M, K/1024], one scale per token and block
  *   code_sums_out  [M] int32, sum_k c_ik (used by the GEMM for the weight zero point);

@@ -20,7 +20,7 @@ OK, ERR_NULL, ERR_SHAPE, ERR_BITS, ERR_ROT_BLOCK, ERR_ALIGN, ERR_WORKSPACE, ERR_
     ERR_CUDA, ERR_DEVICE_TIMEOUT, ERR_UNSUPPORTED = range(12)
 
 EXPORTS = [
-    "dvdq_status_string", "dvdq_version", "dvdq_act_codes_bytes", "dvdq_act_scales_count", "dvdq_weight_blob_bytes",
+    "dvdq_status_string", "dvdq_version", "dvdq_act_codes_bytes", "dvdq_act_codes_bytes_q", "dvdq_act_scales_count", "dvdq_weight_blob_bytes",
     "dvdq_qlinear_workspace_bytes", "dvdq_rotate_quantize", "dvdq_pack_weights", "dvdq_qgemm",
     "dvdq_qlinear", "dvdq_qlinear_static", "dvdq_qgemm_int32", "dvdq_pack_act_codes", "dvdq_unpack_act_codes",
     "dvdq_unpack_weights", "dvdq_last_device_status",
@@ -35,8 +35,10 @@ class DvdqError(RuntimeError):
 
 
 class ActQuant(C.Structure):
-    """dvdq_act_quant: the activation quantizer of Eq. 10 (bits, rotation block, scale granularity)."""
-    _fields_ = [("bits", C.c_int32), ("rot_block", C.c_int32), ("scale_group", C.c_int32)]
+    """dvdq_act_quant: the activation quantizer of Eq. 10 (bits, rotation block, scale granularity)
+    and how its codes are stored (container_bits: 0 = packed, 8 = one int8 per code)."""
+    _fields_ = [("bits", C.c_int32), ("rot_block", C.c_int32), ("scale_group", C.c_int32),
+                ("container_bits", C.c_int32)]
 
 
 class Weights(C.Structure):
@@ -78,6 +80,7 @@ def load():
         "dvdq_status_string": (C.c_char_p, [C.c_int]),
         "dvdq_version": (i32, []),
         "dvdq_act_codes_bytes": (sz, [i64, i64, i32]),
+        "dvdq_act_codes_bytes_q": (sz, [i64, i64, aq]),
         "dvdq_act_scales_count": (sz, [i64, i64, aq]),
         "dvdq_weight_blob_bytes": (sz, [i64, i64]),
         "dvdq_qlinear_workspace_bytes": (sz, [i64, i64, aq]),
@@ -144,6 +147,10 @@ def dvdq_version() -> int:
 
 def dvdq_act_codes_bytes(M: int, K: int, bits: int) -> int:
     return int(load().dvdq_act_codes_bytes(M, K, bits))
+
+
+def dvdq_act_codes_bytes_q(M: int, K: int, q: ActQuant) -> int:
+    return int(load().dvdq_act_codes_bytes_q(M, K, C.byref(q)))
 
 
 def dvdq_act_scales_count(M: int, K: int, q: ActQuant) -> int:

@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libdvdq.so")
 SOURCES = ["dvdq_lib.cu"]
-DEPS = ["dvdq_lib.cu", "dvdq_common.cuh", "rotate_quantize.cuh", "pack.cuh", "qgemm.cuh", "gbs.cuh", "bgr.cuh"]
+DEPS = ["dvdq_lib.cu", "dvdq_common.cuh", "rotate_quantize.cuh", "pack.cuh", "qgemm.cuh", "qgemm_ss.cuh", "gbs.cuh", "bgr.cuh"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

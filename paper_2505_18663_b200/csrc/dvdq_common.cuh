@@ -56,6 +56,8 @@ __host__ __device__ inline BlobLayout blob_layout(int64_t N, int64_t K) {
 // widening of 16 codes into four int8 words a shift and a mask per word.  A8 = K bytes: int8 codes,
 // each group of 8 channels as its four even channels followed by its four odd ones.
 __host__ __device__ inline int64_t act_row_bytes(int64_t K, int bits) { return K * bits / 8; }
+// bits per stored code: the container's, or the code width when the codes are packed
+inline int storage_bits(const dvdq_act_quant& q) { return q.container_bits ? q.container_bits : q.bits; }
 __host__ __device__ inline int hi_field_shift(int a, int i) { return 2 * (4 * (i >> 1) + 2 * a + (i & 1)); }
 
 // ------------------------------------------------------------------ device status word
@@ -167,6 +169,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* m, 
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y)
         : "memory");
+}
+
+// Asks L2 for the tile a later tma_load_2d with the same coordinates will copy.
+__device__ __forceinline__ void tma_prefetch_l2_2d(const CUtensorMap* m, int32_t x, int32_t y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(x), "r"(y)
+                 : "memory");
 }
 
 // 2-D tiled TMA store shared -> global (bulk async-group completion); elements outside the

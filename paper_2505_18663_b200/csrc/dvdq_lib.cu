@@ -7,6 +7,7 @@
 #include "gbs.cuh"
 #include "pack.cuh"
 #include "qgemm.cuh"
+#include "qgemm_ss.cuh"
 #include "rotate_quantize.cuh"
 
 namespace dvdq {
@@ -40,6 +41,7 @@ static dvdq_status validate_k(int64_t K) {
 dvdq_status validate_act_quant(const dvdq_act_quant* q, int64_t K) {
     if (!q) return DVDQ_ERR_NULL;
     if (q->bits != 4 && q->bits != 6 && q->bits != 8) return DVDQ_ERR_BITS;
+    if (q->container_bits != 0 && q->container_bits != 8) return DVDQ_ERR_UNSUPPORTED;
     // block-wise scales: one per token and per 1024-channel block (the unit a warp of the transform
     // and eight k-blocks of the GEMM work on); other block sizes are not built
     if (q->scale_group != 0 && q->scale_group != kScaleBlock) return DVDQ_ERR_UNSUPPORTED;
@@ -69,7 +71,7 @@ static WorkspacePlan workspace_plan(int64_t M, int64_t K, const dvdq_act_quant& 
     WorkspacePlan p;
     const int64_t per_token = scales_per_token(K, q);
     p.codes_off = 0;
-    p.scales_off = align_up(M * act_row_bytes(K, q.bits), 256);
+    p.scales_off = align_up(M * act_row_bytes(K, storage_bits(q)), 256);
     p.sums_off = p.scales_off + align_up(M * per_token * 4, 256);
     p.total = p.sums_off + align_up(M * per_token * 4, 256);
     return p;
@@ -104,6 +106,11 @@ int32_t dvdq_version(void) { return kLibVersion; }
 size_t dvdq_act_codes_bytes(int64_t M, int64_t K, int32_t bits) {
     if (M < 0 || validate_k(K) != DVDQ_OK || (bits != 4 && bits != 6 && bits != 8)) return 0;
     return (size_t)(M * act_row_bytes(K, bits));
+}
+
+size_t dvdq_act_codes_bytes_q(int64_t M, int64_t K, const dvdq_act_quant* q) {
+    if (M < 0 || validate_k(K) != DVDQ_OK || validate_act_quant(q, K) != DVDQ_OK) return 0;
+    return (size_t)(M * act_row_bytes(K, storage_bits(*q)));
 }
 
 size_t dvdq_act_scales_count(int64_t M, int64_t K, const dvdq_act_quant* q) {
@@ -255,8 +262,9 @@ dvdq_status dvdq_pack_act_codes(const int8_t* codes_nat, int64_t M, int64_t K, c
     if ((s = check_device_arch()) != DVDQ_OK) return s;
     cudaStream_t st = (cudaStream_t)stream;
     const unsigned g = grid_for(M * (K / 16), 256);
-    if (q->bits == 4) pack_act_codes_kernel<4><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
-    else if (q->bits == 6) pack_act_codes_kernel<6><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
+    const int sb = storage_bits(*q);
+    if (sb == 4) pack_act_codes_kernel<4><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
+    else if (sb == 6) pack_act_codes_kernel<6><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
     else pack_act_codes_kernel<8><<<g, 256, 0, st>>>(codes_nat, M, K, static_cast<uint8_t*>(codes_out));
     const int64_t block = q->scale_group ? q->scale_group : K;
     code_sums_kernel<<<(unsigned)((M * (K / block) * 32 + 255) / 256), 256, 0, st>>>(codes_nat, M, K, block, code_sums_out);
@@ -273,8 +281,9 @@ dvdq_status dvdq_unpack_act_codes(const void* codes, int64_t M, int64_t K, const
     if (!aligned(codes, 16)) return DVDQ_ERR_ALIGN;
     if ((s = check_device_arch()) != DVDQ_OK) return s;
     const unsigned g = grid_for(M * (K / 16), 256);
-    if (q->bits == 4) unpack_act_codes_kernel<4><<<g, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint8_t*>(codes), M, K, codes_nat);
-    else if (q->bits == 6) unpack_act_codes_kernel<6><<<g, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint8_t*>(codes), M, K, codes_nat);
+    const int sb = storage_bits(*q);
+    if (sb == 4) unpack_act_codes_kernel<4><<<g, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint8_t*>(codes), M, K, codes_nat);
+    else if (sb == 6) unpack_act_codes_kernel<6><<<g, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint8_t*>(codes), M, K, codes_nat);
     else unpack_act_codes_kernel<8><<<g, 256, 0, (cudaStream_t)stream>>>(static_cast<const uint8_t*>(codes), M, K, codes_nat);
     return cuda_status(cudaGetLastError());
 }

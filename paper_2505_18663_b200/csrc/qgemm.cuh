@@ -702,6 +702,12 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
     return cuda_status(cudaGetLastError());
 }
 
+// qgemm_ss.cuh: activation codes stored one int8 per code
+template <bool RAW>
+static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+                                   const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
+                                   int32_t* acc_out, int64_t ldacc, cudaStream_t st);
+
 inline dvdq_status launch_qgemm(const void* codes, const float* scales, const int32_t* sums, int64_t M,
                                 const dvdq_act_quant& q, const dvdq_weights& w, const void* bias, int act,
                                 void* Y, int64_t ldy, int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
@@ -710,8 +716,12 @@ inline dvdq_status launch_qgemm(const void* codes, const float* scales, const in
     // adds up the code sums of a token's blocks itself.
     const bool raw = acc_out != nullptr;
     const int spr = q.scale_group != 0 ? (int)(w.K / q.scale_group) : 1;  // code sums (and scales) per token
+    const int sb = storage_bits(q);
+    if (sb == 8 && (raw || q.scale_group == 0))
+        return raw ? launch_qgemm_ss<true>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
+                   : launch_qgemm_ss<false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
 #define DVDQ_GEMM_CASE(B)                                                                                          \
-    if (q.bits == B) {                                                                                             \
+    if (sb == B) {                                                                                                 \
         if (raw) return launch_qgemm_t<B, true, false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st); \
         if (q.scale_group != 0)                                                                                    \
             return launch_qgemm_t<B, false, true>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);      \

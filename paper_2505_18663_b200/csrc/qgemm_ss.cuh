@@ -1,0 +1,459 @@
+// The GEMM for activation codes that are stored one int8 per code (8-bit activations, or 4- and
+// 6-bit codes kept in byte containers): the same contraction and epilogue as qgemm.cuh,
+//
+//   acc_in = sum_k c_ik (u_nk - z_n),   y_in = bf16(acc_in * s_i * Delta_n + bias_n),
+//
+// but the activation operand needs no widening, so TMA puts it into shared memory in the layout
+// the tensor core reads (K-major rows of 128 bytes, 128-byte swizzle) and no warp ever touches
+// it.  With no activation stages in tensor memory both accumulators can be 256 columns wide:
+// a CTA pair owns a tile of 256 tokens x 256 channels, tcgen05.mma.cta_group::2.kind::i8
+// 256x256x32 with both operands from shared memory.  Only the 4-bit weights are still widened
+// by warps (each CTA its 128 of the 256 rows), as in qgemm.cuh.
+//
+// Roles per CTA (16 warps):
+//   warp 0      TMA producer of the activation operand: this CTA's 128 token rows of a k-block
+//               straight into a ring of operand stages, deep enough to cover the copy's latency.
+//   warp 15     TMA producer of packed weight rows, into a ring for the widening warps.
+//   warp 1      (leader CTA) issues the MMAs; tcgen05.commit frees the stage in both CTAs.
+//   warps 2-5   epilogue (tcgen05.ld, zero-point term, scales, bias, GELU, bf16, TMA stores).
+//   warps 6-13  widen weight codes into the operand stage (two groups, alternate k-blocks).
+//   warp 14     tells the leader that this CTA's activation rows of a stage have landed (a TMA
+//               copy completes on a barrier of its own CTA).
+// Every wait is bounded, as in qgemm.cuh.
+#pragma once
+
+#include "qgemm.cuh"
+
+namespace dvdq {
+
+constexpr int kSsBN = 256, kSsBNh = kSsBN / 2;
+constexpr int kSsAStages = 6;        // activation tiles of one k-block (filled by TMA: its latency sets the depth)
+constexpr int kSsStages = 4;         // widened weight half-tiles of one k-block (filled by warps)
+constexpr int kSsWPackedStages = 4;  // ring of packed weight half-tiles
+constexpr int kSsFirstWWarp = 6, kSsWWarps = 8, kSsFwdWarp = kSsFirstWWarp + kSsWWarps, kSsWProducerWarp = kSsFwdWarp + 1;
+constexpr int kSsThreads = (kSsWProducerWarp + 1) * 32;
+static_assert(kSsStages % 2 == 0, "the MMA warp takes the weight stages in pairs");
+
+struct SsSmem {
+    static constexpr int kA = kBM * kBK;              // activation tile of one k-block (int8, swizzled)
+    static constexpr int kW = kSsBNh * kBK;           // widened weight half-tile
+    static constexpr int kWPacked = kSsBNh * kBK / 2; // packed weight half-tile (64-byte rows)
+    static constexpr int kAOff = 0;
+    static constexpr int kWOff = kAOff + kSsAStages * kA;
+    static constexpr int kWPackedOff = kWOff + kSsStages * kW;
+    static constexpr int kStageOutOff = kWPackedOff + kSsWPackedStages * kWPacked;  // 1024-byte aligned
+    static constexpr int kStageOutPerWarp = 32 * 128;  // one buffer of 32 rows x 64 bf16: the operand rings get the rest
+    static constexpr int kConstOff = kStageOutOff + kEpilogueWarps * kStageOutPerWarp;
+    static constexpr int kConstPerWarp = 3 * kSsBN * 4;
+    static constexpr int kBarOff = kConstOff + kEpilogueWarps * kConstPerWarp;
+    static constexpr int kNumBars = 3 * kSsAStages + 2 * kSsStages + 5 + 2 * kSsWPackedStages;
+    static constexpr int kMiscOff = kBarOff + kNumBars * 8;
+    static constexpr int kTotal = kMiscOff + 16 + 1024;
+    static_assert(kStageOutOff % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+    static_assert(kTotal <= 232448, "more than the 227 KB of shared memory a CTA can have");
+};
+
+// D[tmem] (+)= A[smem] * B[smem]^T for a CTA pair, int8 operands, int32 accumulators: each CTA
+// holds its 128 rows of A and half of B's rows at the same shared-memory offsets.
+__device__ __forceinline__ void tc_mma_i8_ss_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+template <bool RAW>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSsThreads, 1)
+qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                const __grid_constant__ CUtensorMap tmY, const float* __restrict__ scales,
+                const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
+                const __nv_bfloat16* __restrict__ bias, int32_t* __restrict__ acc_out, int64_t ldacc,
+                int M, int N, int K, int act, int spr) {
+    using S = SsSmem;
+    constexpr int BN = kSsBN, BNh = kSsBNh;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int num_n = (N + BN - 1) / BN, num_m = (M + 2 * kBM - 1) / (2 * kBM);
+    const int num_tiles = num_m * num_n;
+    const int KB = 2 * ((K + 2 * kBK - 1) / (2 * kBK));  // even; a k-block past K reads zeros
+
+    const uint32_t bar0 = sbase + S::kBarOff;
+    auto a_full = [&](int s) { return bar0 + 8u * s; };                          // this CTA's TMA copy of the stage
+    auto a_ready = [&](int s) { return bar0 + 8u * (kSsAStages + s); };          // leader's copy: both CTAs' copies landed
+    auto a_empty = [&](int s) { return bar0 + 8u * (2 * kSsAStages + s); };      // one per CTA
+    const uint32_t barw = bar0 + 8u * (3 * kSsAStages);
+    auto ops_full = [&](int s) { return barw + 8u * s; };                        // widened weights; leader's copy is used
+    auto ops_empty = [&](int s) { return barw + 8u * (kSsStages + s); };         // one per CTA
+    auto acc_full = [&](int s) { return barw + 8u * (2 * kSsStages + s); };      // one per CTA
+    auto acc_empty = [&](int s) { return barw + 8u * (2 * kSsStages + 2 + s); }; // leader's copy
+    const uint32_t drain_bar = barw + 8u * (2 * kSsStages + 4);
+    auto wp_full = [&](int s) { return drain_bar + 8u * (1 + s); };
+    auto wp_empty = [&](int s) { return drain_bar + 8u * (1 + kSsWPackedStages + s); };
+    volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + S::kMiscOff);  // [0] tmem base, [1] abort
+    volatile uint32_t* abort_flag = misc + 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kSsAStages; ++s) { mbar_init(a_full(s), 1); mbar_init(a_ready(s), 2); mbar_init(a_empty(s), 1); }
+        for (int s = 0; s < kSsStages; ++s) { mbar_init(ops_full(s), 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * kEpilogueWarps); }
+        mbar_init(drain_bar, 1);
+        for (int s = 0; s < kSsWPackedStages; ++s) { mbar_init(wp_full(s), 1); mbar_init(wp_empty(s), kSsWWarps / kUnpackGroups); }
+        misc[1] = 0u;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(sbase + S::kMiscOff, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = misc[0];
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer, activation rows
+        if (lane == 0) {
+            tma_prefetch_desc(&tmA);
+            uint32_t st = 0, ph = 0, issued = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
+                for (int kb = 0; ok && kb < KB; ++kb) {
+                    if (!mbar_wait(a_empty(st), ph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                    mbar_arrive_expect_tx(a_full(st), S::kA);
+                    tma_load_2d(sbase + S::kAOff + st * S::kA, &tmA, a_full(st), kb * kBK, m0);
+                    ++issued;
+                    if (++st == kSsAStages) { st = 0; ph ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // Giving up: let copies already in flight land before the CTA exits (bounded).
+                const uint32_t n_out = issued < (uint32_t)kSsAStages ? issued : (uint32_t)kSsAStages;
+                for (uint32_t i = 0; i < n_out; ++i) {
+                    const uint32_t s = (st + kSsAStages - 1 - i) % kSsAStages;
+                    const uint32_t p = (s < st) ? ph : (ph ^ 1u);
+                    for (int it = 0; it < (1 << 16) && !mbar_try_wait(a_full(s), p); ++it) {}
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == kSsWProducerWarp) {
+        // ------------------------------------------------------------ TMA producer, packed weight rows
+        if (lane == 0) {
+            tma_prefetch_desc(&tmW);
+            uint32_t wst = 0, wph = 0, wissued = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                const int n0 = (tile % num_n) * BN + (int)rank * BNh;
+                for (int kb = 0; ok && kb < KB; ++kb) {
+                    if (!mbar_wait(wp_empty(wst), wph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
+                    mbar_arrive_expect_tx(wp_full(wst), S::kWPacked);
+                    tma_load_2d(sbase + S::kWPackedOff + wst * S::kWPacked, &tmW, wp_full(wst), kb * (kBK / 2), n0);
+                    ++wissued;
+                    if (++wst == kSsWPackedStages) { wst = 0; wph ^= 1u; }
+                }
+            }
+            if (!ok) {
+                const uint32_t w_out = wissued < (uint32_t)kSsWPackedStages ? wissued : (uint32_t)kSsWPackedStages;
+                for (uint32_t i = 0; i < w_out; ++i) {
+                    const uint32_t s = (wst + kSsWPackedStages - 1 - i) % kSsWPackedStages;
+                    const uint32_t p = (s < wst) ? wph : (wph ^ 1u);
+                    for (int it = 0; it < (1 << 16) && !mbar_try_wait(wp_full(s), p); ++it) {}
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (rank == 0) {
+            constexpr uint32_t idesc = umma_idesc_s8s8s32(2 * kBM, BN);
+            uint32_t st = 0, ph = 0, sa = 0, pa = 0, lt = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++lt) {
+                const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
+                if (!mbar_wait_warp(acc_empty(a), aph ^ 1u, abort_flag, kWaitAccEmpty)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + a * BN;
+                for (int kb = 0; kb < KB; kb += 2) {
+                    // the activation ring may have an odd number of stages: its second stage of the trip can wrap
+                    const uint32_t sa1 = sa + 1 == kSsAStages ? 0u : sa + 1, pa1 = sa + 1 == kSsAStages ? pa ^ 1u : pa;
+                    if (!mbar_wait_warp(a_ready(sa), pa, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                    if (!mbar_wait_warp(ops_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
+                    if (!mbar_wait_warp(a_ready(sa1), pa1, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                    if (!mbar_wait_warp(ops_full(st + 1), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
+                    tc_fence_after();
+                    if (elect_one()) {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint64_t adesc = umma_desc_sw128_kmajor(sbase + S::kAOff + (h ? sa1 : sa) * S::kA);
+                            const uint64_t bdesc = umma_desc_sw128_kmajor(sbase + S::kWOff + (st + h) * S::kW);
+#pragma unroll
+                            for (int k = 0; k < kBK / 32; ++k)  // +32 int8 along K = +2 in the 16-byte address field
+                                tc_mma_i8_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | h | k) != 0 ? 1u : 0u);
+                            tc_commit_pair(ops_empty(st + h), 3);
+                            tc_commit_pair(a_empty(h ? sa1 : sa), 3);
+                        }
+                    }
+                    __syncwarp();
+                    st += 2;
+                    if (st == kSsStages) { st = 0; ph ^= 1u; }
+                    sa = sa1 + 1;
+                    pa = pa1;
+                    if (sa == kSsAStages) { sa = 0; pa ^= 1u; }
+                }
+                if (ok && elect_one()) tc_commit_pair(acc_full(a), 3);
+                __syncwarp();
+            }
+            if (elect_one()) tc_commit_pair(drain_bar, 1);
+            __syncwarp();
+            mbar_wait(drain_bar, 0u, abort_flag, kWaitDrain);
+        }
+        __syncwarp();
+    } else if (warp < kSsFirstWWarp) {
+        // ------------------------------------------------------------ epilogue
+        const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+        const int ew = warp - kFirstEpilogueWarp;
+        const uint32_t c_delta = sbase + S::kConstOff + ew * S::kConstPerWarp;  // shared addresses of float[BN] each
+        const uint32_t c_zc = c_delta + BN * 4;    // (z_n - 8) as a float: exact, |.| <= 8
+        const uint32_t c_bias = c_zc + BN * 4;
+        const uint32_t stg0 = sbase + S::kStageOutOff + ew * S::kStageOutPerWarp;
+        constexpr int kShift = 4;  // the widened weights are 16 x (u - 8)
+        if (!RAW && lane == 0) tma_prefetch_desc(&tmY);
+        uint32_t lt = 0, nstore = 0;
+        for (int tile = pair; tile < num_tiles; tile += num_pairs, ++lt) {
+            const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
+            const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM, n0 = (tile % num_n) * BN;
+            __syncwarp();
+            {   // per-channel constants of this tile: all loads in flight at once, then the stores
+                float cd[BN / 32], cz[BN / 32], cb[BN / 32];
+#pragma unroll
+                for (int i = 0; i < BN / 32; ++i) {
+                    const int n = n0 + lane + 32 * i;
+                    const bool okn = n < N;
+                    cd[i] = okn ? __ldg(delta + n) : 0.f;
+                    cz[i] = okn ? (float)__ldg(zc + n) : 0.f;
+                    cb[i] = (okn && bias != nullptr) ? __bfloat162float(bias[n]) : 0.f;
+                }
+#pragma unroll
+                for (int i = 0; i < BN / 32; ++i) {
+                    const int c = lane + 32 * i;
+                    sts32f(c_delta + 4 * c, cd[i]);
+                    sts32f(c_zc + 4 * c, cz[i]);
+                    sts32f(c_bias + 4 * c, cb[i]);
+                }
+            }
+            __syncwarp();
+            if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) break;
+            tc_fence_after();
+            const int row = m0 + q * 32 + lane;
+            const bool row_ok = row < M;
+            const float s_i = (!RAW && row_ok) ? scales[row] : 0.f;
+            int32_t S_i = row_ok ? sums[(int64_t)row * spr] : 0;
+            if (RAW && row_ok)
+                for (int g = 1; g < spr; ++g) S_i += sums[(int64_t)row * spr + g];  // spr == 1 unless the scales are block-wise
+            const float S_f = (float)S_i;  // |sum of codes| <= K * 32 < 2^24: exact
+            const float s_k = s_i * (1.0f / (float)(1 << kShift)), nS_k = -S_f * (float)(1 << kShift);
+            const uint64_t s2 = f2_pack(s_k, s_k), negS2 = f2_pack(nS_k, nS_k);
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + a * BN + c * 32 + ((uint32_t)(q * 32) << 16), r);
+                tmem_ld_wait();
+                const int nb = n0 + c * 32;
+                if (RAW) {
+                    int32_t* dst = acc_out + (int64_t)row * ldacc + nb;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 zq = lds128f(c_zc + 4 * (c * 32 + j));
+                        int4 o;
+                        o.x = ((int32_t)r[j] >> kShift) - __float2int_rn(zq.x) * S_i;
+                        o.y = ((int32_t)r[j + 1] >> kShift) - __float2int_rn(zq.y) * S_i;
+                        o.z = ((int32_t)r[j + 2] >> kShift) - __float2int_rn(zq.z) * S_i;
+                        o.w = ((int32_t)r[j + 3] >> kShift) - __float2int_rn(zq.w) * S_i;
+                        if (row_ok && nb + j < N) *reinterpret_cast<int4*>(dst + j) = o;
+                    }
+                } else {
+                    // Two chunks of 32 columns fill one staging buffer of 32 rows x 128 bytes, which
+                    // leaves as ONE TMA store (128-byte rows are what TMA moves at full rate).  The
+                    // buffer used two stores ago must have been read by its store.
+                    if ((c & 1) == 0) {
+                        if (lane == 0) tma_store_wait_read<0>();
+                        __syncwarp();
+                    }
+                    const uint32_t buf = stg0;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        const float4 d0 = lds128f(c_delta + 4 * (c * 32 + j)), d1 = lds128f(c_delta + 4 * (c * 32 + j + 4));
+                        const float4 z0 = lds128f(c_zc + 4 * (c * 32 + j)), z1 = lds128f(c_zc + 4 * (c * 32 + j + 4));
+                        const float4 b0 = lds128f(c_bias + 4 * (c * 32 + j)), b1 = lds128f(c_bias + 4 * (c * 32 + j + 4));
+                        const float dl[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+                        const float zz[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
+                        const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                        float v[8];
+                        // The raw accumulator is (256 or 64) x the true one: at most 22 significant
+                        // bits, so its conversion is exact and the factor moves into the per-row
+                        // constants: y = (raw - zz * S * 2^k) * (s * 2^-k * delta) + bias, on fp32 pairs.
+#pragma unroll
+                        for (int t = 0; t < 8; t += 2) {
+                            const uint64_t raw2 = f2_pack((float)(int32_t)r[j + t], (float)(int32_t)r[j + t + 1]);
+                            const uint64_t acc2 = f2_fma(f2_pack(zz[t], zz[t + 1]), negS2, raw2);   // exact
+                            const uint64_t y2 = f2_fma(acc2, f2_mul(f2_pack(dl[t], dl[t + 1]), s2), f2_pack(bb[t], bb[t + 1]));
+                            f2_unpack(y2, v[t], v[t + 1]);
+                        }
+                        if (act == 1) {
+#pragma unroll
+                            for (int t = 0; t < 8; ++t) v[t] = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(v[t])));
+                        }
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * t], v[2 * t + 1]);
+                            pk[t] = *reinterpret_cast<uint32_t*>(&b2);
+                        }
+                        // 128-byte rows, 16-byte chunk index XORed with row % 8: the layout a
+                        // 128B-swizzled TMA store reads, and conflict-free for this per-row write.
+                        const int ch = (4 * (c & 1) + (j >> 3)) ^ (lane & 7);
+                        sts128(buf + lane * 128 + ch * 16, pk[0], pk[1], pk[2], pk[3]);
+                    }
+                    if (c & 1) {
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0 && nb - 32 < N && m0 + q * 32 < M) {
+                            tma_store_2d(&tmY, buf, nb - 32, m0 + q * 32);
+                            tma_store_commit();
+                        }
+                        ++nstore;
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty(a), 0));
+        }
+        if (!RAW && lane == 0) tma_store_wait_all();
+        __syncwarp();
+
+    } else if (warp < kSsFwdWarp) {
+        // ------------------------------------------------------------ widen weight codes -> shared memory
+        const uint32_t grp = (uint32_t)(warp - kSsFirstWWarp) >> 2;
+        const int u = (threadIdx.x - kSsFirstWWarp * 32) & 127;  // thread of its group of four warps
+        uint32_t j = 0;
+        bool ok = true;
+        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+            for (int kb = 0; kb < KB; ++kb) {
+            const uint32_t jj = j++;
+            if (jj % kUnpackGroups != grp) continue;
+            const uint32_t pst = jj % kSsWPackedStages, pph = (jj / kSsWPackedStages) & 1u;
+            const uint32_t wst = jj % kSsStages, wph = (jj / kSsStages) & 1u;
+            if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+            const uint32_t pw = sbase + S::kWPackedOff + pst * S::kWPacked;
+            const uint32_t wdW = sbase + S::kWOff + wst * S::kW;
+            // BNh rows x 4 chunks of 32 nibbles, stored as (u - 8); widened in registers before the
+            // wide stage is known to be free
+            constexpr int kPieces = (BNh * 4) / 128;
+            uint32_t e[kPieces][4], o[kPieces][4];
+#pragma unroll
+            for (int it = 0; it < kPieces; ++it) {
+                const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                const uint4 p = lds128(pw + row * (kBK / 2) + ck * 16);
+                const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+#pragma unroll
+                for (int jw = 0; jw < 4; ++jw) { e[it][jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[it][jw] = w[jw] & 0xF0F0F0F0u; }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(wp_empty(pst));  // the packed rows are in registers
+            if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int it = 0; it < kPieces; ++it) {
+                const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                const uint32_t drow = wdW + (row >> 3) * 1024 + (row & 7) * 128;
+                sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[it][0], o[it][0], e[it][1], o[it][1]);
+                sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[it][2], o[it][2], e[it][3], o[it][3]);
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(wst), 0));
+            }
+        }
+    } else if (warp == kSsFwdWarp) {
+        // ------------------------------------------------------------ "activation rows landed" -> leader
+        uint32_t st = 0, ph = 0;
+        bool ok = true;
+        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!mbar_wait_warp(a_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(st), 0));
+                __syncwarp();
+                if (++st == kSsAStages) { st = 0; ph ^= 1u; }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the peer may read this CTA's shared and tensor memory until it is done too
+    tc_fence_after();
+    if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ------------------------------------------------------------------ host side
+
+template <bool RAW>
+static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+                                   const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
+                                   int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
+    using S = SsSmem;
+    const int64_t K = w.K, N = w.N;
+    const BlobLayout L = blob_layout(N, K);
+    const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
+    CUtensorMap tmA, tmW, tmY;
+    if (!make_byte_map(&tmA, codes, (uint64_t)K, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B))
+        return DVDQ_ERR_CUDA;
+    if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, kSsBNh,
+                       CU_TENSOR_MAP_SWIZZLE_NONE))
+        return DVDQ_ERR_CUDA;
+    if (RAW) {
+        tmY = tmA;  // unused
+    } else if (!make_out_map(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)) {
+        return DVDQ_ERR_CUDA;
+    }
+    auto kern = qgemm_ss_kernel<RAW>;
+    static int max_pairs = 0;
+    if (max_pairs == 0) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) return DVDQ_ERR_CUDA;
+        int dev = 0, sm_count = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return DVDQ_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DVDQ_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(sm_count & ~1), 1, 1);
+        cfg.blockDim = dim3(kSsThreads, 1, 1);
+        cfg.dynamicSmemBytes = S::kTotal;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) != cudaSuccess || clusters < 1) return DVDQ_ERR_CUDA;
+        max_pairs = clusters < sm_count / 2 ? clusters : sm_count / 2;
+    }
+    const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + kSsBN - 1) / kSsBN);
+    const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
+    kern<<<2 * pairs, kSsThreads, S::kTotal, st>>>(tmA, tmW, tmY, scales, sums,
+                                                   reinterpret_cast<const float*>(blob + L.delta_offset),
+                                                   reinterpret_cast<const int32_t*>(blob + L.zc_offset),
+                                                   static_cast<const __nv_bfloat16*>(bias), acc_out, ldacc, (int)M, (int)N, (int)K,
+                                                   act, spr);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace dvdq

@@ -62,12 +62,13 @@ template <int LOG2B, int BITS, bool FULL>
 __global__ void __maxnreg__(80)  // two CTAs of 12 warps per SM
 rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
           uint8_t* __restrict__ codes, float* __restrict__ scales, int32_t* __restrict__ sums,
-          int spans, int tokens_per_cta, int num_groups, int blockwise) {
+          int spans, int tokens_per_cta, int num_groups, int blockwise, int code_bits) {
     extern __shared__ float4 s_turn[];  // 256 float4 per warp
     __shared__ unsigned s_max[3][kRqMaxWarps];  // [slot set][token of the CTA]: bits of the token absmax
     __shared__ int s_sum[3][kRqMaxWarps];       // sum of the token's codes
     constexpr bool kRot = LOG2B > 0;
-    constexpr float qmax = (float)((1 << (BITS - 1)) - 1);
+    // BITS is the width a code is STORED in; the quantizer's own width may be smaller (codes kept in bytes)
+    const float qmax = (float)((1 << (code_bits - 1)) - 1);
     constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: ulp 1, so the fma rounds to an integer
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int tl = warp / spans, sp = warp - tl * spans;
@@ -361,7 +362,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
 
 template <int LOG2B, int BITS, bool FULL>
 static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t ldx, void* codes, float* scales,
-                                    int32_t* sums, int blockwise, cudaStream_t st) {
+                                    int32_t* sums, int blockwise, int code_bits, cudaStream_t st) {
     const int spans = (int)((K + kRqSpan - 1) / kRqSpan);
     if (spans > kRqMaxWarps) return DVDQ_ERR_SHAPE;
     int tpc = 12 / spans;  // at most 12 tokens per CTA: named barriers 1..12
@@ -392,20 +393,20 @@ static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t
     const int64_t resident = (int64_t)sm_count * blocks_per_sm[warps];
     const unsigned grid = (unsigned)(groups < resident ? groups : resident);
     kern<<<grid, threads, smem, st>>>((const __nv_bfloat16*)X, (int)M, (int)K, (int)ldx, (uint8_t*)codes, scales, sums, spans, tpc,
-                                      (int)groups, blockwise);
+                                      (int)groups, blockwise, code_bits);
     return cuda_status(cudaGetLastError());
 }
 
 template <int BITS>
 static dvdq_status launch_rq_bits(const void* X, int64_t M, int64_t K, int64_t ldx, int rot_block, void* codes,
-                                  float* scales, int32_t* sums, int blockwise, cudaStream_t st) {
+                                  float* scales, int32_t* sums, int blockwise, int code_bits, cudaStream_t st) {
     int log2b = 0;
     while ((1 << log2b) < rot_block) ++log2b;
     const bool full = K % kRqSpan == 0;
 #define DVDQ_RQ_CASE(L)                                                                              \
     case L:                                                                                          \
-        return full ? launch_rq_kernel<L, BITS, true>(X, M, K, ldx, codes, scales, sums, blockwise, st)         \
-                    : launch_rq_kernel<L, BITS, false>(X, M, K, ldx, codes, scales, sums, blockwise, st);
+        return full ? launch_rq_kernel<L, BITS, true>(X, M, K, ldx, codes, scales, sums, blockwise, code_bits, st)         \
+                    : launch_rq_kernel<L, BITS, false>(X, M, K, ldx, codes, scales, sums, blockwise, code_bits, st);
     switch (log2b) {
         DVDQ_RQ_CASE(0)
         DVDQ_RQ_CASE(6)
@@ -422,9 +423,10 @@ static dvdq_status launch_rq_bits(const void* X, int64_t M, int64_t K, int64_t l
 inline dvdq_status launch_rotate_quantize(const void* X, int64_t M, int64_t K, int64_t ldx, const dvdq_act_quant& q,
                                           void* codes, float* scales, int32_t* sums, cudaStream_t st) {
     if (M == 0) return DVDQ_OK;
-    if (q.bits == 4) return launch_rq_bits<4>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, st);
-    if (q.bits == 6) return launch_rq_bits<6>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, st);
-    return launch_rq_bits<8>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, st);
+    const int sb = storage_bits(q);
+    if (sb == 4) return launch_rq_bits<4>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, q.bits, st);
+    if (sb == 6) return launch_rq_bits<6>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, q.bits, st);
+    return launch_rq_bits<8>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, q.bits, st);
 }
 
 }  // namespace dvdq

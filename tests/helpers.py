@@ -18,15 +18,15 @@ def bf16_values(bits: np.ndarray) -> np.ndarray:
     return from_bits(bits).to(torch.float64).numpy()
 
 
-def act_quant(bits: int, rot_block: int) -> B.ActQuant:
-    return B.ActQuant(bits, rot_block, 0)
+def act_quant(bits: int, rot_block: int, container: int = 0) -> B.ActQuant:
+    return B.ActQuant(bits, rot_block, 0, container)
 
 
-def gpu_rotate_quantize(x_dev: torch.Tensor, bits: int, rot_block: int):
+def gpu_rotate_quantize(x_dev: torch.Tensor, bits: int, rot_block: int, container: int = 0):
     """Runs the CUDA transform; returns (packed codes, scales, sums, natural-order int8 codes)."""
     M, K = x_dev.shape
-    q = act_quant(bits, rot_block)
-    codes = torch.empty(max(1, B.dvdq_act_codes_bytes(M, K, bits)), dtype=torch.uint8, device=x_dev.device)
+    q = act_quant(bits, rot_block, container)
+    codes = torch.empty(max(1, B.dvdq_act_codes_bytes_q(M, K, q)), dtype=torch.uint8, device=x_dev.device)
     scales = torch.empty(max(1, M), dtype=torch.float32, device=x_dev.device)
     sums = torch.empty(max(1, M), dtype=torch.int32, device=x_dev.device)
     B.dvdq_rotate_quantize(x_dev, q, codes, scales, sums)
@@ -44,11 +44,11 @@ def gpu_pack_weights(u: np.ndarray, delta: np.ndarray, z: np.ndarray, rot_block:
     return w, blob
 
 
-def gpu_pack_codes(codes_np: np.ndarray, bits: int, rot_block: int, device="cuda"):
+def gpu_pack_codes(codes_np: np.ndarray, bits: int, rot_block: int, device="cuda", container: int = 0):
     M, K = codes_np.shape
-    q = act_quant(bits, rot_block)
+    q = act_quant(bits, rot_block, container)
     nat = torch.from_numpy(codes_np.astype(np.int8)).to(device)
-    packed = torch.empty(B.dvdq_act_codes_bytes(M, K, bits), dtype=torch.uint8, device=device)
+    packed = torch.empty(B.dvdq_act_codes_bytes_q(M, K, q), dtype=torch.uint8, device=device)
     sums = torch.empty(M, dtype=torch.int32, device=device)
     B.dvdq_pack_act_codes(nat, q, packed, sums)
     return packed, sums
