@@ -286,6 +286,11 @@ def run_cuda(args, wl):
                        "rq_ms": rq_ms[li], "rq_gbs": rq_bytes(M, layer, args.scale_group, args.container) / (rq_ms[li] * 1e-3) / 1e9,
                        "qgemm_ms": gm_ms[li], "qgemm_tops": layer_ops(M, layer) / (gm_ms[li] * 1e-3) / 1e12})
 
+    # ---- the same step with the codes packed b bits each (container 0), for the record: fewer steps
+    packed = None
+    if args.container != 0 and not args.no_packed and world == 1:
+        packed = run_packed_leg(args, wl, layers, xs, dev, B, M)
+
     # ---- end to end through dvdq_qlinear with HOST buffers (pinned), copies inside the timed region
     e2e = None
     if not args.no_e2e:
@@ -297,12 +302,12 @@ def run_cuda(args, wl):
         return
 
     # the ncu counters were taken on the default workload (hunyuan, its own bit widths, per-token scales)
-    captured = wl.name == "hunyuan" and wl.M == 65536 and args.bits == 0 and args.scale_group == 0 and args.container == 0
+    captured = wl.name == "hunyuan" and wl.M == 65536 and args.bits == 0 and args.scale_group == 0 and args.container == 8
     line = {
         "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "i8", "data": "synthetic", "config": config_of(wl, args),
-        "roofline": {"kernel": "qgemm_kernel (tcgen05.mma kind::i8)", "bound": "tensor", "achieved": gemm_tops,
+        "roofline": {"kernel": ("qgemm_ss_kernel" if args.container == 8 and args.scale_group == 0 else "qgemm_kernel") + " (tcgen05.mma kind::i8)", "bound": "tensor", "achieved": gemm_tops,
                      "peak": int8_peak, "unit": "TOPS", "frac": gemm_tops / int8_peak,
                      "peak_source": f"{peaks['source']}: bf16_tflops_sustained x {INT8_OVER_BF16} (nominal int8:bf16)",
                      "frac_of_nominal_4500": gemm_tops / NOMINAL_INT8_TOPS,
@@ -312,6 +317,7 @@ def run_cuda(args, wl):
                                      "peak_source": peaks["source"], "frac_of_nominal_8000": rq_gbs / 8000.0,
                                      "avg_launch_ms": sum(rq_ms) / len(rq_ms), "traffic": RQ_DRAM_TRAFFIC_PER_LAUNCH if captured else None},
         "stages": stages,
+        "packed_codes": packed,
         "e2e": e2e,
         "gpu_launches": 2 * len(layers) * args.steps,
         "clocks": clocks,
@@ -327,8 +333,49 @@ def run_cuda(args, wl):
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/; None
 # until a capture of the corresponding kernel exists.
-QGEMM_DRAM_TRAFFIC_PER_LAUNCH = 0.97e9   # bytes: 16384-token capture x 4 (traffic grows with M), mean of the 4 layers
-RQ_DRAM_TRAFFIC_PER_LAUNCH = 0.82e9
+QGEMM_DRAM_TRAFFIC_PER_LAUNCH = 1.15e9   # bytes: 16384-token capture x 4 (traffic grows with M), mean of the 4 layers
+RQ_DRAM_TRAFFIC_PER_LAUNCH = 0.94e9
+
+
+def run_packed_leg(args, wl, layers, xs, dev, B, M):
+    """The step with activation codes packed b bits each (the layout the GEMM widens in shared and
+    tensor memory), timed on max(5, steps / 5) steps after 3 warm-up steps.  Same inputs, same outputs."""
+    packed_layers = []
+    for L in layers:
+        layer = L["layer"]
+        q = B.ActQuant(layer.bits, layer.rot_block, args.scale_group, 0)
+        codes = torch.empty(B.dvdq_act_codes_bytes_q(M, layer.K, q), dtype=torch.uint8, device=dev)
+        packed_layers.append((layer, q, codes, L))
+    n_steps = max(5, args.steps // 5)
+    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in packed_layers] for _ in range(n_steps)]
+
+    def step(events=None):
+        for li, (layer, q, codes, L) in enumerate(packed_layers):
+            if events is not None:
+                events[li][0].record()
+            B.dvdq_rotate_quantize(xs[layer.K], q, codes, L["scales"], L["sums"])
+            if events is not None:
+                events[li][1].record()
+            B.dvdq_qgemm(codes, L["scales"], L["sums"], M, q, L["w"], L["bias"], layer.act, L["Y"])
+            if events is not None:
+                events[li][2].record()
+
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for s in range(n_steps):
+        step(ev[s])
+    t1.record()
+    torch.cuda.synchronize()
+    ms = t0.elapsed_time(t1) / n_steps
+    rq_ms = sum(ev[s][li][0].elapsed_time(ev[s][li][1]) for s in range(n_steps) for li in range(len(packed_layers))) / n_steps
+    gm_ms = sum(ev[s][li][1].elapsed_time(ev[s][li][2]) for s in range(n_steps) for li in range(len(packed_layers))) / n_steps
+    ops = sum(layer_ops(M, l) for l, _, _, _ in packed_layers)
+    nbytes = sum(rq_bytes(M, l, args.scale_group, 0) for l, _, _, _ in packed_layers)
+    return {"value": ops / (ms * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": ms, "steps": n_steps,
+            "qgemm_tops": ops / (gm_ms * 1e-3) / 1e12, "rq_gbs": nbytes / (rq_ms * 1e-3) / 1e9}
 
 
 def run_e2e(args, wl, layers, xs, dev, B, dist, world):
@@ -414,8 +461,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling runs)")
-    ap.add_argument("--container", type=int, default=0,
-                    help="0: activation codes packed (b bits each); 8: one int8 per code")
+    ap.add_argument("--container", type=int, default=8,
+                    help="8: one int8 per activation code (default, the faster GEMM); 0: codes packed b bits each")
+    ap.add_argument("--no-packed", action="store_true", help="skip the extra leg that times the packed layout")
     ap.add_argument("--scale-group", type=int, default=0,
                     help="0: one activation scale per token; 1024: one per token and block of 1024 channels")
     ap.add_argument("--bits", type=int, default=0, help="override the activation bit width of every layer (4, 6 or 8)")

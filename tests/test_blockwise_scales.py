@@ -162,6 +162,26 @@ def test_qlinear_blockwise_matches_oracle_end_to_end(M, N, K, Bk, bits, mode):
         assert torch.equal(Y, Y2)
 
 
+@pytest.mark.parametrize("bits", [4, 6])
+def test_blockwise_with_codes_kept_in_bytes_equals_packed(bits):
+    """container_bits = 8 changes where a code is stored, not the code, the block scales or the output."""
+    M, N, K, Bk = 200, 392, 2048, 256
+    x = synth_x(M, K, seed=21 + bits).to(DEV)
+    u, d, z = orc.prepare_weights(to_bits(synth_w(N, K, 22, "minmax")), Bk, "minmax")
+    w, blob = gpu_pack_weights(u, d, z, Bk)
+    ys = []
+    for container in (0, 8):
+        q = B.ActQuant(bits, Bk, G, container)
+        ws = torch.empty(B.dvdq_qlinear_workspace_bytes(M, K, q), dtype=torch.uint8, device=DEV)
+        Y = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
+        B.dvdq_qlinear(x, q, w, None, 0, Y, ws)
+        nat = torch.empty(M, K, dtype=torch.int8, device=DEV)
+        B.dvdq_unpack_act_codes(ws, M, K, q, nat)
+        assert_device_ok()
+        ys.append((Y, nat))
+    assert torch.equal(ys[0][1], ys[1][1]) and torch.equal(ys[0][0], ys[1][0])
+
+
 def test_blockwise_scales_lower_the_quantization_error():
     """What the option is for: with outlier channels confined to one block, the other blocks get a
     finer grid, so the layer output is closer to the unquantized product than with one scale per token."""
