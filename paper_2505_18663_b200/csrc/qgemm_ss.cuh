@@ -10,12 +10,17 @@
 // 256x256x32 with both operands from shared memory.  Only the 4-bit weights are still widened
 // by warps (each CTA its 128 of the 256 rows), as in qgemm.cuh.
 //
-// Roles per CTA (16 warps):
+// Roles per CTA (16 or 20 warps):
 //   warp 0      TMA producer of the activation operand: this CTA's 128 token rows of a k-block
 //               straight into a ring of operand stages, deep enough to cover the copy's latency.
 //   warp 15     TMA producer of packed weight rows, into a ring for the widening warps.
 //   warp 1      (leader CTA) issues the MMAs; tcgen05.commit frees the stage in both CTAs.
-//   warps 2-5   epilogue (tcgen05.ld, zero-point term, scales, bias, GELU, bf16, TMA stores).
+//   warps 2-5  epilogue (tcgen05.ld, zero-point term, scales, bias, GELU, bf16, TMA stores), one
+//               warp per tensor-memory lane quarter.
+//   warps 16-19 (EW = 8 only) a second epilogue warp per lane quarter; each then takes 128 of the
+//               256 columns.  With one warp per quarter the epilogue, not the MMA, sets the pace
+//               of layers with a short K or a GELU (+13..25 % there); where the mainloop sets it,
+//               the extra warps only compete with the widening warps (-2..7 %).  The host picks.
 //   warps 6-13  widen weight codes into the operand stage (two groups, alternate k-blocks).
 //   warp 14     tells the leader that this CTA's activation rows of a stage have landed (a TMA
 //               copy completes on a barrier of its own CTA).
@@ -31,7 +36,9 @@ constexpr int kSsAStages = 6;        // activation tiles of one k-block (filled 
 constexpr int kSsStages = 4;         // widened weight half-tiles of one k-block (filled by warps)
 constexpr int kSsWPackedStages = 4;  // ring of packed weight half-tiles
 constexpr int kSsFirstWWarp = 6, kSsWWarps = 8, kSsFwdWarp = kSsFirstWWarp + kSsWWarps, kSsWProducerWarp = kSsFwdWarp + 1;
-constexpr int kSsThreads = (kSsWProducerWarp + 1) * 32;
+constexpr int kSsFirstEpilogueWarp2 = kSsWProducerWarp + 1;  // a multiple of 4: warp w reads tensor-memory lanes 32 * (w % 4)..
+constexpr int kSsMaxEpilogueWarps = 8;
+static_assert(kSsFirstEpilogueWarp2 % 4 == 0, "lane quarters");
 static_assert(kSsStages % 2 == 0, "the MMA warp takes the weight stages in pairs");
 
 struct SsSmem {
@@ -42,10 +49,12 @@ struct SsSmem {
     static constexpr int kWOff = kAOff + kSsAStages * kA;
     static constexpr int kWPackedOff = kWOff + kSsStages * kW;
     static constexpr int kStageOutOff = kWPackedOff + kSsWPackedStages * kWPacked;  // 1024-byte aligned
-    static constexpr int kStageOutPerWarp = 32 * 128;  // one buffer of 32 rows x 64 bf16: the operand rings get the rest
-    static constexpr int kConstOff = kStageOutOff + kEpilogueWarps * kStageOutPerWarp;
-    static constexpr int kConstPerWarp = 3 * kSsBN * 4;
-    static constexpr int kBarOff = kConstOff + kEpilogueWarps * kConstPerWarp;
+    // 16 KB of staging and 12 KB of constants whether four or eight epilogue warps share them: one
+    // buffer of 32 rows x 64 (or 32) bf16 each, and delta / zero-point rest / bias of 256 (or 128) columns
+    static constexpr int kStageOutBytes = 4 * 32 * 128;
+    static constexpr int kConstOff = kStageOutOff + kStageOutBytes;
+    static constexpr int kConstBytes = 4 * 3 * kSsBN * 4;
+    static constexpr int kBarOff = kConstOff + kConstBytes;
     static constexpr int kNumBars = 3 * kSsAStages + 2 * kSsStages + 5 + 2 * kSsWPackedStages;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kTotal = kMiscOff + 16 + 1024;
@@ -64,8 +73,8 @@ __device__ __forceinline__ void tc_mma_i8_ss_pair(uint32_t d_tmem, uint64_t a_de
         : "memory");
 }
 
-template <bool RAW>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kSsThreads, 1)
+template <bool RAW, int EW>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((EW == 8 ? kSsFirstEpilogueWarp2 + 4 : kSsFirstEpilogueWarp2) * 32, 1)
 qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                 const __grid_constant__ CUtensorMap tmY, const float* __restrict__ scales,
                 const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
@@ -102,7 +111,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (threadIdx.x == 0) {
         for (int s = 0; s < kSsAStages; ++s) { mbar_init(a_full(s), 1); mbar_init(a_ready(s), 2); mbar_init(a_empty(s), 1); }
         for (int s = 0; s < kSsStages; ++s) { mbar_init(ops_full(s), 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
-        for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * kEpilogueWarps); }
+        for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * EW); }
         mbar_init(drain_bar, 1);
         for (int s = 0; s < kSsWPackedStages; ++s) { mbar_init(wp_full(s), 1); mbar_init(wp_empty(s), kSsWWarps / kUnpackGroups); }
         misc[1] = 0u;
@@ -217,25 +226,28 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             mbar_wait(drain_bar, 0u, abort_flag, kWaitDrain);
         }
         __syncwarp();
-    } else if (warp < kSsFirstWWarp) {
+    } else if (warp < kSsFirstWWarp || warp >= kSsFirstEpilogueWarp2) {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;  // tensor-memory lane quarter this warp may read
-        const int ew = warp - kFirstEpilogueWarp;
-        const uint32_t c_delta = sbase + S::kConstOff + ew * S::kConstPerWarp;  // shared addresses of float[BN] each
-        const uint32_t c_zc = c_delta + BN * 4;    // (z_n - 8) as a float: exact, |.| <= 8
-        const uint32_t c_bias = c_zc + BN * 4;
-        const uint32_t stg0 = sbase + S::kStageOutOff + ew * S::kStageOutPerWarp;
+        const int half = warp >= kSsFirstEpilogueWarp2 ? 1 : 0;  // EW = 8: which 128 of the tile's 256 columns
+        const int ew = 4 * half + q;
+        constexpr int CW = BN / (EW / 4);           // columns per warp
+        constexpr int RB = EW == 8 ? 64 : 128;      // bytes per row of the staging buffer = of a TMA store
+        const uint32_t c_delta = sbase + S::kConstOff + ew * (3 * CW * 4);  // shared addresses of float[CW] each
+        const uint32_t c_zc = c_delta + CW * 4;    // (z_n - 8) as a float: exact, |.| <= 8
+        const uint32_t c_bias = c_zc + CW * 4;
+        const uint32_t stg0 = sbase + S::kStageOutOff + ew * (32 * RB);
         constexpr int kShift = 4;  // the widened weights are 16 x (u - 8)
         if (!RAW && lane == 0) tma_prefetch_desc(&tmY);
-        uint32_t lt = 0, nstore = 0;
+        uint32_t lt = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++lt) {
             const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
-            const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM, n0 = (tile % num_n) * BN;
+            const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM, n0 = (tile % num_n) * BN + half * CW;
             __syncwarp();
-            {   // per-channel constants of this tile: all loads in flight at once, then the stores
-                float cd[BN / 32], cz[BN / 32], cb[BN / 32];
+            {   // per-channel constants of this warp's columns: all loads in flight at once, then the stores
+                float cd[CW / 32], cz[CW / 32], cb[CW / 32];
 #pragma unroll
-                for (int i = 0; i < BN / 32; ++i) {
+                for (int i = 0; i < CW / 32; ++i) {
                     const int n = n0 + lane + 32 * i;
                     const bool okn = n < N;
                     cd[i] = okn ? __ldg(delta + n) : 0.f;
@@ -243,7 +255,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     cb[i] = (okn && bias != nullptr) ? __bfloat162float(bias[n]) : 0.f;
                 }
 #pragma unroll
-                for (int i = 0; i < BN / 32; ++i) {
+                for (int i = 0; i < CW / 32; ++i) {
                     const int c = lane + 32 * i;
                     sts32f(c_delta + 4 * c, cd[i]);
                     sts32f(c_zc + 4 * c, cz[i]);
@@ -263,9 +275,9 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const float s_k = s_i * (1.0f / (float)(1 << kShift)), nS_k = -S_f * (float)(1 << kShift);
             const uint64_t s2 = f2_pack(s_k, s_k), negS2 = f2_pack(nS_k, nS_k);
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = 0; c < CW / 32; ++c) {
                 uint32_t r[32];
-                tmem_ld_32x32(tmem_base + a * BN + c * 32 + ((uint32_t)(q * 32) << 16), r);
+                tmem_ld_32x32(tmem_base + a * BN + half * CW + c * 32 + ((uint32_t)(q * 32) << 16), r);
                 tmem_ld_wait();
                 const int nb = n0 + c * 32;
                 if (RAW) {
@@ -281,10 +293,9 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         if (row_ok && nb + j < N) *reinterpret_cast<int4*>(dst + j) = o;
                     }
                 } else {
-                    // Two chunks of 32 columns fill one staging buffer of 32 rows x 128 bytes, which
-                    // leaves as ONE TMA store (128-byte rows are what TMA moves at full rate).  The
-                    // buffer used two stores ago must have been read by its store.
-                    if ((c & 1) == 0) {
+                    // RB / 64 chunks of 32 columns fill the staging buffer (32 rows x RB bytes), which
+                    // leaves as one TMA store; the previous store must have read the buffer.
+                    if (RB == 64 || (c & 1) == 0) {
                         if (lane == 0) tma_store_wait_read<0>();
                         __syncwarp();
                     }
@@ -318,19 +329,20 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * t], v[2 * t + 1]);
                             pk[t] = *reinterpret_cast<uint32_t*>(&b2);
                         }
-                        // 128-byte rows, 16-byte chunk index XORed with row % 8: the layout a
-                        // 128B-swizzled TMA store reads, and conflict-free for this per-row write.
-                        const int ch = (4 * (c & 1) + (j >> 3)) ^ (lane & 7);
-                        sts128(buf + lane * 128 + ch * 16, pk[0], pk[1], pk[2], pk[3]);
+                        // The layout a swizzled TMA store reads, conflict-free for this per-row write:
+                        // 128-byte rows, 16-byte chunk index XORed with row % 8, or 64-byte rows, chunk
+                        // index XORed with (row / 2) % 4.
+                        const int ch = RB == 128 ? (4 * (c & 1) + (j >> 3)) ^ (lane & 7) : (j >> 3) ^ ((lane >> 1) & 3);
+                        sts128(buf + lane * RB + ch * 16, pk[0], pk[1], pk[2], pk[3]);
                     }
-                    if (c & 1) {
+                    if (RB == 64 || (c & 1)) {
+                        const int x0 = RB == 64 ? nb : nb - 32;
                         fence_proxy_async_smem();
                         __syncwarp();
-                        if (lane == 0 && nb - 32 < N && m0 + q * 32 < M) {
-                            tma_store_2d(&tmY, buf, nb - 32, m0 + q * 32);
+                        if (lane == 0 && x0 < N && m0 + q * 32 < M) {
+                            tma_store_2d(&tmY, buf, x0, m0 + q * 32);
                             tma_store_commit();
                         }
-                        ++nstore;
                     }
                 }
             }
@@ -407,8 +419,22 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
 // ------------------------------------------------------------------ host side
 
-template <bool RAW>
-static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+// bf16 matrix [rows, cols] with row pitch ld elements, tiles of 32 rows x 32 columns, 64-byte
+// swizzle (the layout this kernel's epilogue stages its output in).
+inline bool make_out_map32(CUtensorMap* tm, const void* base, uint64_t cols, uint64_t rows, uint64_t ld) {
+    PFN_encodeTiled enc = get_encode_tiled();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {ld * 2};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool RAW, int EW>
+static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
                                    int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
     using S = SsSmem;
@@ -423,10 +449,12 @@ static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const
         return DVDQ_ERR_CUDA;
     if (RAW) {
         tmY = tmA;  // unused
-    } else if (!make_out_map(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)) {
+    } else if (!(EW == 8 ? make_out_map32(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)
+                         : make_out_map(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy))) {
         return DVDQ_ERR_CUDA;
     }
-    auto kern = qgemm_ss_kernel<RAW>;
+    constexpr int kThreads = (EW == 8 ? kSsFirstEpilogueWarp2 + 4 : kSsFirstEpilogueWarp2) * 32;
+    auto kern = qgemm_ss_kernel<RAW, EW>;
     static int max_pairs = 0;
     if (max_pairs == 0) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) return DVDQ_ERR_CUDA;
@@ -435,7 +463,7 @@ static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const
         if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DVDQ_ERR_CUDA;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(sm_count & ~1), 1, 1);
-        cfg.blockDim = dim3(kSsThreads, 1, 1);
+        cfg.blockDim = dim3(kThreads, 1, 1);
         cfg.dynamicSmemBytes = S::kTotal;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -448,12 +476,23 @@ static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const
     }
     const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + kSsBN - 1) / kSsBN);
     const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
-    kern<<<2 * pairs, kSsThreads, S::kTotal, st>>>(tmA, tmW, tmY, scales, sums,
+    kern<<<2 * pairs, kThreads, S::kTotal, st>>>(tmA, tmW, tmY, scales, sums,
                                                    reinterpret_cast<const float*>(blob + L.delta_offset),
                                                    reinterpret_cast<const int32_t*>(blob + L.zc_offset),
                                                    static_cast<const __nv_bfloat16*>(bias), acc_out, ldacc, (int)M, (int)N, (int)K,
                                                    act, spr);
     return cuda_status(cudaGetLastError());
+}
+
+// Eight epilogue warps where the epilogue would otherwise set the pace: a tile's mainloop is K / 128
+// k-blocks long, its epilogue always 256 columns, and a GELU about doubles the epilogue's work.
+template <bool RAW>
+static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+                                   const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
+                                   int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
+    const bool wide_epilogue = w.K <= 2048 || (act != 0 && w.K <= 6144);
+    return wide_epilogue ? launch_qgemm_ss_t<RAW, 8>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
+                         : launch_qgemm_ss_t<RAW, 4>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
 }
 
 }  // namespace dvdq
