@@ -65,6 +65,7 @@ def test_rotate_quantize_into_bytes_matches_oracle_and_packed_layout(M, K, Bk, b
 
 CASES = [
     # M, N, K, B, bits, weight mode: M and N tails (N against the 256-wide tile), odd and even numbers of k-blocks, z != 8
+    (1, 8, 64, 64, 6, "minmax"),
     (256, 256, 256, 256, 4, "symmetric"),
     (130, 264, 320, 64, 4, "minmax"),
     (300, 520, 1536, 512, 6, "symmetric"),
@@ -87,7 +88,7 @@ def test_int32_accumulators_are_bit_exact(M, N, K, Bk, bits, mode):
 
 
 @pytest.mark.parametrize("act", [0, 1])
-@pytest.mark.parametrize("M,N,K,Bk,bits,mode", CASES[1:4])
+@pytest.mark.parametrize("M,N,K,Bk,bits,mode", CASES[2:5])
 def test_qlinear_matches_oracle_and_packed_layout(M, N, K, Bk, bits, mode, act):
     x = synth_x(M, K, seed=7 * M + N)
     u, d, z = orc.prepare_weights(to_bits(synth_w(N, K, M + N + 2, mode)), Bk, mode)
@@ -110,3 +111,12 @@ def test_qlinear_matches_oracle_and_packed_layout(M, N, K, Bk, bits, mode, act):
             assert np.abs(y - y_or).max() <= Y_MAXNORM_RTOL * np.abs(y_or).max()
     # same integers, and the epilogues differ only by exact powers of two: identical outputs
     assert torch.equal(ys[0], ys[1])
+
+
+def test_empty_input_is_a_no_op():
+    q = act_quant(4, 256, 8)
+    x = torch.empty(0, 256, dtype=torch.bfloat16, device=DEV)
+    one = torch.zeros(256, dtype=torch.uint8, device=DEV)
+    B.dvdq_rotate_quantize(x, q, one, torch.zeros(1, device=DEV), torch.zeros(1, dtype=torch.int32, device=DEV))
+    assert_device_ok()
+    assert B.dvdq_act_codes_bytes_q(0, 256, q) == 0
