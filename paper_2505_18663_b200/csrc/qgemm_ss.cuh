@@ -37,7 +37,6 @@ constexpr int kSsStages = 4;         // widened weight half-tiles of one k-block
 constexpr int kSsWPackedStages = 4;  // ring of packed weight half-tiles
 constexpr int kSsFirstWWarp = 6, kSsWWarps = 8, kSsFwdWarp = kSsFirstWWarp + kSsWWarps, kSsWProducerWarp = kSsFwdWarp + 1;
 constexpr int kSsFirstEpilogueWarp2 = kSsWProducerWarp + 1;  // a multiple of 4: warp w reads tensor-memory lanes 32 * (w % 4)..
-constexpr int kSsMaxEpilogueWarps = 8;
 static_assert(kSsFirstEpilogueWarp2 % 4 == 0, "lane quarters");
 static_assert(kSsStages % 2 == 0, "the MMA warp takes the weight stages in pairs");
 
