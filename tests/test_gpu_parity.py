@@ -326,11 +326,13 @@ FULL_SIZE_CASES = [
 ]
 
 
+@pytest.mark.parametrize("container", [8, 0])
 @pytest.mark.parametrize("workload,layer_idx", FULL_SIZE_CASES)
-def test_full_size_layer_on_sampled_rows(workload, layer_idx):
-    """Full token counts of the benchmark configurations: scales, codes and bf16 outputs on
-    sampled rows (first tile, last full tile, ragged tail, seeded rows), computed one row at a
-    time by the oracle; plus a property of the whole output."""
+def test_full_size_layer_on_sampled_rows(workload, layer_idx, container):
+    """Full token counts of the benchmark configurations, with the codes kept one int8 each (what
+    the benchmark times by default) and packed: scales, codes and bf16 outputs on sampled rows
+    (first tile, last full tile, ragged tail, seeded rows), computed one row at a time by the
+    oracle; plus a property of the whole output."""
     wl = W.WORKLOADS[workload]
     layer = wl.layers[layer_idx]
     M = wl.M
@@ -338,7 +340,7 @@ def test_full_size_layer_on_sampled_rows(workload, layer_idx):
     u, d, z = W.make_weight_codes(layer, seed=layer_idx, device=DEV, symmetric=(layer_idx != 3))
     blob = torch.empty(B.dvdq_weight_blob_bytes(layer.N, layer.K), dtype=torch.uint8, device=DEV)
     w = B.dvdq_pack_weights(u, d, z, layer.rot_block, blob)
-    q = act_quant(layer.bits, layer.rot_block)
+    q = act_quant(layer.bits, layer.rot_block, container)
     ws = torch.empty(B.dvdq_qlinear_workspace_bytes(M, layer.K, q), dtype=torch.uint8, device=DEV)
     Y = torch.empty(M, layer.N, dtype=torch.bfloat16, device=DEV)
     bias = W.make_bias(wl, layer, device=DEV)
