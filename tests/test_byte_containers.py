@@ -120,3 +120,26 @@ def test_empty_input_is_a_no_op():
     B.dvdq_rotate_quantize(x, q, one, torch.zeros(1, device=DEV), torch.zeros(1, dtype=torch.int32, device=DEV))
     assert_device_ok()
     assert B.dvdq_act_codes_bytes_q(0, 256, q) == 0
+
+
+@pytest.mark.parametrize("bits", [4, 6, 8])
+def test_int32_accumulators_at_code_extremes_and_the_largest_k(bits):
+    # every product at its largest magnitude, K at the library's limit: |acc| = K * 2^(bits-1) * 15,
+    # and 16 x that inside the tensor core (the widened weights are 16 (u - 8)): still below 2^31
+    M, N, K = 128, 264, 16384
+    lim = 2 ** (bits - 1)
+    codes = np.full((M, K), -lim, dtype=np.int32)
+    codes[1::2] = lim - 1
+    u = np.zeros((N, K), dtype=np.uint8)
+    u[::2] = 15
+    z = np.zeros(N, dtype=np.int32)
+    z[1::2] = 15
+    d = np.ones(N, dtype=np.float32)
+    acc_or = orc.int_gemm(codes, u, z)
+    assert np.abs(acc_or).max() == lim * 15 * K
+    w, blob = gpu_pack_weights(u, d, z, 1024)
+    packed, sums = gpu_pack_codes(codes, bits, 1024, container=8)
+    acc = torch.zeros(M, N, dtype=torch.int32, device=DEV)
+    B.dvdq_qgemm_int32(packed, sums, M, act_quant(bits, 1024, 8), w, acc)
+    assert_device_ok()
+    assert np.array_equal(acc.cpu().numpy(), acc_or)
