@@ -157,6 +157,14 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
     return __all_sync(0xFFFFFFFFu, ok);
 }
 
+// Before a buffer that this thread has READ is handed back to whoever overwrites it (a TMA copy
+// armed by the arrive that follows): a CTA-scope fence, which waits until the thread's loads have
+// delivered.  An mbarrier arrive is not a shared-memory access in the load pipeline: without the
+// fence it could be performed while a load issued before it was still waiting, and the refill
+// landed first -- seen as one stale 32-byte piece of an operand row in about one kernel in two
+// at 65536 tokens, never in small cases.
+__device__ __forceinline__ void fence_loads_done() { asm volatile("fence.acq_rel.cta;" ::: "memory"); }
+
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* m) {

@@ -532,6 +532,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     }
                 }
                 // the codes are widened in registers before the stage of tensor memory is known to be free
+                fence_loads_done();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pk_empty(pst));
                 if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
@@ -570,6 +571,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
 #pragma unroll
                 for (int jw = 0; jw < 4; ++jw) { e[it][jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[it][jw] = w[jw] & 0xF0F0F0F0u; }
             }
+            fence_loads_done();
             __syncwarp();
             if (lane == 0) mbar_arrive(wp_empty(pst));  // the packed rows are in registers
             if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }

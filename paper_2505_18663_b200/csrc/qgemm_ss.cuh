@@ -489,6 +489,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
                 for (int jw = 0; jw < 4; ++jw) { e[it][jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[it][jw] = w[jw] & 0xF0F0F0F0u; }
             }
+            fence_loads_done();
             __syncwarp();
             if (lane == 0) mbar_arrive(wp_empty(pst));  // the packed rows are in registers
             if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
