@@ -286,6 +286,21 @@ def run_cuda(args, wl):
                        "rq_ms": rq_ms[li], "rq_gbs": rq_bytes(M, layer, args.scale_group, args.container) / (rq_ms[li] * 1e-3) / 1e9,
                        "qgemm_ms": gm_ms[li], "qgemm_tops": layer_ops(M, layer) / (gm_ms[li] * 1e-3) / 1e12})
 
+    # ---- rotate-quantize on its own (no GEMM between the launches, so no GEMM drawing the power budget down)
+    n_alone = max(5, args.steps // 5)
+    ev_alone = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers] for _ in range(n_alone)]
+    for it in range(3 + n_alone):
+        for li, L in enumerate(layers):
+            layer = L["layer"]
+            if it >= 3:
+                ev_alone[it - 3][li][0].record()
+            B.dvdq_rotate_quantize(xs[layer.K], L["q"], L["codes"], L["scales"], L["sums"])
+            if it >= 3:
+                ev_alone[it - 3][li][1].record()
+    torch.cuda.synchronize()
+    rq_alone_ms = sum(a.elapsed_time(b) for row in ev_alone for a, b in row) / n_alone
+    rq_alone_gbs = rq_total_bytes / (rq_alone_ms * 1e-3) / 1e9
+
     # ---- the same step with the codes packed b bits each (container 0), for the record: fewer steps
     packed = None
     if args.container != 0 and not args.no_packed and world == 1:
@@ -315,7 +330,9 @@ def run_cuda(args, wl):
         "roofline_rotate_quantize": {"kernel": "rq_kernel", "bound": "hbm", "achieved": rq_gbs,
                                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rq_gbs / peaks["hbm_gbs"],
                                      "peak_source": peaks["source"], "frac_of_nominal_8000": rq_gbs / 8000.0,
-                                     "avg_launch_ms": sum(rq_ms) / len(rq_ms), "traffic": RQ_DRAM_TRAFFIC_PER_LAUNCH if captured else None},
+                                     "avg_launch_ms": sum(rq_ms) / len(rq_ms), "traffic": RQ_DRAM_TRAFFIC_PER_LAUNCH if captured else None,
+                                     "alone": {"achieved": rq_alone_gbs, "frac": rq_alone_gbs / peaks["hbm_gbs"], "steps": n_alone,
+                                               "note": "the same launches without the GEMMs between them"}},
         "stages": stages,
         "packed_codes": packed,
         "e2e": e2e,
