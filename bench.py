@@ -287,9 +287,9 @@ def run_cuda(args, wl):
                        "qgemm_ms": gm_ms[li], "qgemm_tops": layer_ops(M, layer) / (gm_ms[li] * 1e-3) / 1e12})
 
     # ---- rotate-quantize on its own (no GEMM between the launches, so no GEMM drawing the power budget down)
-    n_alone = max(5, args.steps // 5)
+    n_alone = 0 if args.no_alone else max(5, args.steps // 5)
     ev_alone = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers] for _ in range(n_alone)]
-    for it in range(3 + n_alone):
+    for it in range(3 + n_alone if n_alone else 0):
         for li, L in enumerate(layers):
             layer = L["layer"]
             if it >= 3:
@@ -298,8 +298,12 @@ def run_cuda(args, wl):
             if it >= 3:
                 ev_alone[it - 3][li][1].record()
     torch.cuda.synchronize()
-    rq_alone_ms = sum(a.elapsed_time(b) for row in ev_alone for a, b in row) / n_alone
-    rq_alone_gbs = rq_total_bytes / (rq_alone_ms * 1e-3) / 1e9
+    rq_alone = None
+    if n_alone:
+        rq_alone_ms = sum(a.elapsed_time(b) for row in ev_alone for a, b in row) / n_alone
+        rq_alone_gbs = rq_total_bytes / (rq_alone_ms * 1e-3) / 1e9
+        rq_alone = {"achieved": rq_alone_gbs, "frac": rq_alone_gbs / load_peaks()["hbm_gbs"], "steps": n_alone,
+                    "note": "the same launches without the GEMMs between them"}
 
     # ---- the same step with the codes packed b bits each (container 0), for the record: fewer steps
     packed = None
@@ -331,8 +335,7 @@ def run_cuda(args, wl):
                                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rq_gbs / peaks["hbm_gbs"],
                                      "peak_source": peaks["source"], "frac_of_nominal_8000": rq_gbs / 8000.0,
                                      "avg_launch_ms": sum(rq_ms) / len(rq_ms), "traffic": RQ_DRAM_TRAFFIC_PER_LAUNCH if captured else None,
-                                     "alone": {"achieved": rq_alone_gbs, "frac": rq_alone_gbs / peaks["hbm_gbs"], "steps": n_alone,
-                                               "note": "the same launches without the GEMMs between them"}},
+                                     "alone": rq_alone},
         "stages": stages,
         "packed_codes": packed,
         "e2e": e2e,
@@ -481,6 +484,7 @@ def main():
     ap.add_argument("--container", type=int, default=8,
                     help="8: one int8 per activation code (default, the faster GEMM); 0: codes packed b bits each")
     ap.add_argument("--no-packed", action="store_true", help="skip the extra leg that times the packed layout")
+    ap.add_argument("--no-alone", action="store_true", help="skip the extra leg that times rotate-quantize on its own")
     ap.add_argument("--scale-group", type=int, default=0,
                     help="0: one activation scale per token; 1024: one per token and block of 1024 channels")
     ap.add_argument("--bits", type=int, default=0, help="override the activation bit width of every layer (4, 6 or 8)")
