@@ -143,3 +143,32 @@ def test_int32_accumulators_at_code_extremes_and_the_largest_k(bits):
     B.dvdq_qgemm_int32(packed, sums, M, act_quant(bits, 1024, 8), w, acc)
     assert_device_ok()
     assert np.array_equal(acc.cpu().numpy(), acc_or)
+
+
+@pytest.mark.parametrize("workload,layer_idx", [("hunyuan", 3), ("hunyuan", 0), ("wan1p3b", 1), ("ffn_chain", 0)])
+def test_full_size_outputs_repeat_and_agree_across_layouts(workload, layer_idx):
+    """At the benchmark's token counts every launch must give the same bits, in both code layouts
+    (long K, 6-bit codes, the eight-epilogue-warp variant with and without GELU): a stage handed
+    back to its producer too early, or read too early, shows here as a few columns of one tile."""
+    from paper_2505_18663_b200 import workloads as W
+    wl = W.WORKLOADS[workload]
+    layer = wl.layers[layer_idx]
+    M = min(wl.M, 65536)
+    x = W.make_activations(wl, layer.K, device=DEV)[:M]
+    u, d, z = W.make_weight_codes(layer, seed=layer_idx, device=DEV, symmetric=False)
+    blob = torch.empty(B.dvdq_weight_blob_bytes(layer.N, layer.K), dtype=torch.uint8, device=DEV)
+    w = B.dvdq_pack_weights(u, d, z, layer.rot_block, blob)
+    bias = W.make_bias(wl, layer, device=DEV)
+    ref = None
+    for container in (0, 8):
+        q = act_quant(layer.bits, layer.rot_block, container)
+        ws = torch.empty(B.dvdq_qlinear_workspace_bytes(M, layer.K, q), dtype=torch.uint8, device=DEV)
+        for rep in range(6):
+            Y = torch.empty(M, layer.N, dtype=torch.bfloat16, device=DEV)
+            B.dvdq_qlinear(x, q, w, bias, layer.act, Y, ws)
+            assert_device_ok()
+            if ref is None:
+                ref = Y
+            else:
+                bad = int((Y != ref).sum())
+                assert bad == 0, f"container_bits={container}, launch {rep}: {bad} outputs differ"
