@@ -203,3 +203,30 @@ def test_blockwise_scales_lower_the_quantization_error():
         assert_device_ok()
         errs.append(np.linalg.norm(Y.to(torch.float64).cpu().numpy() - exact))
     assert errs[1] < 0.85 * errs[0], errs
+
+
+@pytest.mark.parametrize("layer_idx", [3, 0])
+def test_full_size_blockwise_outputs_repeat_and_agree_across_layouts(layer_idx):
+    """The benchmark's token count with block-wise scales: every launch gives the same bits, with
+    the codes packed and kept in bytes (twelve blocks of 1024 per token on the long layer)."""
+    from paper_2505_18663_b200 import workloads as W
+    wl = W.WORKLOADS["hunyuan"]
+    layer = wl.layers[layer_idx]
+    M = wl.M
+    x = W.make_activations(wl, layer.K, device=DEV)
+    u, d, z = W.make_weight_codes(layer, seed=layer_idx, device=DEV, symmetric=False)
+    blob = torch.empty(B.dvdq_weight_blob_bytes(layer.N, layer.K), dtype=torch.uint8, device=DEV)
+    w = B.dvdq_pack_weights(u, d, z, layer.rot_block, blob)
+    ref = None
+    for container in (0, 8):
+        q = B.ActQuant(layer.bits, layer.rot_block, G, container)
+        ws = torch.empty(B.dvdq_qlinear_workspace_bytes(M, layer.K, q), dtype=torch.uint8, device=DEV)
+        for rep in range(4):
+            Y = torch.empty(M, layer.N, dtype=torch.bfloat16, device=DEV)
+            B.dvdq_qlinear(x, q, w, None, 0, Y, ws)
+            assert_device_ok()
+            if ref is None:
+                ref = Y
+            else:
+                bad = int((Y != ref).sum())
+                assert bad == 0, f"container_bits={container}, launch {rep}: {bad} outputs differ"
