@@ -211,6 +211,17 @@ def epilogue(acc: np.ndarray, scale32: np.ndarray, delta32: np.ndarray, bias_bf1
     return y
 
 
+def round_output(v: np.ndarray, bias_bf16=None, act: int = 0) -> np.ndarray:
+    """The tail of the epilogue on values already dequantized in fp64:
+    y = bf16(v + bias_n) [then GELU-tanh and a second bf16 rounding if act == 1].  bf16 bits [M,N]."""
+    v = _c(v, np.float64)
+    M, N = v.shape
+    b = None if bias_bf16 is None else _c(bias_bf16, np.uint16)
+    y = np.empty((M, N), dtype=np.uint16)
+    _load().oracle_round_output(_ptr(v), None if b is None else _ptr(b), act, M, N, _ptr(y))
+    return y
+
+
 def exact_linear(x: np.ndarray, w: np.ndarray) -> np.ndarray:
     """Y = X W^T in fp64 (the product the method approximates)."""
     x = _c(x, np.float64)
@@ -302,11 +313,7 @@ def combine_grouped(codes, u, z, s32, delta32, group: int, bias_bf16=None, act: 
         acc = int_gemm(np.ascontiguousarray(codes[:, sl]), np.ascontiguousarray(u[:, sl]), z)
         v += acc.astype(np.float64) * s32[:, g].astype(np.float64)[:, None]
     v *= np.asarray(delta32, dtype=np.float32).astype(np.float64)[None, :]
-    v = np.ascontiguousarray(v)
-    b = None if bias_bf16 is None else _c(bias_bf16, np.uint16)
-    y = np.empty((M, N), dtype=np.uint16)
-    _load().oracle_round_output(_ptr(v), None if b is None else _ptr(b), act, M, N, _ptr(y))
-    return y
+    return round_output(v, bias_bf16, act)
 
 
 def qlinear_grouped(x_bf16, u, delta32, z, B: int, bits: int, group: int, bias_bf16=None, act: int = 0):

@@ -341,20 +341,26 @@ def test_full_size_layer_on_sampled_rows(workload, layer_idx, container):
     blob = torch.empty(B.dvdq_weight_blob_bytes(layer.N, layer.K), dtype=torch.uint8, device=DEV)
     w = B.dvdq_pack_weights(u, d, z, layer.rot_block, blob)
     q = act_quant(layer.bits, layer.rot_block, container)
-    ws = torch.empty(B.dvdq_qlinear_workspace_bytes(M, layer.K, q), dtype=torch.uint8, device=DEV)
+    codes = torch.empty(B.dvdq_act_codes_bytes_q(M, layer.K, q), dtype=torch.uint8, device=DEV)
+    scales = torch.empty(M, dtype=torch.float32, device=DEV)
+    sums = torch.empty(M, dtype=torch.int32, device=DEV)
     Y = torch.empty(M, layer.N, dtype=torch.bfloat16, device=DEV)
     bias = W.make_bias(wl, layer, device=DEV)
-    B.dvdq_qlinear(x, q, w, bias, layer.act, Y, ws)
+    # the two launches of a layer, as the benchmark issues them
+    B.dvdq_rotate_quantize(x, q, codes, scales, sums)
+    B.dvdq_qgemm(codes, scales, sums, M, q, w, bias, layer.act, Y)
     assert_device_ok()
     rows = W.sample_rows(M, 40, tile=256, seed=layer_idx)
     xs = x[rows.to(DEV)].cpu()
     un, dn, zn = u.cpu().numpy(), d.cpu().numpy(), z.cpu().numpy()
     bias_bits = None if bias is None else to_bits(bias)
     out = orc.qlinear(to_bits(xs), un, dn, zn, layer.rot_block, layer.bits, bias_bits, layer.act)
-    # the workspace starts with the packed codes of every token; unpack only the sampled rows' worth
+    s_gpu = scales[rows.to(DEV)].cpu().numpy().astype(np.float64)
+    assert np.abs(s_gpu / out["scale64"] - 1.0).max() <= SCALE_RTOL
     nat = torch.empty(M, layer.K, dtype=torch.int8, device=DEV)
-    B.dvdq_unpack_act_codes(ws, M, layer.K, q, nat)
+    B.dvdq_unpack_act_codes(codes, M, layer.K, q, nat)
     nat_s = nat[rows.to(DEV)].cpu().numpy()
+    assert np.array_equal(sums[rows.to(DEV)].cpu().numpy(), nat_s.astype(np.int64).sum(axis=1))
     del nat
     y = Y[rows.to(DEV)].to(torch.float64).cpu().numpy()
     y_or = oracle_y_for_validated_codes(nat_s, out, un, dn, zn, bias_bits, layer.act)

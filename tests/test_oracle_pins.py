@@ -344,3 +344,33 @@ def test_grouped_quantizer_reduces_to_the_per_token_one_and_keeps_its_invariants
     err_tok = np.linalg.norm(bf16_values(b["y"]) - exact)
     err_blk = np.linalg.norm(bf16_values(c["y"]) - exact)
     assert err_blk < err_tok
+
+
+def test_round_output_adds_the_bias_before_the_rounding_and_rounds_twice_around_the_gelu():
+    # Hand-set fp64 values and bf16 biases; the expected bits come from torch alone: fp64 add, its
+    # cast to bf16 (ties to even), its tanh-GELU in fp64 on the rounded value, its cast again.
+    # 1.00390625 = 1 + 2^-8 is a bf16 tie (rounds down to 1.0 on its own); the bias 2^-9 lifts the
+    # sum above the tie, so adding the bias AFTER the rounding gives a different bit pattern.
+    v = np.array([[1.00390625, -2.7, 0.3333, 117.25, -0.0625, 3.0e-3],
+                  [0.0, 5.5, -1.00390625, 0.49, 12.0, -40.0]], dtype=np.float64)
+    bias = torch.tensor([2.0 ** -9, 0.5, -0.25, 3.0, 0.0625, -1.0e-3]).to(torch.bfloat16)
+    bias_bits = to_bits(bias)
+    summed = torch.from_numpy(v) + bias.to(torch.float64)[None, :]
+    ref0 = summed.to(torch.bfloat16)
+    ref1 = torch.nn.functional.gelu(ref0.to(torch.float64), approximate="tanh").to(torch.bfloat16)
+    y0 = orc.round_output(v, bias_bits, 0)
+    y1 = orc.round_output(v, bias_bits, 1)
+    assert np.array_equal(y0, to_bits(ref0))
+    assert np.array_equal(y1, to_bits(ref1))
+    # the tie really is decided by the bias: without it the first element rounds to 1.0
+    assert bf16_values(orc.round_output(v, None, 0))[0, 0] == 1.0 and bf16_values(y0)[0, 0] > 1.0
+    # one rounding after the GELU is not the same thing: a fused fp64 GELU of the unrounded sum differs somewhere
+    fused = torch.nn.functional.gelu(summed, approximate="tanh").to(torch.bfloat16)
+    assert not np.array_equal(y1, to_bits(fused))
+    # and it agrees with the per-token epilogue on the same numbers (acc * s * Delta formed here in fp64)
+    acc = np.array([[3, -5, 100, 7, -9, 1]], dtype=np.int32)
+    s = np.array([0.37], dtype=np.float32)
+    dl = np.array([0.11, 0.23, 0.01, 0.5, 0.07, 0.9], dtype=np.float32)
+    vv = acc.astype(np.float64) * s.astype(np.float64)[:, None] * dl.astype(np.float64)[None, :]
+    for act in (0, 1):
+        assert np.array_equal(orc.round_output(vv, bias_bits, act), orc.epilogue(acc, s, dl, bias_bits, act))
