@@ -127,7 +127,7 @@ dvdq_status dvdq_rotate_quantize(const void* X_bf16, int64_t M, int64_t K, int64
 
 /* ---- (0) offline weight packing: Sec. 3.1 Quant/DeQuant format, Eq. 10 W^ ----------
  *
- * Takes weights that are ALREADY rotated (W~ = W R, same B as the activations) and
+ * Takes weights that are ALREADY rotated (W~ = W R, same B as the activations: dvdq_rotate_weights) and
  * quantized to the format W^ = Delta (W_q - z):
  *   Wq     [N, K] uint8, values 0..15 (upper bits ignored)
  *   delta  [N] fp32 step sizes
@@ -140,6 +140,28 @@ dvdq_status dvdq_rotate_quantize(const void* X_bf16, int64_t M, int64_t K, int64
 dvdq_status dvdq_pack_weights(const uint8_t* Wq, const float* delta, const int32_t* zero,
                               int64_t N, int64_t K, int32_t rot_block,
                               void* blob_out, dvdq_weights* out /* host */, void* cuda_stream);
+
+/* ---- (0) offline weight rotation: Eq. 10, W^ = Quant(W H); Sec. 3.2 ------------------------
+ *
+ * W~ = W R along K with the same R = I_{K/B} (x) H_B / sqrt(B) as the activations, so that
+ * X~ W~^T = X W^T.  Butterflies and the normalisation in fp64, one rounding to fp32 at the end.
+ *   W_bf16     [N, K] bf16, row pitch ldw elements
+ *   W_rot_out  [N, K] fp32, dense: the input of dvdq_bgr_quantize
+ * K % 64 == 0, K <= 16384; rot_block as in dvdq_act_quant.  N == 0 is a no-op. */
+dvdq_status dvdq_rotate_weights(const void* W_bf16, int64_t N, int64_t K, int64_t ldw, int32_t rot_block,
+                                float* W_rot_out, void* cuda_stream);
+
+/* ---- (0) offline, in one call: rotate and quantize symmetrically into a blob -----------------
+ *
+ * The plain per-output-channel 4-bit quantizer in the format of Sec. 3.1 with the zero point
+ * pinned (not the paper's grid refinement, which is dvdq_bgr_quantize): W~ = W R as above, then
+ *     Delta_n = max_k |w~_nk| / 7,  W_q = clamp(round(w~ / Delta), -8, 7) + 8,  z_n = 8
+ * (fp64, round half to even; an all-zero row gets Delta = 1), written in the layout of
+ * dvdq_pack_weights.  blob_out: dvdq_weight_blob_bytes(N, K) bytes, 256-byte aligned; `out`
+ * (host) describes it.  N % 8 == 0, N > 0. */
+dvdq_status dvdq_quantize_weights_symmetric(const void* W_bf16, int64_t N, int64_t K, int64_t ldw,
+                                            int32_t rot_block, void* blob_out,
+                                            dvdq_weights* out /* host */, void* cuda_stream);
 
 /* ---- (0') offline weight quantizer: Bounded-init Grid Refinement, Alg. 1 / Sec. 3.1 ---------
  *
@@ -264,6 +286,18 @@ dvdq_status dvdq_unpack_act_codes(const void* codes, int64_t M, int64_t K,
 /* Blob -> Wq [N, K] uint8 (0..15), delta [N], zero [N]. */
 dvdq_status dvdq_unpack_weights(const dvdq_weights* w /* host */, uint8_t* Wq, float* delta,
                                 int32_t* zero, void* cuda_stream);
+
+/* Ceiling of the int8 tensor pipe for the roofline of dvdq_qgemm (Eq. 10's contraction): every
+ * CTA pair issues `iters` (1 .. 2^20) k-blocks of four 256 x 256 x 32 tcgen05.mma.kind::i8 on
+ * operands that stay in shared memory -- no loads, no widening, no epilogue.  *ops_out (host,
+ * may be NULL) receives the integer operations of the launch (2 per multiply-add); time the
+ * call with CUDA events on the stream. */
+dvdq_status dvdq_int8_mma_ceiling(int32_t iters, int64_t* ops_out /* host */, void* cuda_stream);
+
+/* Exercises the bounded-wait error path without harming the device: one warp waits on a
+ * barrier nobody arrives on, gives up after limit_ns (1 .. 1e9) and returns normally; afterwards
+ * dvdq_last_device_status() reports DVDQ_ERR_DEVICE_TIMEOUT with detail 8. */
+dvdq_status dvdq_debug_wait_timeout(uint64_t limit_ns, void* cuda_stream);
 
 /* Reads (and clears) the device-side status word of the current device; synchronizes
  * the device.  DVDQ_OK, or DVDQ_ERR_DEVICE_TIMEOUT with `detail` (host, may be NULL)

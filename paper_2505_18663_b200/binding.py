@@ -24,6 +24,7 @@ EXPORTS = [
     "dvdq_qlinear_workspace_bytes", "dvdq_rotate_quantize", "dvdq_pack_weights", "dvdq_qgemm",
     "dvdq_qlinear", "dvdq_qlinear_static", "dvdq_qgemm_int32", "dvdq_pack_act_codes", "dvdq_unpack_act_codes",
     "dvdq_unpack_weights", "dvdq_last_device_status",
+    "dvdq_rotate_weights", "dvdq_quantize_weights_symmetric", "dvdq_int8_mma_ceiling", "dvdq_debug_wait_timeout",
     "dvdq_bgr_quantize", "dvdq_gbs_l1_terms", "dvdq_gbs_init", "dvdq_gbs_next_bits", "dvdq_gbs_observe",
 ]
 
@@ -95,6 +96,10 @@ def load():
         "dvdq_unpack_weights": (C.c_int, [wp, p, p, p, p]),
         "dvdq_last_device_status": (C.c_int, [C.POINTER(C.c_uint32)]),
         "dvdq_bgr_quantize": (C.c_int, [p, i64, i64, i32, C.c_double, i32, p, p, p, p]),
+        "dvdq_rotate_weights": (C.c_int, [p, i64, i64, i64, i32, p, p]),
+        "dvdq_quantize_weights_symmetric": (C.c_int, [p, i64, i64, i64, i32, p, wp, p]),
+        "dvdq_int8_mma_ceiling": (C.c_int, [i32, C.POINTER(C.c_int64), p]),
+        "dvdq_debug_wait_timeout": (C.c_int, [C.c_uint64, p]),
         "dvdq_gbs_l1_terms": (C.c_int, [p, p, i64, p, p]),
         "dvdq_gbs_init": (C.c_int, [C.POINTER(GbsState), C.c_double, i32, i32]),
         "dvdq_gbs_next_bits": (i32, [C.POINTER(GbsState)]),
@@ -259,6 +264,38 @@ def dvdq_unpack_weights(w: Weights, Wq: torch.Tensor, delta: torch.Tensor, zero:
         raise TypeError("Wq must be contiguous")
     _check(load().dvdq_unpack_weights(C.byref(w), _ptr(Wq, torch.uint8, "Wq"), _ptr(delta, torch.float32, "delta"),
                                       _ptr(zero, torch.int32, "zero"), _stream(stream)), "dvdq_unpack_weights")
+
+
+def dvdq_rotate_weights(W: torch.Tensor, rot_block: int, W_rot: torch.Tensor, stream=None) -> None:
+    """W~ = W R along K: bf16 [N, K] -> dense fp32 [N, K]."""
+    ldw = _row_major(W, "W")
+    N, K = W.shape
+    if not W_rot.is_contiguous() or tuple(W_rot.shape) != (N, K):
+        raise TypeError("W_rot must be dense [N, K]")
+    _check(load().dvdq_rotate_weights(_ptr(W, torch.bfloat16, "W"), N, K, ldw, rot_block,
+                                      _ptr(W_rot, torch.float32, "W_rot"), _stream(stream)), "dvdq_rotate_weights")
+
+
+def dvdq_quantize_weights_symmetric(W: torch.Tensor, rot_block: int, blob: torch.Tensor, stream=None) -> Weights:
+    """bf16 [N, K] weights -> rotated, symmetric 4-bit codes (z = 8, Delta = absmax / 7) in a blob."""
+    ldw = _row_major(W, "W")
+    N, K = W.shape
+    w = Weights()
+    _check(load().dvdq_quantize_weights_symmetric(_ptr(W, torch.bfloat16, "W"), N, K, ldw, rot_block,
+                                                  _ptr(blob, torch.uint8, "blob"), C.byref(w), _stream(stream)),
+           "dvdq_quantize_weights_symmetric")
+    return w
+
+
+def dvdq_int8_mma_ceiling(iters: int, stream=None) -> int:
+    """Launches the int8 tensor-pipe issue loop; returns the integer operations of the launch."""
+    ops = C.c_int64(0)
+    _check(load().dvdq_int8_mma_ceiling(iters, C.byref(ops), _stream(stream)), "dvdq_int8_mma_ceiling")
+    return int(ops.value)
+
+
+def dvdq_debug_wait_timeout(limit_ns: int, stream=None) -> None:
+    _check(load().dvdq_debug_wait_timeout(int(limit_ns), _stream(stream)), "dvdq_debug_wait_timeout")
 
 
 def dvdq_bgr_quantize(W_rot: torch.Tensor, n_steps: int, eps: float, max_iter: int, Wq: torch.Tensor,

@@ -9,7 +9,6 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libdvdq.so")
 SOURCES = ["dvdq_lib.cu"]
-DEPS = ["dvdq_lib.cu", "dvdq_common.cuh", "rotate_quantize.cuh", "pack.cuh", "qgemm.cuh", "qgemm_ss.cuh", "gbs.cuh", "bgr.cuh"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 
@@ -25,7 +24,8 @@ def is_stale() -> bool:
     if not os.path.exists(LIB_PATH):
         return True
     t = os.path.getmtime(LIB_PATH)
-    deps = [os.path.join(CSRC, d) for d in DEPS] + [os.path.join(os.path.dirname(_HERE), "include", "dvdq.h")]
+    deps = [os.path.join(CSRC, d) for d in os.listdir(CSRC) if d.endswith((".cu", ".cuh"))]
+    deps.append(os.path.join(os.path.dirname(_HERE), "include", "dvdq.h"))
     return any(os.path.getmtime(d) > t for d in deps)
 
 

@@ -8,6 +8,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/dvdq.h"
 
 namespace dvdq {
@@ -22,7 +24,6 @@ constexpr int32_t kLibVersion = 1;
 // Storage order of the K axis, shared by activation codes and weight codes.  The integer
 // GEMM is a dot product over k, so any permutation applied to both operands gives the same
 // accumulators.
-constexpr int32_t kScaleBlock = 1024;          // channels per scale in the block-wise variant
 constexpr int32_t kKLayoutNatural = 0;        // position p holds logical channel p
 
 __host__ __device__ inline int64_t align_up(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
@@ -68,7 +69,7 @@ __device__ uint32_t g_device_status[2] = {0u, 0u};
 
 enum WaitId : uint32_t {
     kWaitPackedEmpty = 1, kWaitPackedFull = 2, kWaitWideEmpty = 3, kWaitWideFull = 4,
-    kWaitAccEmpty = 5, kWaitAccFull = 6, kWaitDrain = 7
+    kWaitAccEmpty = 5, kWaitAccFull = 6, kWaitDrain = 7, kWaitDebug = 8
 };
 
 __device__ __forceinline__ void report_timeout(uint32_t detail) {
@@ -131,7 +132,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // abort flag and returns false.  The caller then leaves its loop and walks to the common exit.
 constexpr uint64_t kWaitLimitNs = 4000000000ull;  // 4 s
 
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t wait_id) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t wait_id,
+                                                uint64_t limit_ns) {
     // Reading %globaltimer costs hundreds of cycles, so the clock is consulted only every 1024
     // failed polls (each poll already suspends the thread for a while in hardware).
     uint64_t t0 = 0;
@@ -141,13 +143,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const uint64_t now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            if (now - t0 > kWaitLimitNs) {
+            if (now - t0 > limit_ns) {
                 *abort_flag = 1u;
                 report_timeout(wait_id);
                 return false;
             }
         }
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag, uint32_t wait_id) {
+    return mbar_wait_limit(bar, parity, abort_flag, wait_id, kWaitLimitNs);
 }
 
 // mbar_wait by a fully converged warp with one answer for all lanes (a wait that gives up in some
@@ -164,6 +169,18 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
 // landed first -- seen as one stale 32-byte piece of an operand row in about one kernel in two
 // at 65536 tokens, never in small cases.
 __device__ __forceinline__ void fence_loads_done() { asm volatile("fence.acq_rel.cta;" ::: "memory"); }
+
+// The hand-back is also tied to the loaded data itself: the arrive's address is formed from a word of
+// every load (ANDed with a zero the compiler cannot see through, so the address does not change),
+// and an instruction cannot issue before its operands have been delivered.
+__device__ __forceinline__ uint32_t runtime_zero() {
+    uint32_t v;
+    asm volatile("mov.u32 %0, %%nctaid.y;" : "=r"(v));  // the grids here are one-dimensional: nctaid.y == 1
+    return v - 1u;
+}
+__device__ __forceinline__ void mbar_arrive_after_loads(uint32_t bar, uint32_t loaded_words_masked) {
+    mbar_arrive(bar + loaded_words_masked);
+}
 
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
@@ -366,7 +383,32 @@ __host__ __device__ constexpr uint32_t umma_idesc_s8s8s32(int m, int n) {
     return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-// ------------------------------------------------------------------ host helpers (api.cu)
+// ------------------------------------------------------------------ host helpers (dvdq_lib.cu)
+
+// Launch-time set-up that CUDA keeps per device (the opt-in to large dynamic shared memory, the
+// SM count, occupancy) is cached per device ordinal: one slot per device, filled with that
+// device current, under a lock so that host threads may share the library.
+constexpr int kMaxDevices = 64;
+
+template <typename T>
+struct PerDevice {
+    T slot[kMaxDevices] = {};
+    bool ready[kMaxDevices] = {};
+    std::mutex lock;
+    // Returns the current device's slot, calling init(slot, device) the first time; nullptr if
+    // the device cannot be queried or init reports failure.
+    template <typename Init>
+    T* get(Init init) {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+        std::lock_guard<std::mutex> g(lock);
+        if (!ready[dev]) {
+            if (!init(slot[dev], dev)) return nullptr;
+            ready[dev] = true;
+        }
+        return &slot[dev];
+    }
+};
 
 dvdq_status check_device_arch();
 dvdq_status validate_act_quant(const dvdq_act_quant* q, int64_t K);

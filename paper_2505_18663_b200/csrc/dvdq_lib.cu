@@ -1,6 +1,6 @@
 // C ABI of the library (see include/dvdq.h): argument validation, size queries and the
-// launches of the kernels in rotate_quantize.cuh, pack.cuh and qgemm.cuh.  One translation
-// unit, so that the device status word is a single symbol.
+// launches of the kernels in rotate_quantize.cuh, pack.cuh, weights.cuh, qgemm.cuh and
+// qgemm_ss.cuh.  One translation unit, so that the device status word is a single symbol.
 #include "dvdq_common.cuh"
 
 #include "bgr.cuh"
@@ -9,22 +9,20 @@
 #include "qgemm.cuh"
 #include "qgemm_ss.cuh"
 #include "rotate_quantize.cuh"
+#include "weights.cuh"
+#include "diag.cuh"
 
 namespace dvdq {
 
 dvdq_status cuda_status(cudaError_t e) { return e == cudaSuccess ? DVDQ_OK : DVDQ_ERR_CUDA; }
 
 dvdq_status check_device_arch() {
-    static int cached_dev = -1;
-    static dvdq_status cached = DVDQ_ERR_ARCH;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return DVDQ_ERR_CUDA;
-    if (dev == cached_dev) return cached;
-    int major = 0;
-    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return DVDQ_ERR_CUDA;
-    cached_dev = dev;
-    cached = (major == 10) ? DVDQ_OK : DVDQ_ERR_ARCH;
-    return cached;
+    static PerDevice<int> cache;  // compute-capability major of each device
+    int* major = cache.get([](int& m, int dev) {
+        return cudaDeviceGetAttribute(&m, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess;
+    });
+    if (!major) return DVDQ_ERR_CUDA;
+    return *major == 10 ? DVDQ_OK : DVDQ_ERR_ARCH;
 }
 
 static bool is_pow2(int64_t v) { return v > 0 && (v & (v - 1)) == 0; }
@@ -32,7 +30,7 @@ static bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintp
 
 // Shape rules shared by every entry point: K a multiple of 64 (16-byte TMA pitches for both
 // code widths and whole 16-code groups of the 6-bit high plane), K <= 16384 (one CTA holds a
-// token), rot_block 0 or a power of two in [64, 1024] dividing K.
+// token), rot_block 0 or a power of two in [64, 4096] dividing K.
 static dvdq_status validate_k(int64_t K) {
     if (K <= 0 || K % 64 != 0 || K > 16384) return DVDQ_ERR_SHAPE;
     return DVDQ_OK;
@@ -42,12 +40,12 @@ dvdq_status validate_act_quant(const dvdq_act_quant* q, int64_t K) {
     if (!q) return DVDQ_ERR_NULL;
     if (q->bits != 4 && q->bits != 6 && q->bits != 8) return DVDQ_ERR_BITS;
     if (q->container_bits != 0 && q->container_bits != 8) return DVDQ_ERR_UNSUPPORTED;
-    // block-wise scales: one per token and per 1024-channel block (the unit a warp of the transform
-    // and eight k-blocks of the GEMM work on); other block sizes are not built
-    if (q->scale_group != 0 && q->scale_group != kScaleBlock) return DVDQ_ERR_UNSUPPORTED;
-    if (q->scale_group != 0 && K % kScaleBlock != 0) return DVDQ_ERR_SHAPE;
+    // block-wise scales: one per token and per group of 128, 256 or 1024 consecutive rotated channels
+    // (whole k-blocks of the GEMM, which takes them in pairs: K a multiple of 256 and of the group)
+    if (q->scale_group != 0 && q->scale_group != 128 && q->scale_group != 256 && q->scale_group != 1024) return DVDQ_ERR_UNSUPPORTED;
+    if (q->scale_group != 0 && (K % q->scale_group != 0 || K % 256 != 0)) return DVDQ_ERR_SHAPE;
     if (q->rot_block != 0) {
-        if (!is_pow2(q->rot_block) || q->rot_block < 64 || q->rot_block > 1024) return DVDQ_ERR_ROT_BLOCK;
+        if (!is_pow2(q->rot_block) || q->rot_block < 64 || q->rot_block > 4096) return DVDQ_ERR_ROT_BLOCK;
         if (K % q->rot_block != 0) return DVDQ_ERR_ROT_BLOCK;
     }
     return DVDQ_OK;
@@ -164,6 +162,62 @@ dvdq_status dvdq_pack_weights(const uint8_t* Wq, const float* delta, const int32
     return DVDQ_OK;
 }
 
+// ---- offline weight preparation on the GPU (Eq. 10: W^ = Quant(W H)) ------------------------
+
+static int log2_of(int32_t b) {
+    int l = 0;
+    while ((1 << l) < b) ++l;
+    return l;
+}
+
+static dvdq_status check_weight_prep_args(const void* W, int64_t N, int64_t K, int64_t ldw, int32_t rot_block, const void* out) {
+    if (N < 0 || N > 0x7FFFFFFFll || validate_k(K) != DVDQ_OK || ldw < K) return DVDQ_ERR_SHAPE;
+    dvdq_act_quant probe = {4, rot_block, 0, 0};
+    dvdq_status s = validate_act_quant(&probe, K);
+    if (s != DVDQ_OK) return s;
+    if (N == 0) return DVDQ_OK;
+    if (!W || !out) return DVDQ_ERR_NULL;
+    if (!aligned(W, 2)) return DVDQ_ERR_ALIGN;
+    return DVDQ_OK;
+}
+
+dvdq_status dvdq_rotate_weights(const void* W, int64_t N, int64_t K, int64_t ldw, int32_t rot_block, float* W_rot_out,
+                                void* stream) {
+    dvdq_status s = check_weight_prep_args(W, N, K, ldw, rot_block, W_rot_out);
+    if (s != DVDQ_OK || N == 0) return s;
+    if (!aligned(W_rot_out, 4)) return DVDQ_ERR_ALIGN;
+    if ((s = check_device_arch()) != DVDQ_OK) return s;
+    static PerDevice<int> cache;
+    if (!weight_kernel_setup(cache, rotate_weights_kernel)) return DVDQ_ERR_CUDA;
+    rotate_weights_kernel<<<(unsigned)N, kWeightThreads, (size_t)K * sizeof(double), (cudaStream_t)stream>>>(
+        static_cast<const __nv_bfloat16*>(W), ldw, (int)K, log2_of(rot_block), W_rot_out);
+    return cuda_status(cudaGetLastError());
+}
+
+dvdq_status dvdq_quantize_weights_symmetric(const void* W, int64_t N, int64_t K, int64_t ldw, int32_t rot_block,
+                                            void* blob_out, dvdq_weights* out, void* stream) {
+    if (!out) return DVDQ_ERR_NULL;
+    if (N <= 0 || N % 8 != 0) return DVDQ_ERR_SHAPE;
+    dvdq_status s = check_weight_prep_args(W, N, K, ldw, rot_block, blob_out);
+    if (s != DVDQ_OK) return s;
+    if (!aligned(blob_out, 256)) return DVDQ_ERR_ALIGN;
+    if ((s = check_device_arch()) != DVDQ_OK) return s;
+    static PerDevice<int> cache;
+    if (!weight_kernel_setup(cache, quantize_weights_symmetric_kernel)) return DVDQ_ERR_CUDA;
+    quantize_weights_symmetric_kernel<<<(unsigned)N, kWeightThreads, (size_t)K * sizeof(double), (cudaStream_t)stream>>>(
+        static_cast<const __nv_bfloat16*>(W), ldw, N, (int)K, log2_of(rot_block), rot_block, static_cast<uint8_t*>(blob_out));
+    if ((s = cuda_status(cudaGetLastError())) != DVDQ_OK) return s;
+    out->magic = kBlobMagic;
+    out->version = kBlobVersion;
+    out->N = N;
+    out->K = K;
+    out->rot_block = rot_block;
+    out->k_layout = kKLayoutNatural;
+    out->blob = blob_out;
+    out->blob_bytes = (uint64_t)blob_layout(N, K).total;
+    return DVDQ_OK;
+}
+
 static dvdq_status check_gemm_args(const void* codes, const int32_t* sums, int64_t M, const dvdq_act_quant* q,
                                    const dvdq_weights* w) {
     dvdq_status s = validate_weights(w);
@@ -201,24 +255,44 @@ dvdq_status dvdq_qgemm_int32(const void* codes, const int32_t* code_sums, int64_
     return launch_qgemm(codes, nullptr, code_sums, M, *q, *w, nullptr, 0, nullptr, 0, acc_out, ldacc, (cudaStream_t)stream);
 }
 
-dvdq_status dvdq_qlinear(const void* X, int64_t M, int64_t ldx, const dvdq_act_quant* q, const dvdq_weights* w,
-                         const void* bias, int32_t act, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
-                         void* stream) {
+// Everything dvdq_qlinear and dvdq_qlinear_static check before their first launch: the union of
+// what dvdq_rotate_quantize and dvdq_qgemm check on their own.
+static dvdq_status check_qlinear_args(const void* X, int64_t M, int64_t ldx, const dvdq_act_quant* q, const dvdq_weights* w,
+                                      const void* bias, int32_t act, const void* Y, int64_t ldy) {
     dvdq_status s = validate_weights(w);
     if (s != DVDQ_OK) return s;
     if ((s = validate_act_quant(q, w->K)) != DVDQ_OK) return s;
-    if (M < 0) return DVDQ_ERR_SHAPE;
+    if (q->rot_block != w->rot_block) return DVDQ_ERR_ROT_BLOCK;
+    if (M < 0 || M > 0x7FFFFF00ll) return DVDQ_ERR_SHAPE;
+    if (ldx < w->K || ldx % 8 != 0 || ldx > 0x7FFFFFFFll || ldy < w->N || ldy % 8 != 0) return DVDQ_ERR_SHAPE;
+    if (act != 0 && act != 1) return DVDQ_ERR_UNSUPPORTED;
     if (M == 0) return DVDQ_OK;
-    if (!workspace) return DVDQ_ERR_NULL;
-    if (!aligned(workspace, 256)) return DVDQ_ERR_ALIGN;
+    if (!X || !Y) return DVDQ_ERR_NULL;
+    if (!aligned(X, 16) || !aligned(Y, 16) || (bias && !aligned(bias, 2))) return DVDQ_ERR_ALIGN;
+    return check_device_arch();
+}
+
+static dvdq_status qlinear_on_workspace(const void* X, int64_t M, int64_t ldx, const dvdq_act_quant* q, const dvdq_weights* w,
+                                        const void* bias, int32_t act, void* Y, int64_t ldy, uint8_t* ws, void* stream) {
     const WorkspacePlan p = workspace_plan(M, w->K, *q);
-    if (workspace_bytes < (size_t)p.total) return DVDQ_ERR_WORKSPACE;
-    uint8_t* ws = static_cast<uint8_t*>(workspace);
     void* codes = ws + p.codes_off;
     float* scales = reinterpret_cast<float*>(ws + p.scales_off);
     int32_t* sums = reinterpret_cast<int32_t*>(ws + p.sums_off);
-    if ((s = dvdq_rotate_quantize(X, M, w->K, ldx, q, codes, scales, sums, stream)) != DVDQ_OK) return s;
-    return dvdq_qgemm(codes, scales, sums, M, q, w, bias, act, Y, ldy, stream);
+    dvdq_status s = launch_rotate_quantize(X, M, w->K, ldx, *q, codes, scales, sums, (cudaStream_t)stream);
+    if (s != DVDQ_OK) return s;
+    return launch_qgemm(codes, scales, sums, M, *q, *w, bias, act, Y, ldy, nullptr, 0, (cudaStream_t)stream);
+}
+
+dvdq_status dvdq_qlinear(const void* X, int64_t M, int64_t ldx, const dvdq_act_quant* q, const dvdq_weights* w,
+                         const void* bias, int32_t act, void* Y, int64_t ldy, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+    dvdq_status s = check_qlinear_args(X, M, ldx, q, w, bias, act, Y, ldy);
+    if (s != DVDQ_OK) return s;
+    if (M == 0) return DVDQ_OK;
+    if (!workspace) return DVDQ_ERR_NULL;
+    if (!aligned(workspace, 256)) return DVDQ_ERR_ALIGN;
+    if (workspace_bytes < (size_t)workspace_plan(M, w->K, *q).total) return DVDQ_ERR_WORKSPACE;
+    return qlinear_on_workspace(X, M, ldx, q, w, bias, act, Y, ldy, static_cast<uint8_t*>(workspace), stream);
 }
 
 // Scratch of dvdq_qlinear_static: part of the library image, so no allocation is ever needed.
@@ -227,28 +301,16 @@ static __device__ __align__(256) uint8_t g_static_scratch[DVDQ_STATIC_SCRATCH_BY
 
 dvdq_status dvdq_qlinear_static(const void* X, int64_t M, int64_t ldx, const dvdq_act_quant* q, const dvdq_weights* w,
                                 const void* bias, int32_t act, void* Y, int64_t ldy, void* stream) {
-    constexpr int kMaxDevices = 64;
-    static void* scratch_of_device[kMaxDevices] = {nullptr};
-    dvdq_status s = validate_weights(w);
+    static PerDevice<void*> scratch_of_device;
+    dvdq_status s = check_qlinear_args(X, M, ldx, q, w, bias, act, Y, ldy);
     if (s != DVDQ_OK) return s;
-    if ((s = validate_act_quant(q, w->K)) != DVDQ_OK) return s;
-    if (M < 0) return DVDQ_ERR_SHAPE;
     if (M == 0) return DVDQ_OK;
-    const WorkspacePlan p = workspace_plan(M, w->K, *q);
-    if (p.total > (int64_t)DVDQ_STATIC_SCRATCH_BYTES) return DVDQ_ERR_WORKSPACE;
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return DVDQ_ERR_CUDA;
-    if (scratch_of_device[dev] == nullptr) {  // set-up, once per device, with that device current
-        void* ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return DVDQ_ERR_CUDA;
-        scratch_of_device[dev] = ptr;
-    }
-    uint8_t* ws = static_cast<uint8_t*>(scratch_of_device[dev]);
-    void* codes = ws + p.codes_off;
-    float* scales = reinterpret_cast<float*>(ws + p.scales_off);
-    int32_t* sums = reinterpret_cast<int32_t*>(ws + p.sums_off);
-    if ((s = dvdq_rotate_quantize(X, M, w->K, ldx, q, codes, scales, sums, stream)) != DVDQ_OK) return s;
-    return dvdq_qgemm(codes, scales, sums, M, q, w, bias, act, Y, ldy, stream);
+    if (workspace_plan(M, w->K, *q).total > (int64_t)DVDQ_STATIC_SCRATCH_BYTES) return DVDQ_ERR_WORKSPACE;
+    void** ws = scratch_of_device.get([](void*& ptr, int) {  // set-up, once per device, with that device current
+        return cudaGetSymbolAddress(&ptr, g_static_scratch) == cudaSuccess && ptr != nullptr;
+    });
+    if (!ws) return DVDQ_ERR_CUDA;
+    return qlinear_on_workspace(X, M, ldx, q, w, bias, act, Y, ldy, static_cast<uint8_t*>(*ws), stream);
 }
 
 dvdq_status dvdq_pack_act_codes(const int8_t* codes_nat, int64_t M, int64_t K, const dvdq_act_quant* q,
@@ -309,12 +371,11 @@ dvdq_status dvdq_bgr_quantize(const float* W_rot, int64_t N, int64_t K, int32_t 
     dvdq_status s = check_device_arch();
     if (s != DVDQ_OK) return s;
     const size_t smem = (size_t)K * sizeof(float);
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(bgr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 16384 * (int)sizeof(float)) != cudaSuccess)
-            return DVDQ_ERR_CUDA;
-        attr_set = true;
-    }
+    static PerDevice<int> attr_set;
+    if (!attr_set.get([](int&, int) {
+            return cudaFuncSetAttribute(bgr_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 16384 * (int)sizeof(float)) == cudaSuccess;
+        }))
+        return DVDQ_ERR_CUDA;
     bgr_kernel<<<(unsigned)N, kBgrThreads, smem, (cudaStream_t)stream>>>(W_rot, (int)K, n_steps, eps, max_iter, Wq_out,
                                                                          delta_out, zero_out);
     return cuda_status(cudaGetLastError());
@@ -373,6 +434,28 @@ dvdq_status dvdq_gbs_observe(dvdq_gbs_state* g, double l1_change, double l1_prev
     const double rel = l1_prev > 0.0 ? l1_change / l1_prev : (l1_change > 0.0 ? 1.0 : 0.0);
     g->accumulated += rel;
     return DVDQ_OK;
+}
+
+// ---- measurement and diagnostics ---------------------------------------------------------------
+
+dvdq_status dvdq_int8_mma_ceiling(int32_t iters, int64_t* ops_out, void* stream) {
+    if (iters < 1 || iters > (1 << 20)) return DVDQ_ERR_SHAPE;
+    dvdq_status s = check_device_arch();
+    if (s != DVDQ_OK) return s;
+    static PerDevice<int> cache;
+    const int pairs = resident_pairs(cache, int8_ceiling_kernel, kCeilThreads, kCeilSmem);
+    if (pairs == 0) return DVDQ_ERR_CUDA;
+    int8_ceiling_kernel<<<2 * pairs, kCeilThreads, kCeilSmem, (cudaStream_t)stream>>>(iters);
+    if (ops_out) *ops_out = (int64_t)pairs * iters * (kBK / 32) * 2ll * (2 * kBM) * kSsBN * 32;
+    return cuda_status(cudaGetLastError());
+}
+
+dvdq_status dvdq_debug_wait_timeout(uint64_t limit_ns, void* stream) {
+    if (limit_ns == 0 || limit_ns > 1000000000ull) return DVDQ_ERR_SHAPE;  // at most a second
+    dvdq_status s = check_device_arch();
+    if (s != DVDQ_OK) return s;
+    wait_timeout_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(limit_ns);
+    return cuda_status(cudaGetLastError());
 }
 
 dvdq_status dvdq_last_device_status(uint32_t* detail) {

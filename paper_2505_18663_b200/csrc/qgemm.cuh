@@ -65,8 +65,9 @@ struct GemmSmem {
     static constexpr int BN = BLK ? 128 : kBN, BNh = BN / 2;
     static constexpr int kWideW = BNh * kBK;                     // int8 weight half-tile, swizzled
     static constexpr int kWideOff = 0;                            // 1024-byte aligned tiles first
-    static constexpr int kALo = (BITS == 8) ? kBM * kPK : kBM * kPK / 2;  // A4 codes / A6 low plane (128-byte rows); A8: two tiles of 128-byte rows, one per k-block
-    static constexpr int kPStages = (BITS == 8) ? 3 : kPackedStages;  // what fits
+    static_assert(BITS == 4 || BITS == 6, "codes stored one int8 each take qgemm_ss_kernel");
+    static constexpr int kALo = kBM * kPK / 2;  // A4 codes / A6 low plane (128-byte rows)
+    static constexpr int kPStages = kPackedStages;
     static constexpr int kAHi = (BITS == 6) ? kBM * kPK / 4 : 0;  // packed high plane (64-byte rows)
     static constexpr int kPackedStage = kALo + kAHi;              // activation codes of two k-blocks
     static constexpr int kPackedOff = kWideOff + kWideStages * kWideW;
@@ -118,9 +119,10 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     const int num_tiles = num_m * num_n;
     const int KB2 = (K + kPK - 1) / kPK;  // activation loads per tile; a k-block past K reads zeros
     const int KB = 2 * KB2;
-    // one accumulator per tile, or (block-wise scales) one per tile and block of 1024 codes
-    const int NG = BLK ? K / kScaleBlock : 1;
-    const int KBG = BLK ? kScaleBlock / kBK : KB;  // k-blocks per accumulator
+    // one accumulator per tile, or (block-wise scales) one per tile and scale group: spr groups of
+    // 128, 256 or 1024 codes per token, i.e. 1, 2 or 8 k-blocks per accumulator (K is a multiple of 256)
+    const int NG = BLK ? spr : 1;
+    const int KBG = BLK ? KB / spr : KB;  // k-blocks per accumulator
 
     const uint32_t bar0 = sbase + S::kBarOff;
     auto pk_full = [&](int s) { return bar0 + 8u * s; };
@@ -170,12 +172,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     if (!mbar_wait(pk_empty(st), ph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
                     const uint32_t dst = sbase + S::kPackedOff + st * S::kPackedStage;
                     mbar_arrive_expect_tx(pk_full(st), S::kPackedStage);
-                    if (BITS == 8) {
-                        tma_load_2d(dst, &tmA, pk_full(st), sb * kPK, m0);
-                        tma_load_2d(dst + S::kALo / 2, &tmA, pk_full(st), sb * kPK + kBK, m0);
-                    } else {
-                        tma_load_2d(dst, &tmA, pk_full(st), sb * (kPK / 2), m0);
-                    }
+                    tma_load_2d(dst, &tmA, pk_full(st), sb * (kPK / 2), m0);
                     if (BITS == 6) tma_load_2d(dst + S::kALo, &tmAhi, pk_full(st), sb * (kPK / 4), m0);
                     ++issued;
                     if (++st == S::kPStages) { st = 0; ph ^= 1u; }
@@ -210,38 +207,55 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         // The whole warp walks the loop (warp-uniform control flow); one elected lane issues.
         if (rank == 0) {
             constexpr uint32_t idesc = umma_idesc_s8s8s32(2 * kBM, BN);
-            uint32_t st = 0, ph = 0, lt = 0;
+            uint32_t st = 0, ph = 0, lt = 0;  // lt: accumulators started so far
+            uint32_t acc = 0;                  // the accumulator in use (0 or 1)
             bool ok = true;
-            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs)
-            for (int g = 0; ok && g < NG; ++g, ++lt) {
-                const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
-                if (!mbar_wait_warp(acc_empty(a), aph ^ 1u, abort_flag, kWaitAccEmpty)) { ok = false; break; }
+            // Starts the next accumulator once the epilogue has drained its previous contents.
+            auto acquire = [&]() {
+                acc = lt & 1u;
+                if (!mbar_wait_warp(acc_empty(acc), ((lt >> 1) & 1u) ^ 1u, abort_flag, kWaitAccEmpty)) ok = false;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + a * BN;
+                ++lt;
+            };
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 // Two k-blocks per trip (KB is even, and so is kWideStages): the tensor core's queue
                 // is short, so every cycle this warp spends between two issues is a bubble in the
-                // MMA stream; pairing halves the waits, votes and bookkeeping per k-block.
-                for (int kb = 0; kb < KBG; kb += 2) {
+                // MMA stream; pairing halves the waits, votes and bookkeeping per k-block.  An
+                // accumulator covers KBG k-blocks (a power of two, or the whole of K): with KBG = 1
+                // the two blocks of a trip go to different accumulators.
+                int kin = 0;  // k-blocks issued into the accumulator in use
+                for (int kb = 0; ok && kb < KB; kb += 2) {
+                    uint32_t acc_h[2];
+                    bool first_h[2], last_h[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        first_h[h] = kin == 0;
+                        if (first_h[h]) acquire();
+                        acc_h[h] = acc;
+                        last_h[h] = ++kin == KBG;
+                        if (last_h[h]) kin = 0;
+                    }
+                    if (!ok) break;
                     if (!mbar_wait_warp(wd_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     if (!mbar_wait_warp(wd_full(st + 1), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     tc_fence_after();
                     if (elect_one()) {
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
+                            const uint32_t d_tmem = tmem_base + acc_h[h] * BN;
                             const uint32_t a_tmem = tmem_base + kTmemACol + (st + h) * kAColsPerStage;
                             const uint64_t bdesc = umma_desc_sw128_kmajor(sbase + S::kWideOff + (st + h) * S::kWideW);
 #pragma unroll
                             for (int k = 0; k < kBK / 32; ++k)  // +32 int8 along K = +8 columns of A, +2 in B's 16-byte address field
-                                tc_mma_i8_ts_pair(d_tmem, a_tmem + 8u * k, bdesc + 2u * k, idesc, (kb | h | k) != 0 ? 1u : 0u);
+                                tc_mma_i8_ts_pair(d_tmem, a_tmem + 8u * k, bdesc + 2u * k, idesc, (first_h[h] && k == 0) ? 0u : 1u);
                             tc_commit_pair(wd_empty(st + h), 3);
+                            if (last_h[h]) tc_commit_pair(acc_full(acc_h[h]), 3);
                         }
                     }
                     __syncwarp();
                     st += 2;
                     if (st == kWideStages) { st = 0; ph ^= 1u; }
                 }
-                if (ok && elect_one()) tc_commit_pair(acc_full(a), 3);
-                __syncwarp();
             }
             // nothing issued by this warp may still be running when the pair leaves
             if (elect_one()) tc_commit_pair(drain_bar, 1);
@@ -257,7 +271,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const uint32_t c_zc = c_delta + BN * 4;    // (z_n - 8) as a float: exact, |.| <= 8
         const uint32_t c_bias = c_zc + BN * 4;
         const uint32_t stg0 = sbase + S::kStageOutOff + ew * S::kStageOutPerWarp;
-        constexpr int kShift = (BITS == 4) ? 8 : (BITS == 6) ? 6 : 4;  // log2 of (A factor 16 / 4 / 1) x (W factor 16)
+        constexpr int kShift = (BITS == 4) ? 8 : 6;  // log2 of (A factor 16 or 4) x (W factor 16)
         if (!RAW && lane == 0) tma_prefetch_desc(&tmY);
         if constexpr (BLK) {
             // Block-wise scales: every block of 1024 codes has its own int32 accumulator (the two
@@ -484,6 +498,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         uint32_t j = 0;  // k-blocks seen so far; this warp takes those with j % kUnpackGroups == grp
         bool ok = true;
+        const uint32_t rt_zero = runtime_zero();
         for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
             for (int kb = 0; kb < KB; ++kb) {
                 const uint32_t jj = j++;
@@ -496,27 +511,21 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 const uint32_t prow = pk + row * (kPK / 2);
                 uint32_t r[32];  // r[2i] / r[2i+1]: even / odd codes of packed word i, the K order the weights use too
                 uint32_t h[8];
+                uint32_t loaded = 0u;
                 if (BITS == 6) {
                     const uint32_t hrow = pk + S::kALo + row * (kPK / 4);
 #pragma unroll
                     for (int c = 0; c < 2; ++c) {
                         const uint4 p = lds128(hrow + (((2u * grp + (uint32_t)c) ^ sw_hi) << 4));
                         h[4 * c] = p.x; h[4 * c + 1] = p.y; h[4 * c + 2] = p.z; h[4 * c + 3] = p.w;
-                    }
-                }
-                if (BITS == 8) {
-                    // int8 codes, already in the even/odd order of the weight operand: no widening
-                    const uint32_t prow8 = pk + grp * (S::kALo / 2) + row * kBK;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const uint4 p = lds128(prow8 + (((uint32_t)c ^ sw_lo) << 4));
-                        r[4 * c] = p.x; r[4 * c + 1] = p.y; r[4 * c + 2] = p.z; r[4 * c + 3] = p.w;
+                        loaded ^= p.w;
                     }
                 }
 #pragma unroll
-                for (int c = 0; c < (BITS == 8 ? 0 : 4); ++c) {
+                for (int c = 0; c < 4; ++c) {
                     const uint4 p = lds128(prow + (((4u * grp + (uint32_t)c) ^ sw_lo) << 4));
                     const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+                    loaded ^= p.w;
 #pragma unroll
                     for (int jw = 0; jw < 4; ++jw) {
                         const int i = 4 * c + jw;
@@ -532,9 +541,10 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     }
                 }
                 // the codes are widened in registers before the stage of tensor memory is known to be free
+                loaded &= rt_zero;
                 fence_loads_done();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(pk_empty(pst));
+                if (lane == 0) mbar_arrive_after_loads(pk_empty(pst), loaded);
                 if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
                 tc_fence_after();
                 tmem_st_32x32(tmem_base + kTmemACol + wst * kAColsPerStage + lane_addr, r);
@@ -550,6 +560,7 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
         const int u = (threadIdx.x - kFirstWWarp * 32) & 127;  // thread of its group of four warps
         uint32_t j = 0;
         bool ok = true;
+        const uint32_t rt_zero = runtime_zero();
         for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
             for (int kb = 0; kb < KB; ++kb) {
             const uint32_t jj = j++;
@@ -563,17 +574,20 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             // wide stage is known to be free
             constexpr int kPieces = (BNh * 4) / 128;
             uint32_t e[kPieces][4], o[kPieces][4];
+            uint32_t loaded = 0u;
 #pragma unroll
             for (int it = 0; it < kPieces; ++it) {
                 const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
                 const uint4 p = lds128(pw + row * (kBK / 2) + ck * 16);
                 const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+                loaded ^= p.w;
 #pragma unroll
                 for (int jw = 0; jw < 4; ++jw) { e[it][jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[it][jw] = w[jw] & 0xF0F0F0F0u; }
             }
+            loaded &= rt_zero;
             fence_loads_done();
             __syncwarp();
-            if (lane == 0) mbar_arrive(wp_empty(pst));  // the packed rows are in registers
+            if (lane == 0) mbar_arrive_after_loads(wp_empty(pst), loaded);  // the packed rows are in registers
             if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
             tc_fence_after();
 #pragma unroll
@@ -644,6 +658,31 @@ inline bool make_byte_map(CUtensorMap* tm, const void* base, uint64_t row_len, u
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// One-time set-up of a pair kernel on the current device: the opt-in to its dynamic shared memory and
+// the number of CTA pairs the device keeps resident at once (one CTA per SM).  0 on failure.
+template <typename Kern>
+static int resident_pairs(PerDevice<int>& cache, Kern kern, int threads, int smem_bytes) {
+    int* mp = cache.get([&](int& max_pairs, int dev) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess) return false;
+        int sm_count = 0;
+        if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(sm_count & ~1), 1, 1);
+        cfg.blockDim = dim3((unsigned)threads, 1, 1);
+        cfg.dynamicSmemBytes = (size_t)smem_bytes;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) != cudaSuccess || clusters < 1) return false;
+        max_pairs = clusters < sm_count / 2 ? clusters : sm_count / 2;
+        return true;
+    });
+    return mp ? *mp : 0;
+}
+
 template <int BITS, bool RAW, bool BLK>
 static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                   const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
@@ -654,7 +693,7 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
     const uint64_t pitch = (uint64_t)act_row_bytes(K, BITS);
     CUtensorMap tmA, tmAhi, tmW, tmY;
-    if (!make_byte_map(&tmA, codes, (uint64_t)(BITS == 8 ? K : K / 2), (uint64_t)M, pitch, kPK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_128B))
+    if (!make_byte_map(&tmA, codes, (uint64_t)K / 2, (uint64_t)M, pitch, kPK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_128B))
         return DVDQ_ERR_CUDA;
     if (BITS == 6) {
         if (!make_byte_map(&tmAhi, static_cast<const uint8_t*>(codes) + K / 2, (uint64_t)K / 4, (uint64_t)M, pitch,
@@ -674,26 +713,9 @@ static dvdq_status launch_qgemm_t(const void* codes, const float* scales, const 
     }
 
     auto kern = qgemm_kernel<BITS, RAW, BLK>;
-    static int max_pairs = 0;
-    if (max_pairs == 0) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) return DVDQ_ERR_CUDA;
-        int dev = 0, sm_count = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return DVDQ_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DVDQ_ERR_CUDA;
-        // how many CTA pairs the device can keep resident at once (one CTA per SM)
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(sm_count & ~1), 1, 1);
-        cfg.blockDim = dim3(kGemmThreads, 1, 1);
-        cfg.dynamicSmemBytes = S::kTotal;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        int clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) != cudaSuccess || clusters < 1) return DVDQ_ERR_CUDA;
-        max_pairs = clusters < sm_count / 2 ? clusters : sm_count / 2;
-    }
+    static PerDevice<int> cache;
+    const int max_pairs = resident_pairs(cache, kern, kGemmThreads, S::kTotal);
+    if (max_pairs == 0) return DVDQ_ERR_CUDA;
     const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + S::BN - 1) / S::BN);
     const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
     kern<<<2 * pairs, kGemmThreads, S::kTotal, st>>>(tmA, tmAhi, tmW, tmY, scales, sums,
@@ -736,7 +758,6 @@ inline dvdq_status launch_qgemm(const void* codes, const float* scales, const in
     }
     DVDQ_GEMM_CASE(4)
     DVDQ_GEMM_CASE(6)
-    DVDQ_GEMM_CASE(8)
 #undef DVDQ_GEMM_CASE
     return DVDQ_ERR_BITS;
 }

@@ -96,9 +96,10 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int num_n = (N + BN - 1) / BN, num_m = (M + 2 * kBM - 1) / (2 * kBM);
     const int num_tiles = num_m * num_n;
     const int KB = 2 * ((K + 2 * kBK - 1) / (2 * kBK));  // even; a k-block past K reads zeros
-    // one accumulator per tile, or (block-wise scales) one per tile and block of 1024 codes
-    const int NG = BLK ? K / kScaleBlock : 1;
-    const int KBG = BLK ? kScaleBlock / kBK : KB;  // k-blocks per accumulator
+    // one accumulator per tile, or (block-wise scales) one per tile and scale group: spr groups of
+    // 128, 256 or 1024 codes per token, i.e. 1, 2 or 8 k-blocks per accumulator (K is a multiple of 256)
+    const int NG = BLK ? spr : 1;
+    const int KBG = BLK ? KB / spr : KB;  // k-blocks per accumulator
 
     const uint32_t bar0 = sbase + S::kBarOff;
     auto a_full = [&](int s) { return bar0 + 8u * s; };                          // this CTA's TMA copy of the stage
@@ -191,15 +192,32 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (rank == 0) {
             constexpr uint32_t idesc = umma_idesc_s8s8s32(2 * kBM, BN);
-            uint32_t st = 0, ph = 0, sa = 0, pa = 0, lt = 0;
+            uint32_t st = 0, ph = 0, sa = 0, pa = 0, lt = 0;  // lt: accumulators started so far
+            uint32_t acc = 0;                                  // the accumulator in use (0 or 1)
             bool ok = true;
-            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs)
-            for (int g = 0; ok && g < NG; ++g, ++lt) {
-                const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
-                if (!mbar_wait_warp(acc_empty(a), aph ^ 1u, abort_flag, kWaitAccEmpty)) { ok = false; break; }
+            // Starts the next accumulator once the epilogue has drained its previous contents.
+            auto acquire = [&]() {
+                acc = lt & 1u;
+                if (!mbar_wait_warp(acc_empty(acc), ((lt >> 1) & 1u) ^ 1u, abort_flag, kWaitAccEmpty)) ok = false;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + a * BN;
-                for (int kb = 0; kb < KBG; kb += 2) {
+                ++lt;
+            };
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                // Two k-blocks per trip.  An accumulator covers KBG k-blocks (a power of two, or the
+                // whole of K): with KBG = 1 the two blocks of a trip go to different accumulators.
+                int kin = 0;  // k-blocks issued into the accumulator in use
+                for (int kb = 0; ok && kb < KB; kb += 2) {
+                    uint32_t acc_h[2];
+                    bool first_h[2], last_h[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        first_h[h] = kin == 0;
+                        if (first_h[h]) acquire();
+                        acc_h[h] = acc;
+                        last_h[h] = ++kin == KBG;
+                        if (last_h[h]) kin = 0;
+                    }
+                    if (!ok) break;
                     // the activation ring may have an odd number of stages: its second stage of the trip can wrap
                     const uint32_t sa1 = sa + 1 == kSsAStages ? 0u : sa + 1, pa1 = sa + 1 == kSsAStages ? pa ^ 1u : pa;
                     if (!mbar_wait_warp(a_ready(sa), pa, abort_flag, kWaitPackedFull)) { ok = false; break; }
@@ -210,13 +228,15 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (elect_one()) {
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
+                            const uint32_t d_tmem = tmem_base + acc_h[h] * BN;
                             const uint64_t adesc = umma_desc_sw128_kmajor(sbase + S::kAOff + (h ? sa1 : sa) * S::kA);
                             const uint64_t bdesc = umma_desc_sw128_kmajor(sbase + S::kWOff + (st + h) * S::kW);
 #pragma unroll
                             for (int k = 0; k < kBK / 32; ++k)  // +32 int8 along K = +2 in the 16-byte address field
-                                tc_mma_i8_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | h | k) != 0 ? 1u : 0u);
+                                tc_mma_i8_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (first_h[h] && k == 0) ? 0u : 1u);
                             tc_commit_pair(ops_empty(st + h), 3);
                             tc_commit_pair(a_empty(h ? sa1 : sa), 3);
+                            if (last_h[h]) tc_commit_pair(acc_full(acc_h[h]), 3);
                         }
                     }
                     __syncwarp();
@@ -226,8 +246,6 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     pa = pa1;
                     if (sa == kSsAStages) { sa = 0; pa ^= 1u; }
                 }
-                if (ok && elect_one()) tc_commit_pair(acc_full(a), 3);
-                __syncwarp();
             }
             if (elect_one()) tc_commit_pair(drain_bar, 1);
             __syncwarp();
@@ -468,6 +486,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int u = (threadIdx.x - kSsFirstWWarp * 32) & 127;  // thread of its group of four warps
         uint32_t j = 0;
         bool ok = true;
+        const uint32_t rt_zero = runtime_zero();
         for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
             for (int kb = 0; kb < KB; ++kb) {
             const uint32_t jj = j++;
@@ -481,17 +500,20 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             // wide stage is known to be free
             constexpr int kPieces = (BNh * 4) / 128;
             uint32_t e[kPieces][4], o[kPieces][4];
+            uint32_t loaded = 0u;
 #pragma unroll
             for (int it = 0; it < kPieces; ++it) {
                 const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
                 const uint4 p = lds128(pw + row * (kBK / 2) + ck * 16);
                 const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+                loaded ^= p.w;
 #pragma unroll
                 for (int jw = 0; jw < 4; ++jw) { e[it][jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[it][jw] = w[jw] & 0xF0F0F0F0u; }
             }
+            loaded &= rt_zero;
             fence_loads_done();
             __syncwarp();
-            if (lane == 0) mbar_arrive(wp_empty(pst));  // the packed rows are in registers
+            if (lane == 0) mbar_arrive_after_loads(wp_empty(pst), loaded);  // the packed rows are in registers
             if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
             tc_fence_after();
 #pragma unroll
@@ -565,25 +587,9 @@ static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, con
     }
     constexpr int kThreads = (EW == 8 ? kSsFirstEpilogueWarp2 + 4 : kSsFirstEpilogueWarp2) * 32;
     auto kern = qgemm_ss_kernel<RAW, EW, BLK>;
-    static int max_pairs = 0;
-    if (max_pairs == 0) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, S::kTotal) != cudaSuccess) return DVDQ_ERR_CUDA;
-        int dev = 0, sm_count = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return DVDQ_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DVDQ_ERR_CUDA;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)(sm_count & ~1), 1, 1);
-        cfg.blockDim = dim3(kThreads, 1, 1);
-        cfg.dynamicSmemBytes = S::kTotal;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        int clusters = 0;
-        if (cudaOccupancyMaxActiveClusters(&clusters, kern, &cfg) != cudaSuccess || clusters < 1) return DVDQ_ERR_CUDA;
-        max_pairs = clusters < sm_count / 2 ? clusters : sm_count / 2;
-    }
+    static PerDevice<int> cache;
+    const int max_pairs = resident_pairs(cache, kern, kThreads, S::kTotal);
+    if (max_pairs == 0) return DVDQ_ERR_CUDA;
     const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + S::BN - 1) / S::BN);
     const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
     kern<<<2 * pairs, kThreads, S::kTotal, st>>>(tmA, tmW, tmY, scales, sums,

@@ -23,6 +23,14 @@
 // the stages of the upper bits; no rotation (B = 0) runs the same data path with the identity
 // in place of H_16.  The 1/sqrt(B) normalisation is folded into the scale.
 //
+// Blocks of 2048 or 4096 channels span two or four warps: after stage C the warps of a block
+// exchange their spans through shared memory once and each forms its own signed sum of the two
+// or four spans (the butterflies of index bits 10 and 11).
+//
+// Scale granularity: one scale per token (the token's warps meet once for the absmax), per
+// 1024-channel span (the warp's own absmax), or per 256 / 128 channels (SUB: the absmax of the
+// eight lanes that hold the group, for one or for each half of their registers).
+//
 // Rounding: c = rne(x~ * (qmax / absmax)) as one fused multiply-add onto 1.5 * 2^23, which
 // leaves the two's-complement code in the low mantissa bits.  (B = 0 divides instead.)
 #pragma once
@@ -58,15 +66,18 @@ __device__ __forceinline__ uint32_t stage_a_entry(int m, int s) {
 // same way and written out after the next iteration's barrier.  The slots rotate over three sets:
 // a warp's whole iteration is a chain of dependent steps, so the exchange is kept as short as
 // it can be (an atomic, the barrier, one broadcast load).
-template <int LOG2B, int BITS, bool FULL>
+template <int LOG2B, int BITS, bool FULL, bool SUB>
 __global__ void __maxnreg__(80)  // two CTAs of 12 warps per SM
 rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
           uint8_t* __restrict__ codes, float* __restrict__ scales, int32_t* __restrict__ sums,
-          int spans, int tokens_per_cta, int num_groups, int blockwise, int code_bits) {
+          int spans, int tokens_per_cta, int num_groups, int scale_group, int code_bits) {
     extern __shared__ float4 s_turn[];  // 256 float4 per warp
     __shared__ unsigned s_max[3][kRqMaxWarps];  // [slot set][token of the CTA]: bits of the token absmax
     __shared__ int s_sum[3][kRqMaxWarps];       // sum of the token's codes
     constexpr bool kRot = LOG2B > 0;
+    constexpr int kLog2Span = LOG2B > 10 ? 10 : LOG2B;  // butterflies a warp does on its own span
+    constexpr int kCross = 1 << (LOG2B > 10 ? LOG2B - 10 : 0);  // spans per rotation block
+    const int blockwise = scale_group != 0;
     // BITS is the width a code is STORED in; the quantizer's own width may be smaller (codes kept in bytes)
     const float qmax = (float)((1 << (code_bits - 1)) - 1);
     constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: ulp 1, so the fma rounds to an integer
@@ -183,7 +194,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
             for (int p = 0; p < 2; ++p)
 #pragma unroll
                 for (int h = 0; h < 2; ++h) P[c][p][h] = f2_pack(acc[c][p][2 * h], acc[c][p][2 * h + 1]);
-        if (LOG2B > 8) {
+        if (kLog2Span > 8) {
 #pragma unroll
             for (int c = 0; c < 4; c += 2)
 #pragma unroll
@@ -191,7 +202,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
 #pragma unroll
                     for (int h = 0; h < 2; ++h) f2_butterfly(P[c][p][h], P[c + 1][p][h]);
         }
-        if (LOG2B > 9) {
+        if (kLog2Span > 9) {
 #pragma unroll
             for (int c = 0; c < 2; ++c)
 #pragma unroll
@@ -232,7 +243,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
             }
 
         // ---- stage C: bits 6 and 7
-        if (LOG2B > 6) {
+        if (kLog2Span > 6) {
 #pragma unroll
             for (int j = 0; j < 4; j += 2)
 #pragma unroll
@@ -240,7 +251,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
 #pragma unroll
                     for (int h = 0; h < 2; ++h) f2_butterfly(W[j][i0][h], W[j + 1][i0][h]);
         }
-        if (LOG2B > 7) {
+        if (kLog2Span > 7) {
 #pragma unroll
             for (int j = 0; j < 2; ++j)
 #pragma unroll
@@ -249,10 +260,46 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
                     for (int h = 0; h < 2; ++h) f2_butterfly(W[j][i0][h], W[j + 2][i0][h]);
         }
 
+        // ---- index bits 10 (and 11): the kCross warps of a rotation block park their spans in
+        // their turn buffers, meet, and each takes its signed sum over the block's spans
+        if (kCross > 1) {
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int i0 = 0; i0 < 2; ++i0) {
+                    float a, b, c, d;
+                    f2_unpack(W[j][i0][0], a, b);
+                    f2_unpack(W[j][i0][1], c, d);
+                    turn[(2 * j + i0) * 32 + lane] = make_float4(a, b, c, d);
+                    W[j][i0][0] = W[j][i0][1] = f2_pack(0.f, 0.f);
+                }
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
+            const int me = sp & (kCross - 1);
+#pragma unroll
+            for (int o = 0; o < kCross; ++o) {
+                const float sg = (__popc(me & o) & 1) ? -1.f : 1.f;  // entry (me, o) of H_2 or H_4
+                const uint64_t sg2 = f2_pack(sg, sg);
+                const float4* theirs = s_turn + (warp - me + o) * 256;
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                    for (int i0 = 0; i0 < 2; ++i0) {
+                        const float4 f = theirs[(2 * j + i0) * 32 + lane];
+                        W[j][i0][0] = f2_fma(f2_pack(f.x, f.y), sg2, W[j][i0][0]);
+                        W[j][i0][1] = f2_fma(f2_pack(f.z, f.w), sg2, W[j][i0][1]);
+                    }
+            }
+            // without the absmax rendezvous below nothing else keeps a fast warp from refilling its
+            // turn buffer while a partner still reads it
+            if (!team) asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
+        }
+
         // W[j][i0][h] = channels e and e + 2 of word j, e = i0 + 4 * h; the word covers channels
         // (lane >> 3) * 256 + j * 64 + (lane & 7) * 8 + 0..7 of the span
-        // ---- per-token absmax (of the un-normalised transform)
-        float amax = 0.f;
+        // ---- absmax (of the un-normalised transform) of the scale's reach: am[jh] covers this
+        // lane's words j = 2 jh, 2 jh + 1
+        float am[2] = {0.f, 0.f};
 #pragma unroll
         for (int j = 0; j < 4; ++j)
 #pragma unroll
@@ -261,24 +308,34 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
                 for (int h = 0; h < 2; ++h) {
                     float lo, hi;
                     f2_unpack(W[j][i0][h], lo, hi);
-                    amax = fmaxf(amax, fmaxf(fabsf(lo), fabsf(hi)));
+                    am[j >> 1] = fmaxf(am[j >> 1], fmaxf(fabsf(lo), fabsf(hi)));
                 }
-        // non-negative floats order like their bit patterns: one REDUX instead of five shuffles
-        amax = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(amax)));
-        // Block-wise scales (one per token and per 1024-channel span): the warp's own absmax is
-        // the scale's, nothing is shared between warps.  Per-token scale: the token's warps meet.
-        if (team) {
-            if (lane == 0) atomicMax(&s_max[cur][tl], __float_as_uint(amax));
-            // only the warps of this token meet: named barrier 1 + tl, spans * 32 threads
-            asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
-            amax = __uint_as_float(s_max[cur][tl]);
+        const unsigned octet = 0xFFu << (lane & 24);  // the eight lanes that hold one 256-channel group
+        if (SUB) {
+            // non-negative floats order like their bit patterns: one REDUX instead of shuffles
+            if (scale_group == 256) am[0] = am[1] = fmaxf(am[0], am[1]);
+            am[0] = __uint_as_float(__reduce_max_sync(octet, __float_as_uint(am[0])));
+            am[1] = scale_group == 256 ? am[0] : __uint_as_float(__reduce_max_sync(octet, __float_as_uint(am[1])));
+        } else {
+            float amax = __uint_as_float(__reduce_max_sync(0xFFFFFFFFu, __float_as_uint(fmaxf(am[0], am[1]))));
+            // One scale per 1024-channel span: the warp's own absmax is the scale's, nothing is shared
+            // between warps.  Per-token scale: the token's warps meet.
+            if (team) {
+                if (lane == 0) atomicMax(&s_max[cur][tl], __float_as_uint(amax));
+                // only the warps of this token meet: named barrier 1 + tl, spans * 32 threads
+                asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
+                amax = __uint_as_float(s_max[cur][tl]);
+            }
+            am[0] = am[1] = amax;
         }
-        const float inv = amax > 0.f ? qmax / amax : 0.f;
-        const uint64_t inv2 = f2_pack(inv, inv), magic2 = f2_pack(kMagic, kMagic);
+        const float amax = am[0];
+        const float inv0 = am[0] > 0.f ? qmax / am[0] : 0.f, inv1 = am[1] > 0.f ? qmax / am[1] : 0.f;
+        const uint64_t invs[2] = {f2_pack(inv0, inv0), f2_pack(inv1, inv1)};
+        const uint64_t magic2 = f2_pack(kMagic, kMagic);
 
         // ---- quantize, sum, pack, store
         uint8_t* crow = codes + (int64_t)token * row_bytes;
-        int lsum = 0;
+        int lsum = 0, lsum_lo = 0;  // SUB: lsum_lo keeps the words j = 0, 1
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t b[8];
@@ -288,13 +345,14 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
                 for (int h = 0; h < 2; ++h) {
                     float lo, hi;
                     if (kRot) {
-                        f2_unpack(f2_fma(W[j][i0][h], inv2, magic2), lo, hi);
+                        f2_unpack(f2_fma(W[j][i0][h], invs[SUB ? (j >> 1) : 0], magic2), lo, hi);
                     } else {
                         // Without a rotation x~ is a bf16 value, x~ * qmax is exact and exact half-way
                         // quotients are common: take the correctly rounded quotient so that they survive.
                         f2_unpack(W[j][i0][h], lo, hi);
-                        lo = (amax > 0.f ? __fdiv_rn(lo * qmax, amax) : 0.f) + kMagic;
-                        hi = (amax > 0.f ? __fdiv_rn(hi * qmax, amax) : 0.f) + kMagic;
+                        const float aj = am[SUB ? (j >> 1) : 0];
+                        lo = (aj > 0.f ? __fdiv_rn(lo * qmax, aj) : 0.f) + kMagic;
+                        hi = (aj > 0.f ? __fdiv_rn(hi * qmax, aj) : 0.f) + kMagic;
                     }
                     b[i0 + 4 * h] = __float_as_uint(lo);
                     b[i0 + 4 * h + 2] = __float_as_uint(hi);
@@ -304,6 +362,10 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
             const uint32_t O = __byte_perm(__byte_perm(b[1], b[3], 0x0040), __byte_perm(b[5], b[7], 0x0040), 0x5410);
             lsum = __dp4a((int)E, 0x01010101, lsum);
             lsum = __dp4a((int)O, 0x01010101, lsum);
+            if (SUB && j == 1) {
+                lsum_lo = lsum;
+                lsum = 0;
+            }
             const bool ok = FULL || (st_ok >> j & 1u);
             if (BITS == 8) {
                 // 8-bit codes: each group of 8 channels is stored as the word of its even channels
@@ -321,6 +383,26 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
                 hi |= __shfl_xor_sync(0xFFFFFFFFu, hi, 1);
                 if (ok && ((j ^ lane) & 1) == 0) *reinterpret_cast<uint32_t*>(crow + st_h0 + 16 * j) = hi;
             }
+        }
+        if (SUB) {
+            // groups of 256 channels = this octet's 32 words; groups of 128 = its words j = 0, 1 and j = 2, 3
+            const int per_span = kRqSpan / scale_group;  // 4 or 8
+            const int gps = K / scale_group;
+            int s0 = scale_group == 256 ? lsum_lo + lsum : lsum_lo, s1 = lsum;
+            s0 = __reduce_add_sync(octet, s0);
+            if (scale_group != 256) s1 = __reduce_add_sync(octet, s1);
+            if ((lane & 7) == 0) {
+                const int g0 = sp * per_span + (lane >> 3) * (per_span >> 2);
+                if (FULL || g0 < gps) {
+                    scales[(int64_t)token * gps + g0] = (am[0] * rs) / qmax;
+                    sums[(int64_t)token * gps + g0] = s0;
+                }
+                if (scale_group != 256 && (FULL || g0 + 1 < gps)) {
+                    scales[(int64_t)token * gps + g0 + 1] = (am[1] * rs) / qmax;
+                    sums[(int64_t)token * gps + g0 + 1] = s1;
+                }
+            }
+            continue;
         }
         lsum = __reduce_add_sync(0xFFFFFFFFu, lsum);
         if (blockwise) {
@@ -360,53 +442,55 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
     }
 }
 
-template <int LOG2B, int BITS, bool FULL>
+template <int LOG2B, int BITS, bool FULL, bool SUB>
 static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t ldx, void* codes, float* scales,
-                                    int32_t* sums, int blockwise, int code_bits, cudaStream_t st) {
+                                    int32_t* sums, int scale_group, int code_bits, cudaStream_t st) {
     const int spans = (int)((K + kRqSpan - 1) / kRqSpan);
     if (spans > kRqMaxWarps) return DVDQ_ERR_SHAPE;
     int tpc = 12 / spans;  // at most 12 tokens per CTA: named barriers 1..12
     if (tpc < 1) tpc = 1;
+    constexpr int kCross = LOG2B > 10 ? (1 << (LOG2B > 10 ? LOG2B - 10 : 0)) : 1;  // spans per rotation block
+    if (spans % kCross != 0) return DVDQ_ERR_ROT_BLOCK;
     const int warps = spans * tpc;
     const int threads = warps * 32;
     const size_t smem = (size_t)warps * 256 * sizeof(float4);
     const int64_t groups = (M + tpc - 1) / tpc;
     if (M > 0x7FFFFF00ll || ldx > 0x7FFFFFFFll || groups * tpc > 0x7FFFFFFFll) return DVDQ_ERR_SHAPE;
-    auto kern = rq_kernel<LOG2B, BITS, FULL>;
-    static bool attr_set = false;
-    static int sm_count = 0;
-    static int blocks_per_sm[kRqMaxWarps + 1] = {0};
-    if (!attr_set) {
+    auto kern = rq_kernel<LOG2B, BITS, FULL, SUB>;
+    struct Setup {
+        int sm_count;
+        int blocks_per_sm[kRqMaxWarps + 1];
+    };
+    static PerDevice<Setup> cache;
+    Setup* su = cache.get([&](Setup& s, int dev) {
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  kRqMaxWarps * 256 * (int)sizeof(float4)) != cudaSuccess)
-            return DVDQ_ERR_CUDA;
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess) return DVDQ_ERR_CUDA;
-        if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return DVDQ_ERR_CUDA;
-        attr_set = true;
-    }
-    if (blocks_per_sm[warps] == 0) {
+            return false;
+        return cudaDeviceGetAttribute(&s.sm_count, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess;
+    });
+    if (!su) return DVDQ_ERR_CUDA;
+    if (su->blocks_per_sm[warps] == 0) {
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, threads, smem) != cudaSuccess || n < 1) return DVDQ_ERR_CUDA;
-        blocks_per_sm[warps] = n;
+        su->blocks_per_sm[warps] = n;
     }
-    const int64_t resident = (int64_t)sm_count * blocks_per_sm[warps];
+    const int64_t resident = (int64_t)su->sm_count * su->blocks_per_sm[warps];
     const unsigned grid = (unsigned)(groups < resident ? groups : resident);
     kern<<<grid, threads, smem, st>>>((const __nv_bfloat16*)X, (int)M, (int)K, (int)ldx, (uint8_t*)codes, scales, sums, spans, tpc,
-                                      (int)groups, blockwise, code_bits);
+                                      (int)groups, scale_group, code_bits);
     return cuda_status(cudaGetLastError());
 }
 
-template <int BITS>
+template <int BITS, bool SUB>
 static dvdq_status launch_rq_bits(const void* X, int64_t M, int64_t K, int64_t ldx, int rot_block, void* codes,
-                                  float* scales, int32_t* sums, int blockwise, int code_bits, cudaStream_t st) {
+                                  float* scales, int32_t* sums, int scale_group, int code_bits, cudaStream_t st) {
     int log2b = 0;
     while ((1 << log2b) < rot_block) ++log2b;
     const bool full = K % kRqSpan == 0;
 #define DVDQ_RQ_CASE(L)                                                                              \
     case L:                                                                                          \
-        return full ? launch_rq_kernel<L, BITS, true>(X, M, K, ldx, codes, scales, sums, blockwise, code_bits, st)         \
-                    : launch_rq_kernel<L, BITS, false>(X, M, K, ldx, codes, scales, sums, blockwise, code_bits, st);
+        return full ? launch_rq_kernel<L, BITS, true, SUB>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st)  \
+                    : launch_rq_kernel<L, BITS, false, SUB>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st);
     switch (log2b) {
         DVDQ_RQ_CASE(0)
         DVDQ_RQ_CASE(6)
@@ -414,6 +498,10 @@ static dvdq_status launch_rq_bits(const void* X, int64_t M, int64_t K, int64_t l
         DVDQ_RQ_CASE(8)
         DVDQ_RQ_CASE(9)
         DVDQ_RQ_CASE(10)
+        case 11:  // blocks of 2048 and 4096 channels are whole spans: K is a multiple of 1024
+            return full ? launch_rq_kernel<11, BITS, true, SUB>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st) : DVDQ_ERR_ROT_BLOCK;
+        case 12:
+            return full ? launch_rq_kernel<12, BITS, true, SUB>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st) : DVDQ_ERR_ROT_BLOCK;
         default:
             return DVDQ_ERR_ROT_BLOCK;
     }
@@ -424,9 +512,16 @@ inline dvdq_status launch_rotate_quantize(const void* X, int64_t M, int64_t K, i
                                           void* codes, float* scales, int32_t* sums, cudaStream_t st) {
     if (M == 0) return DVDQ_OK;
     const int sb = storage_bits(q);
-    if (sb == 4) return launch_rq_bits<4>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, q.bits, st);
-    if (sb == 6) return launch_rq_bits<6>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, q.bits, st);
-    return launch_rq_bits<8>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group != 0, q.bits, st);
+    const bool sub = q.scale_group != 0 && q.scale_group < kRqSpan;
+#define DVDQ_RQ_BITS(B)                                                                                                  \
+    if (sb == B)                                                                                                         \
+        return sub ? launch_rq_bits<B, true>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group, q.bits, st)  \
+                   : launch_rq_bits<B, false>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group, q.bits, st);
+    DVDQ_RQ_BITS(4)
+    DVDQ_RQ_BITS(6)
+    DVDQ_RQ_BITS(8)
+#undef DVDQ_RQ_BITS
+    return DVDQ_ERR_BITS;
 }
 
 }  // namespace dvdq

@@ -42,10 +42,18 @@ def test_size_queries():
     q = B.ActQuant(4, 1024, 0)
     ws = B.dvdq_qlinear_workspace_bytes(1000, 3072, q)
     assert ws >= 1000 * 1536 + 8000 and ws % 256 == 0
-    assert B.dvdq_qlinear_workspace_bytes(1000, 3072, B.ActQuant(4, 2048, 0)) == 0   # B > 1024
+    assert B.dvdq_qlinear_workspace_bytes(1000, 3072, B.ActQuant(4, 2048, 0)) == 0   # B does not divide K
+    assert B.dvdq_qlinear_workspace_bytes(1000, 4096, B.ActQuant(4, 2048, 0)) > 0
+    assert B.dvdq_qlinear_workspace_bytes(1000, 12288, B.ActQuant(4, 4096, 0)) > 0
+    assert B.dvdq_qlinear_workspace_bytes(1000, 16384, B.ActQuant(4, 8192, 0)) == 0  # B > 4096
     assert B.dvdq_qlinear_workspace_bytes(1000, 1536, B.ActQuant(4, 1024, 0)) == 0   # B does not divide K
     assert B.dvdq_qlinear_workspace_bytes(1000, 3072, B.ActQuant(4, 1024, 64)) == 0  # granularity that is not built
-    # block-wise scales: one scale and one code sum per token and block of 1024 channels
+    # block-wise scales: one scale and one code sum per token and group of 128, 256 or 1024 channels
+    assert B.dvdq_act_scales_count(1000, 3072, B.ActQuant(4, 256, 256)) == 12000
+    assert B.dvdq_act_scales_count(1000, 3072, B.ActQuant(4, 256, 128)) == 24000
+    assert B.dvdq_act_scales_count(1000, 8960, B.ActQuant(4, 256, 256)) == 35000
+    assert B.dvdq_act_scales_count(1000, 8960, B.ActQuant(4, 256, 1024)) == 0         # 8960 is not a multiple of 1024
+    assert B.dvdq_act_scales_count(1000, 384, B.ActQuant(4, 64, 128)) == 0            # the GEMM takes k-blocks in pairs: K % 256
     qb = B.ActQuant(4, 256, 1024)
     assert B.dvdq_act_scales_count(1000, 3072, q) == 1000
     assert B.dvdq_act_scales_count(1000, 3072, qb) == 3000
@@ -76,9 +84,11 @@ def test_validation_happens_before_any_cuda_call():
     assert lib.dvdq_rotate_quantize(one, 4, 256, 128, C.byref(B.ActQuant(4, 256, 0)), one, one, one, None) == B.ERR_SHAPE
     assert lib.dvdq_rotate_quantize(one, 4, 256, 256, C.byref(B.ActQuant(4, 96, 0)), one, one, one, None) == B.ERR_ROT_BLOCK
     assert lib.dvdq_rotate_quantize(one, 4, 256, 256, C.byref(B.ActQuant(4, 512, 0)), one, one, one, None) == B.ERR_ROT_BLOCK
+    assert lib.dvdq_rotate_quantize(one, 4, 16384, 16384, C.byref(B.ActQuant(4, 8192, 0)), one, one, one, None) == B.ERR_ROT_BLOCK
     assert lib.dvdq_rotate_quantize(one, 4, 256, 256, C.byref(B.ActQuant(4, 256, 1)), one, one, one, None) == B.ERR_UNSUPPORTED
     assert lib.dvdq_rotate_quantize(one, 4, 2048, 2048, C.byref(B.ActQuant(4, 256, 512)), one, one, one, None) == B.ERR_UNSUPPORTED
     assert lib.dvdq_rotate_quantize(one, 4, 1536, 1536, C.byref(B.ActQuant(4, 256, 1024)), one, one, one, None) == B.ERR_SHAPE
+    assert lib.dvdq_rotate_quantize(one, 4, 384, 384, C.byref(B.ActQuant(4, 128, 128)), one, one, one, None) == B.ERR_SHAPE
     assert lib.dvdq_rotate_quantize(None, 4, 256, 256, C.byref(B.ActQuant(4, 256, 0)), one, one, one, None) == B.ERR_NULL
     assert lib.dvdq_rotate_quantize(C.c_void_p(8), 4, 256, 256, C.byref(B.ActQuant(4, 256, 0)), one, one, one, None) == B.ERR_ALIGN
     # weight handle checks
@@ -92,6 +102,28 @@ def test_validation_happens_before_any_cuda_call():
     assert lib.dvdq_qgemm(one, one, one, 4, C.byref(B.ActQuant(4, 256, 0)), C.byref(w), None, 0, one, 256, None) == B.ERR_BLOB
     assert lib.dvdq_pack_weights(one, one, one, 250, 256, 256, one, C.byref(w), None) == B.ERR_SHAPE
     assert lib.dvdq_qlinear(one, 4, 256, C.byref(B.ActQuant(4, 256, 0)), C.byref(B.Weights()), None, 0, one, 256, one, 0, None) == B.ERR_BLOB
+    # dvdq_qlinear and dvdq_qlinear_static refuse everything dvdq_qgemm would refuse BEFORE their
+    # first launch (the pointers here are never dereferenced, so nothing was launched)
+    w = B.Weights(0x51445644, 1, 256, 256, 256, 0, 4096, B.dvdq_weight_blob_bytes(256, 256))
+    big = 1 << 30
+    for call in (lambda q, act, ldy, M=4: lib.dvdq_qlinear(one, M, 256, C.byref(q), C.byref(w), None, act, one, ldy, one, big, None),
+                 lambda q, act, ldy, M=4: lib.dvdq_qlinear_static(one, M, 256, C.byref(q), C.byref(w), None, act, one, ldy, None)):
+        assert call(B.ActQuant(4, 128, 0), 0, 256) == B.ERR_ROT_BLOCK       # activations and weights disagree on B
+        assert call(B.ActQuant(4, 256, 0), 7, 256) == B.ERR_UNSUPPORTED     # unknown activation function
+        assert call(B.ActQuant(4, 256, 0), 0, 250) == B.ERR_SHAPE           # ldy < N
+        assert call(B.ActQuant(4, 256, 0), 0, 256, 0x7FFFFF01) == B.ERR_SHAPE
+    assert lib.dvdq_qlinear(one, 4, 256, C.byref(B.ActQuant(4, 256, 0)), C.byref(w), None, 0, None, 256, one, big, None) == B.ERR_NULL
+    assert lib.dvdq_qlinear(one, 4, 256, C.byref(B.ActQuant(4, 256, 0)), C.byref(w), None, 0, C.c_void_p(8), 256, one, big, None) == B.ERR_ALIGN
+    # the offline weight entry points
+    assert lib.dvdq_rotate_weights(one, 8, 250, 256, 0, one, None) == B.ERR_SHAPE
+    assert lib.dvdq_rotate_weights(one, 8, 256, 128, 0, one, None) == B.ERR_SHAPE       # ldw < K
+    assert lib.dvdq_rotate_weights(one, 8, 256, 256, 96, one, None) == B.ERR_ROT_BLOCK
+    assert lib.dvdq_rotate_weights(None, 8, 256, 256, 64, one, None) == B.ERR_NULL
+    assert lib.dvdq_quantize_weights_symmetric(one, 9, 256, 256, 64, one, C.byref(B.Weights()), None) == B.ERR_SHAPE   # N % 8
+    assert lib.dvdq_quantize_weights_symmetric(one, 8, 256, 256, 64, one, None, None) == B.ERR_NULL
+    assert lib.dvdq_quantize_weights_symmetric(one, 8, 256, 256, 64, C.c_void_p(64), C.byref(B.Weights()), None) == B.ERR_ALIGN
+    assert lib.dvdq_int8_mma_ceiling(0, None, None) == B.ERR_SHAPE
+    assert lib.dvdq_debug_wait_timeout(0, None) == B.ERR_SHAPE
 
 
 def test_binding_refuses_cpu_tensors():

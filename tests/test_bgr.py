@@ -117,17 +117,22 @@ def test_bgr_kernel_matches_oracle(N, K, seed):
 
 @pytest.mark.gpu
 def test_bgr_weights_feed_the_quantized_layer():
-    """rotate -> BGR (GPU) -> pack -> qlinear, against the oracle run on the same grid."""
+    """rotate (GPU) -> BGR (GPU) -> pack -> qlinear, against the oracle run on the same grid."""
     from helpers import act_quant, bf16_values, to_bits, oracle_y_for_validated_codes
     M, N, K, Bk, bits = 130, 264, 1536, 512, 4
     g = torch.Generator().manual_seed(11)
     x = torch.randn(M, K, generator=g).to(torch.bfloat16)
     wb = (torch.randn(N, K, generator=g) * 0.02).to(torch.bfloat16)
-    wt32 = orc.rotate(to_bits(wb), Bk).astype(np.float32)
+    wt32 = torch.empty(N, K, dtype=torch.float32, device="cuda")
+    B.dvdq_rotate_weights(wb.cuda(), Bk, wt32)                      # W~ = W R on the GPU: no CPU step feeds the GPU path
     u = torch.empty(N, K, dtype=torch.uint8, device="cuda")
     d = torch.empty(N, dtype=torch.float32, device="cuda")
     z = torch.empty(N, dtype=torch.int32, device="cuda")
-    B.dvdq_bgr_quantize(torch.from_numpy(wt32).cuda(), 100, 1e-5, 50, u, d, z)
+    B.dvdq_bgr_quantize(wt32, 100, 1e-5, 50, u, d, z)
+    # the grid the GPU chose is the oracle's for the same rotated weights
+    u_or, d_or, z_or, _ = orc.bgr_quantize(wt32.cpu().numpy().astype(np.float64))
+    assert np.array_equal(z.cpu().numpy(), z_or) and np.allclose(d.cpu().numpy().astype(np.float64), d_or, rtol=2e-7)
+    assert (u.cpu().numpy() != u_or).mean() <= 1e-4
     blob = torch.empty(B.dvdq_weight_blob_bytes(N, K), dtype=torch.uint8, device="cuda")
     w = B.dvdq_pack_weights(u, d, z, Bk, blob)
     q = act_quant(bits, Bk)

@@ -1,5 +1,6 @@
-"""Block-wise activation scales (one scale per token and per block of 1024 rotated channels; the
-granularity study of Sec. 3.2): the CUDA path against the oracle's block-wise quantizer and layer."""
+"""Block-wise activation scales (one scale per token and per group of 128, 256 or 1024 rotated
+channels; the block-wise variant of Sec. 3.2's last paragraph): the CUDA path against the oracle's
+block-wise quantizer and layer, for every group size the library builds."""
 import numpy as np
 import pytest
 import torch
@@ -11,7 +12,7 @@ from helpers import bf16_values, check_codes_against_oracle, gpu_pack_weights, t
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-G = 1024                # the block the library builds
+GROUPS = [1024, 256, 128]   # the groups the library builds: whole k-blocks of the GEMM
 SCALE_RTOL = 1e-6
 Y_MAXNORM_RTOL = 4e-3
 
@@ -40,7 +41,7 @@ def synth_w(N, K, seed, mode):
     return w.to(torch.bfloat16)
 
 
-def gpu_rotate_quantize_blockwise(x_dev, bits, Bk):
+def gpu_rotate_quantize_blockwise(x_dev, bits, Bk, G):
     M, K = x_dev.shape
     q = B.ActQuant(bits, Bk, G)
     n = B.dvdq_act_scales_count(M, K, q)
@@ -55,24 +56,39 @@ def gpu_rotate_quantize_blockwise(x_dev, bits, Bk):
     return codes, scales.view(M, K // G), sums.view(M, K // G), nat
 
 
-def check_blockwise_codes(nat, codes_or, xt, s64):
+def check_blockwise_codes(nat, codes_or, xt, s64, G, min_agree=0.9999):
+    # the agreement bar is over the whole tensor (one legitimate tie flip in a 77 x 128 slice is
+    # already 1e-4 of it); that every mismatch is +-1 on a tie is checked group by group, each
+    # against its own scale
+    assert (nat.astype(np.int32) == codes_or).mean() >= min_agree
     for g in range(codes_or.shape[1] // G):
         sl = slice(g * G, (g + 1) * G)
-        check_codes_against_oracle(nat[:, sl], codes_or[:, sl], xt[:, sl], s64[:, g])
+        check_codes_against_oracle(nat[:, sl], codes_or[:, sl], xt[:, sl], s64[:, g], min_agree=0.0)
 
 
+@pytest.mark.parametrize("G", GROUPS)
 @pytest.mark.parametrize("bits", [4, 6, 8])
-@pytest.mark.parametrize("M,K,Bk", [(300, 3072, 256), (257, 2048, 1024), (65, 1024, 64), (130, 5120, 128)])
-def test_rotate_quantize_blockwise_matches_oracle(M, K, Bk, bits):
+@pytest.mark.parametrize("M,K,Bk", [(300, 3072, 256), (257, 2048, 1024), (65, 1024, 64), (130, 5120, 128),
+                                    (77, 1536, 512), (41, 8960, 256), (36, 4096, 4096), (50, 1024, 0)])
+def test_rotate_quantize_blockwise_matches_oracle(M, K, Bk, bits, G):
+    if K % G:
+        pytest.skip("K is not a multiple of the group")
     x = synth_x(M, K, seed=M + K + bits)
+    x[M // 3] = 0                                               # an all-zero token: every group scale 0
     xt = orc.rotate(to_bits(x), Bk)
     codes_or, s64, s32 = orc.act_quantize_grouped(xt, bits, G)
-    _, scales, sums, nat = gpu_rotate_quantize_blockwise(x.to(DEV), bits, Bk)
+    _, scales, sums, nat = gpu_rotate_quantize_blockwise(x.to(DEV), bits, Bk, G)
     assert_device_ok()
     s = scales.cpu().numpy().astype(np.float64)
     assert np.all(np.abs(s - s64) <= SCALE_RTOL * s64)
     nat = nat.cpu().numpy()
-    check_blockwise_codes(nat, codes_or, xt, s64)
+    assert np.all(nat[M // 3] == 0) and np.all(s[M // 3] == 0)
+    # Without a rotation x~ is a bf16 value and the group's absmax another: quotients x~ qmax / absmax
+    # that are EXACT half-integers are common (a few per ten thousand elements with short groups).
+    # The GPU rounds the exact quotient half to even; the oracle's two fp64 roundings (s = a / qmax,
+    # then x~ / s) land on either side of it.  Both codes are valid and the check below still
+    # requires every mismatch to be +-1 on such a tie, so only the agreement bar is lower there.
+    check_blockwise_codes(nat, codes_or, xt, s64, G, min_agree=0.9999 if Bk else 0.999)
     # the sums belong to the codes that were written, block by block, exactly
     assert np.array_equal(sums.cpu().numpy(), nat.astype(np.int64).reshape(M, K // G, G).sum(axis=2))
 
@@ -80,7 +96,7 @@ def test_rotate_quantize_blockwise_matches_oracle(M, K, Bk, bits):
 def test_blockwise_equals_per_token_when_there_is_one_block():
     M, K, bits, Bk = 200, 1024, 4, 256
     x = synth_x(M, K, seed=5).to(DEV)
-    pc, ps, pS, pn = gpu_rotate_quantize_blockwise(x, bits, Bk)
+    pc, ps, pS, pn = gpu_rotate_quantize_blockwise(x, bits, Bk, 1024)
     q = B.ActQuant(bits, Bk, 0)
     codes = torch.empty_like(pc)
     scales = torch.empty(M, dtype=torch.float32, device=DEV)
@@ -91,7 +107,7 @@ def test_blockwise_equals_per_token_when_there_is_one_block():
 
 
 LAYER_CASES = [
-    # M, N, K, B, bits, weight mode: M and N tails (N tail against the 128-wide tile), 1 to 5 blocks, z != 8
+    # M, N, K, B, bits, weight mode: M and N tails (N tail against the 128-wide tile), 1 to 40 groups, z != 8
     (257, 392, 3072, 256, 4, "minmax"),
     (300, 128, 1024, 1024, 4, "symmetric"),
     (130, 520, 2048, 128, 6, "minmax"),
@@ -99,7 +115,7 @@ LAYER_CASES = [
 ]
 
 
-def pack_blockwise(codes_np, bits, Bk):
+def pack_blockwise(codes_np, bits, Bk, G):
     M, K = codes_np.shape
     q = B.ActQuant(bits, Bk, G)
     nat = torch.from_numpy(codes_np.astype(np.int8)).to(DEV)
@@ -109,24 +125,25 @@ def pack_blockwise(codes_np, bits, Bk):
     return packed, sums, q
 
 
+@pytest.mark.parametrize("G", GROUPS)
 @pytest.mark.parametrize("act", [0, 1])
 @pytest.mark.parametrize("M,N,K,Bk,bits,mode", LAYER_CASES)
-def test_qgemm_blockwise_on_oracle_codes_and_scales(M, N, K, Bk, bits, mode, act):
+def test_qgemm_blockwise_on_oracle_codes_and_scales(M, N, K, Bk, bits, mode, act, G):
     x = synth_x(M, K, seed=3 * M + N)
     u, d, z = orc.prepare_weights(to_bits(synth_w(N, K, M + N, mode)), Bk, mode)
     codes, s64, s32 = orc.act_quantize_grouped(orc.rotate(to_bits(x), Bk), bits, G)
     bias = (torch.randn(N, generator=torch.Generator().manual_seed(N)) * 0.05).to(torch.bfloat16)
     y_or = bf16_values(orc.combine_grouped(codes, u, z, s32, d, G, to_bits(bias), act))
     w, blob = gpu_pack_weights(u, d, z, Bk)
-    packed, sums, q = pack_blockwise(codes, bits, Bk)
+    packed, sums, q = pack_blockwise(codes, bits, Bk, G)
     assert np.array_equal(sums.cpu().numpy().reshape(M, K // G), codes.reshape(M, K // G, G).sum(axis=2))
     Y = torch.zeros(M, N + 8, dtype=torch.bfloat16, device=DEV)[:, :N]
     B.dvdq_qgemm(packed, torch.from_numpy(np.ascontiguousarray(s32)).to(DEV), sums, M, q, w, bias.to(DEV), act, Y)
     assert_device_ok()
     y = Y.to(torch.float64).cpu().numpy()
     assert np.abs(y - y_or).max() <= Y_MAXNORM_RTOL * np.abs(y_or).max()
-    # same integer inputs: what differs is fp32 against fp64 in the combination of at most five
-    # block terms -- a few ulp of fp32, far below the bf16 rounding, so nearly every output is equal
+    # same integer inputs: what differs is fp32 against fp64 in the combination of at most forty
+    # group terms -- a few ulp of fp32, far below the bf16 rounding, so nearly every output is equal
     assert np.mean(y != y_or) < 0.02
     # the int32 output does not depend on the scales: bit-exact against the whole-K integer GEMM
     acc = torch.zeros(M, N, dtype=torch.int32, device=DEV)
@@ -135,8 +152,9 @@ def test_qgemm_blockwise_on_oracle_codes_and_scales(M, N, K, Bk, bits, mode, act
     assert np.array_equal(acc.cpu().numpy(), orc.int_gemm(codes, u, z))
 
 
+@pytest.mark.parametrize("G", GROUPS)
 @pytest.mark.parametrize("M,N,K,Bk,bits,mode", LAYER_CASES)
-def test_qlinear_blockwise_matches_oracle_end_to_end(M, N, K, Bk, bits, mode):
+def test_qlinear_blockwise_matches_oracle_end_to_end(M, N, K, Bk, bits, mode, G):
     x = synth_x(M, K, seed=7 * M + N)
     u, d, z = orc.prepare_weights(to_bits(synth_w(N, K, M + N + 1, mode)), Bk, mode)
     out = orc.qlinear_grouped(to_bits(x), u, d, z, Bk, bits, G)
@@ -150,7 +168,7 @@ def test_qlinear_blockwise_matches_oracle_end_to_end(M, N, K, Bk, bits, mode):
     assert_device_ok()
     nat = nat.cpu().numpy()
     # codes first (equal, or +-1 on a rounding tie), then the rest of the layer on the validated codes
-    check_blockwise_codes(nat, out["codes"], out["xt"], out["scale64"])
+    check_blockwise_codes(nat, out["codes"], out["xt"], out["scale64"], G)
     y_or = bf16_values(orc.combine_grouped(nat.astype(np.int32), u, z, out["scale32"], d, G))
     y = Y.to(torch.float64).cpu().numpy()
     assert np.abs(y - y_or).max() <= Y_MAXNORM_RTOL * np.abs(y_or).max()
@@ -162,8 +180,9 @@ def test_qlinear_blockwise_matches_oracle_end_to_end(M, N, K, Bk, bits, mode):
         assert torch.equal(Y, Y2)
 
 
+@pytest.mark.parametrize("G", GROUPS)
 @pytest.mark.parametrize("bits", [4, 6])
-def test_blockwise_with_codes_kept_in_bytes_equals_packed(bits):
+def test_blockwise_with_codes_kept_in_bytes_equals_packed(bits, G):
     """container_bits = 8 changes where a code is stored, not the code, the block scales or the output."""
     M, N, K, Bk = 200, 392, 2048, 256
     x = synth_x(M, K, seed=21 + bits).to(DEV)
@@ -182,7 +201,8 @@ def test_blockwise_with_codes_kept_in_bytes_equals_packed(bits):
     assert torch.equal(ys[0][1], ys[1][1]) and torch.equal(ys[0][0], ys[1][0])
 
 
-def test_blockwise_scales_lower_the_quantization_error():
+@pytest.mark.parametrize("G", GROUPS)
+def test_blockwise_scales_lower_the_quantization_error(G):
     """What the option is for: with outlier channels confined to one block, the other blocks get a
     finer grid, so the layer output is closer to the unquantized product than with one scale per token."""
     M, N, K, Bk, bits = 256, 256, 4096, 256, 4
@@ -205,10 +225,11 @@ def test_blockwise_scales_lower_the_quantization_error():
     assert errs[1] < 0.85 * errs[0], errs
 
 
+@pytest.mark.parametrize("G", GROUPS)
 @pytest.mark.parametrize("layer_idx", [3, 0])
-def test_full_size_blockwise_outputs_repeat_and_agree_across_layouts(layer_idx):
+def test_full_size_blockwise_outputs_repeat_and_agree_across_layouts(layer_idx, G):
     """The benchmark's token count with block-wise scales: every launch gives the same bits, with
-    the codes packed and kept in bytes (twelve blocks of 1024 per token on the long layer)."""
+    the codes packed and kept in bytes (12 to 96 groups per token on the long layer)."""
     from paper_2505_18663_b200 import workloads as W
     wl = W.WORKLOADS["hunyuan"]
     layer = wl.layers[layer_idx]

@@ -85,6 +85,8 @@ RQ_CASES = [
     # M, K, B  (several warps per token, ragged last span, every supported block size, no rotation)
     (256, 256, 256), (300, 1536, 512), (130, 3072, 1024), (67, 8960, 256), (33, 13824, 512),
     (129, 320, 64), (65, 640, 128), (40, 5120, 1024), (50, 1024, 0), (9, 12288, 1024),
+    # rotation blocks that span two and four warps
+    (37, 12288, 4096), (70, 4096, 2048), (19, 4096, 4096), (130, 2048, 2048), (11, 16384, 4096),
 ]
 
 
