@@ -2,11 +2,14 @@
 """Benchmark of the quantized-linear hot path (rotate-quantize + int8 tensor-core GEMM with a
 dequantizing epilogue) on HunyuanVideo-shaped layers, one JSON line on stdout.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME|all] [--impl reference]
 
 A step is one pass of the whole path over every layer of the workload (for each layer:
 dvdq_rotate_quantize then dvdq_qgemm, i.e. what dvdq_qlinear runs) on synthetic inputs that
-are already resident in HBM.  With N > 1 (torchrun, one rank per GPU) every rank runs the
+are already resident in HBM.  The headline keeps the activation codes packed b bits each (the
+GEMM widens them); the same step with one int8 per code is timed beside it (`other_layout`).
+Rooflines: the GEMM against the int8 tensor-pipe ceiling measured in the same run (an issue loop
+on resident operands), rotate-quantize against the measured copy rate on its ALGORITHMIC bytes.  With N > 1 (torchrun, one rank per GPU) every rank runs the
 same per-GPU work on its own seeded tokens, there is no data-path collective, and the value
 is the aggregate over ranks divided by the slowest rank's time (weak scaling).
 
@@ -31,6 +34,7 @@ import torch  # noqa: E402
 
 METRIC = "W4A4/W4A6 qlinear throughput (rotate-quantize + int8 tcgen05 GEMM + dequant), TOPS = 2*M*N*K / time"
 NOMINAL_INT8_TOPS = 4500.0
+NOMINAL_HBM_GBS = 8000.0
 INT8_OVER_BF16 = 2.0           # nominal dense ratio, int8 : bf16
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0  # burst; about 1400 sustained
@@ -63,7 +67,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._pump, daemon=True)
             self.thread.start()
@@ -107,8 +111,16 @@ def layer_ops(M, layer):
     return 2.0 * M * layer.N * layer.K
 
 
-def rq_bytes(M, layer, scale_group=0, container=0):
-    """Algorithmic HBM bytes of rotate-quantize: bf16 row in, codes as stored + scales + code sums out."""
+def rq_algorithmic_bytes(M, layer, scale_group=0):
+    """Algorithmic HBM bytes of rotate-quantize per launch: the bf16 row in, b-bit codes and one
+    scale + one code sum per scale group out: 2K + K b / 8 + 8 per token and group, whatever
+    container the codes are kept in."""
+    per_token = layer.K // scale_group if scale_group else 1
+    return M * (2.0 * layer.K + layer.K * layer.bits / 8.0 + 8.0 * per_token)
+
+
+def rq_stored_bytes(M, layer, scale_group=0, container=0):
+    """Bytes the kernel actually moves: as above with the codes at their stored width."""
     per_token = layer.K // scale_group if scale_group else 1
     return M * (2.0 * layer.K + layer.K * (container or layer.bits) / 8.0 + 8.0 * per_token)
 
@@ -181,6 +193,203 @@ def config_of(wl, args):
 
 # ------------------------------------------------------------------ the CUDA leg
 
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/, by code
+# layout (container_bits); None where no capture of that kernel in its present form exists.
+QGEMM_DRAM_TRAFFIC_PER_LAUNCH = {0: None, 8: None}
+RQ_DRAM_TRAFFIC_PER_LAUNCH = {0: None, 8: None}
+
+
+class Leg:
+    """One code layout of the workload: its buffers, and the step that launches rotate-quantize
+    and the GEMM for every layer (what dvdq_qlinear runs), optionally with CUDA events around
+    every launch."""
+
+    def __init__(self, B, W, wl, args, container, dev, rank, shared=None):
+        self.B, self.wl, self.container, self.scale_group = B, wl, container, args.scale_group
+        M = self.M = wl.M
+        if shared is None:
+            xs = {}
+            first = wl.layers[0]
+            for layer in (wl.layers[:1] if wl.chain else wl.layers):
+                if layer.K not in xs:
+                    xs[layer.K] = W.make_activations(wl, layer.K, device=dev, salt=rank)
+            weights = []
+            for i, layer in enumerate(wl.layers):
+                u, d, z = W.make_weight_codes(layer, seed=i, device=dev)
+                blob = torch.empty(B.dvdq_weight_blob_bytes(layer.N, layer.K), dtype=torch.uint8, device=dev)
+                weights.append((B.dvdq_pack_weights(u, d, z, layer.rot_block, blob), blob, W.make_bias(wl, layer, device=dev)))
+                del u
+            Ys = [torch.empty(M, layer.N, dtype=torch.bfloat16, device=dev) for layer in wl.layers]
+            shared = dict(xs=xs, weights=weights, Ys=Ys)
+        self.shared = shared
+        self.layers = []
+        for i, layer in enumerate(wl.layers):
+            q = B.ActQuant(layer.bits, layer.rot_block, args.scale_group, container)
+            n_scales = B.dvdq_act_scales_count(M, layer.K, q)
+            if n_scales == 0:
+                raise SystemExit(f"layer {layer.K}->{layer.N}: activation quantizer options not supported")
+            # in a chain every layer but the first reads the previous layer's output
+            x = shared["Ys"][i - 1] if (wl.chain and i > 0) else shared["xs"][layer.K]
+            w, _, bias = shared["weights"][i]
+            self.layers.append(dict(layer=layer, q=q, x=x, w=w, bias=bias, Y=shared["Ys"][i],
+                                    codes=torch.empty(B.dvdq_act_codes_bytes_q(M, layer.K, q), dtype=torch.uint8, device=dev),
+                                    scales=torch.empty(n_scales, dtype=torch.float32, device=dev),
+                                    sums=torch.empty(n_scales, dtype=torch.int32, device=dev)))
+
+    def step(self, events=None, rq_only=False):
+        B = self.B
+        for li, L in enumerate(self.layers):
+            if events is not None:
+                events[li][0].record()
+            B.dvdq_rotate_quantize(L["x"], L["q"], L["codes"], L["scales"], L["sums"])
+            if events is not None:
+                events[li][1].record()
+            if rq_only:
+                continue
+            B.dvdq_qgemm(L["codes"], L["scales"], L["sums"], self.M, L["q"], L["w"], L["bias"], L["layer"].act, L["Y"])
+            if events is not None:
+                events[li][2].record()
+
+    def timed(self, steps, warmup, barrier, rq_only=False):
+        """(ms per step, per-layer rq ms, per-layer GEMM ms) from CUDA events inside the timed region."""
+        for _ in range(warmup):
+            self.step(rq_only=rq_only)
+        n = len(self.layers)
+        ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(n)] for _ in range(steps)]
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        t0.record()
+        for s in range(steps):
+            self.step(ev[s], rq_only=rq_only)
+        t1.record()
+        barrier()
+        rq_ms = [sum(ev[s][li][0].elapsed_time(ev[s][li][1]) for s in range(steps)) / steps for li in range(n)]
+        gm_ms = [0.0] * n if rq_only else [sum(ev[s][li][1].elapsed_time(ev[s][li][2]) for s in range(steps)) / steps for li in range(n)]
+        return t0.elapsed_time(t1) / steps, rq_ms, gm_ms
+
+
+def measure_int8_ceiling(B, seconds, local_rank):
+    """The int8 tensor-pipe ceiling of this GPU, now: the issue loop of dvdq_int8_mma_ceiling
+    (resident operands, no loads, no epilogue) repeated for about `seconds`, with the SM clock
+    sampled meanwhile."""
+    B.dvdq_int8_mma_ceiling(2000)
+    torch.cuda.synchronize()
+    iters = 20000                        # about 5.5 ms per launch at the nominal rate
+    n = max(3, min(400, int(seconds / 0.0055)))
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    ops = 0
+    for _ in range(n):
+        ops += B.dvdq_int8_mma_ceiling(iters)
+    t1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = t0.elapsed_time(t1)
+    return {"tops": ops / (ms * 1e-3) / 1e12, "ms": ms, "launches": n, "sm_mhz": clocks.get("sm_mhz"),
+            "reasons": clocks.get("reasons"), "what": "tcgen05.mma.cta_group::2.kind::i8 256x256x32 issue loop, operands resident in shared memory"}
+
+
+def roofline_blocks(leg, ms_per_step, rq_ms, gm_ms, args, peaks, ceiling, timed_s):
+    """The two roofline objects of a leg (GEMM: tensor-bound; rotate-quantize: HBM-bound) and its stages."""
+    M, layers, sg, cont = leg.M, leg.layers, leg.scale_group, leg.container
+    gemm_tops = sum(layer_ops(M, L["layer"]) for L in layers) / (sum(gm_ms) * 1e-3) / 1e12
+    alg = sum(rq_algorithmic_bytes(M, L["layer"], sg) for L in layers)
+    stored = sum(rq_stored_bytes(M, L["layer"], sg, cont) for L in layers)
+    rq_gbs = alg / (sum(rq_ms) * 1e-3) / 1e9
+    # which library figure a GEMM timed like this compares with: the burst one for a region well under a second
+    bf16_kind = "bf16_tflops" if timed_s < 1.0 else "bf16_tflops_sustained"
+    gemm_kernel = "qgemm_ss_kernel" if cont == 8 else "qgemm_kernel"
+    peak = ceiling["tops"] if ceiling else peaks[bf16_kind] * INT8_OVER_BF16
+    roof = {"kernel": gemm_kernel + " (tcgen05.mma kind::i8)", "bound": "tensor", "achieved": gemm_tops, "peak": peak, "unit": "TOPS",
+            "frac": gemm_tops / peak,
+            "peak_source": ("measured in this run: int8 issue-loop ceiling (dvdq_int8_mma_ceiling) at a median SM clock of "
+                            f"{ceiling['sm_mhz']} MHz" if ceiling else f"{peaks['source']}: {bf16_kind} x {INT8_OVER_BF16}"),
+            "frac_of_nominal_4500": gemm_tops / NOMINAL_INT8_TOPS,
+            "frac_of_2x_bf16_burst": gemm_tops / (peaks["bf16_tflops"] * INT8_OVER_BF16),
+            "frac_of_2x_bf16_sustained": gemm_tops / (peaks["bf16_tflops_sustained"] * INT8_OVER_BF16),
+            "avg_launch_ms": sum(gm_ms) / len(gm_ms), "traffic": QGEMM_DRAM_TRAFFIC_PER_LAUNCH.get(cont) if args.default_workload else None}
+    rq_roof = {"kernel": "rq_kernel", "bound": "hbm", "achieved": rq_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+               "frac": rq_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"] + ": hbm_gbs (copy rate)",
+               "frac_of_nominal_8000": rq_gbs / NOMINAL_HBM_GBS,
+               "bytes": "algorithmic: 2K + K b/8 + 8 per token and scale group",
+               "stored_bytes_gbs": stored / (sum(rq_ms) * 1e-3) / 1e9,
+               "avg_launch_ms": sum(rq_ms) / len(rq_ms), "traffic": RQ_DRAM_TRAFFIC_PER_LAUNCH.get(cont) if args.default_workload else None}
+    stages = []
+    for li, L in enumerate(layers):
+        layer = L["layer"]
+        stages.append({"layer": f"{layer.K}->{layer.N} A{layer.bits} B{layer.rot_block}" + (" gelu" if layer.act else "") + (" bias" if layer.bias else ""),
+                       "rq_ms": rq_ms[li], "rq_gbs": rq_algorithmic_bytes(M, layer, sg) / (rq_ms[li] * 1e-3) / 1e9,
+                       "rq_frac_of_hbm": rq_algorithmic_bytes(M, layer, sg) / (rq_ms[li] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                       "qgemm_ms": gm_ms[li], "qgemm_tops": layer_ops(M, layer) / (gm_ms[li] * 1e-3) / 1e12,
+                       "qgemm_frac_of_peak": layer_ops(M, layer) / (gm_ms[li] * 1e-3) / 1e12 / peak})
+    return roof, rq_roof, stages
+
+
+def run_workload(args, wl, B, W, D, dist, dev, rank, local_rank, world, peaks, full):
+    """Times one workload; `full` adds the legs of the headline line (other layout, alone, ceiling, e2e, oracle)."""
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def check_status():
+        status, detail = B.dvdq_last_device_status()
+        if status != B.OK:
+            raise SystemExit(f"device status {status} ({B.status_string(status)}), wait id {detail}")
+
+    leg = Leg(B, W, wl, args, args.container, dev, rank)
+    M = wl.M
+    warm = max(args.warmup, 3)
+    leg.timed(1, warm - 1, barrier)   # warm-up (and first-use set-up) outside the sampled region
+    check_status()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ms_local, rq_ms, gm_ms = leg.timed(args.steps, 0, barrier)
+    clocks = sampler.stop() if rank == 0 else None
+    ms_per_step = D.max_over_ranks(ms_local, dist, dev)
+    check_status()
+    ops_per_step = sum(layer_ops(M, L["layer"]) for L in leg.layers)
+    value = D.aggregate_rate(ops_per_step, ms_per_step, world) / 1e12
+    timed_s = ms_per_step * args.steps * 1e-3
+
+    ceiling = None
+    if full and not args.no_ceiling:
+        ceiling = measure_int8_ceiling(B, min(2.0, max(0.1, timed_s)), local_rank)
+        check_status()
+    roof, rq_roof, stages = roofline_blocks(leg, ms_per_step, rq_ms, gm_ms, args, peaks, ceiling, timed_s)
+
+    out = {"value": value, "ms_per_step": ms_per_step, "roofline": roof, "roofline_rotate_quantize": rq_roof, "stages": stages,
+           "clocks": clocks, "gpu_launches": 2 * len(leg.layers) * args.steps, "ceiling": ceiling, "leg": leg}
+    if not full:
+        return out
+
+    # ---- rotate-quantize on its own (no GEMM between the launches drawing the power budget down)
+    if not args.no_alone:
+        n_alone = max(5, args.steps // 2)
+        _, rq_alone_ms, _ = leg.timed(n_alone, 3, barrier, rq_only=True)
+        alg = sum(rq_algorithmic_bytes(M, L["layer"], args.scale_group) for L in leg.layers)
+        g = alg / (sum(rq_alone_ms) * 1e-3) / 1e9
+        rq_roof["alone"] = {"achieved": g, "frac": g / peaks["hbm_gbs"], "frac_of_nominal_8000": g / NOMINAL_HBM_GBS, "steps": n_alone,
+                            "note": "the same launches without the GEMMs between them"}
+
+    # ---- the same step with the other code layout, as a full block of its own
+    if not args.no_other_layout and world == 1:
+        other = 8 if args.container == 0 else 0
+        leg2 = Leg(B, W, wl, args, other, dev, rank, shared=leg.shared)
+        n2 = max(5, min(args.steps, 50))
+        ms2, rq2, gm2 = leg2.timed(n2, 3, barrier)
+        check_status()
+        r2, rr2, st2 = roofline_blocks(leg2, ms2, rq2, gm2, args, peaks, ceiling, ms2 * n2 * 1e-3)
+        out["other_layout"] = {"act_codes": "one int8 per code" if other == 8 else "packed, b bits per code",
+                               "value": ops_per_step / (ms2 * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": ms2, "steps": n2,
+                               "roofline": r2, "roofline_rotate_quantize": rr2, "stages": st2}
+        del leg2
+    return out
+
+
 def run_cuda(args, wl):
     from paper_2505_18663_b200 import binding as B
     from paper_2505_18663_b200 import dist as D
@@ -200,148 +409,51 @@ def run_cuda(args, wl):
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
     B.load()
-    M = wl.M
-
-    # ---- resident inputs (per rank: its own seeded tokens)
-    xs = {}
-    for layer in wl.layers:
-        if layer.K not in xs:
-            xs[layer.K] = W.make_activations(wl, layer.K, device=dev, salt=rank)
-    layers = []
-    for i, layer in enumerate(wl.layers):
-        u, d, z = W.make_weight_codes(layer, seed=i, device=dev)
-        blob = torch.empty(B.dvdq_weight_blob_bytes(layer.N, layer.K), dtype=torch.uint8, device=dev)
-        w = B.dvdq_pack_weights(u, d, z, layer.rot_block, blob)
-        del u
-        q = B.ActQuant(layer.bits, layer.rot_block, args.scale_group, args.container)
-        codes = torch.empty(B.dvdq_act_codes_bytes_q(M, layer.K, q), dtype=torch.uint8, device=dev)
-        n_scales = B.dvdq_act_scales_count(M, layer.K, q)
-        if n_scales == 0:
-            raise SystemExit(f"layer {layer.K}->{layer.N}: activation quantizer options not supported")
-        scales = torch.empty(n_scales, dtype=torch.float32, device=dev)
-        sums = torch.empty(n_scales, dtype=torch.int32, device=dev)
-        Y = torch.empty(M, layer.N, dtype=torch.bfloat16, device=dev)
-        bias = W.make_bias(wl, layer, device=dev)
-        layers.append(dict(layer=layer, w=w, blob=blob, q=q, codes=codes, scales=scales, sums=sums, Y=Y, bias=bias))
-    torch.cuda.synchronize()
-
-    def step(events=None):
-        for li, L in enumerate(layers):
-            layer = L["layer"]
-            if events is not None:
-                events[li][0].record()
-            B.dvdq_rotate_quantize(xs[layer.K], L["q"], L["codes"], L["scales"], L["sums"])
-            if events is not None:
-                events[li][1].record()
-            B.dvdq_qgemm(L["codes"], L["scales"], L["sums"], M, L["q"], L["w"], L["bias"], layer.act, L["Y"])
-            if events is not None:
-                events[li][2].record()
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
-    status, detail = B.dvdq_last_device_status()
-    if status != B.OK:
-        raise SystemExit(f"device status {status} ({B.status_string(status)}), wait id {detail}")
-
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in layers] for _ in range(args.steps)]
-    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    t_begin.record()
-    for s in range(args.steps):
-        step(ev[s])
-    t_end.record()
-    barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    elapsed_ms = D.max_over_ranks(t_begin.elapsed_time(t_end), dist, dev)
-    status, detail = B.dvdq_last_device_status()
-    if status != B.OK:
-        raise SystemExit(f"device status {status} ({B.status_string(status)}), wait id {detail}")
-
-    ms_per_step = elapsed_ms / args.steps
-    ops_per_step = sum(layer_ops(M, L["layer"]) for L in layers)
-    value = D.aggregate_rate(ops_per_step, ms_per_step, world) / 1e12
-
-    # ---- per-kernel durations from the events of the timed region (this rank)
-    rq_ms = [sum(ev[s][li][0].elapsed_time(ev[s][li][1]) for s in range(args.steps)) / args.steps for li in range(len(layers))]
-    gm_ms = [sum(ev[s][li][1].elapsed_time(ev[s][li][2]) for s in range(args.steps)) / args.steps for li in range(len(layers))]
     peaks = load_peaks()
-    int8_peak = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
-    gemm_ops = sum(layer_ops(M, L["layer"]) for L in layers)
-    gemm_tops = gemm_ops / (sum(gm_ms) * 1e-3) / 1e12
-    rq_total_bytes = sum(rq_bytes(M, L["layer"], args.scale_group, args.container) for L in layers)
-    rq_gbs = rq_total_bytes / (sum(rq_ms) * 1e-3) / 1e9
-    stages = []
-    for li, L in enumerate(layers):
-        layer = L["layer"]
-        stages.append({"layer": f"{layer.K}->{layer.N} A{layer.bits}",
-                       "rq_ms": rq_ms[li], "rq_gbs": rq_bytes(M, layer, args.scale_group, args.container) / (rq_ms[li] * 1e-3) / 1e9,
-                       "qgemm_ms": gm_ms[li], "qgemm_tops": layer_ops(M, layer) / (gm_ms[li] * 1e-3) / 1e12})
+    args.default_workload = (wl.name == "hunyuan" and wl.M == 65536 and args.bits == 0 and args.scale_group == 0)
 
-    # ---- rotate-quantize on its own (no GEMM between the launches, so no GEMM drawing the power budget down)
-    n_alone = 0 if args.no_alone else max(5, args.steps // 5)
-    ev_alone = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in layers] for _ in range(n_alone)]
-    for it in range(3 + n_alone if n_alone else 0):
-        for li, L in enumerate(layers):
-            layer = L["layer"]
-            if it >= 3:
-                ev_alone[it - 3][li][0].record()
-            B.dvdq_rotate_quantize(xs[layer.K], L["q"], L["codes"], L["scales"], L["sums"])
-            if it >= 3:
-                ev_alone[it - 3][li][1].record()
-    torch.cuda.synchronize()
-    rq_alone = None
-    if n_alone:
-        rq_alone_ms = sum(a.elapsed_time(b) for row in ev_alone for a, b in row) / n_alone
-        rq_alone_gbs = rq_total_bytes / (rq_alone_ms * 1e-3) / 1e9
-        rq_alone = {"achieved": rq_alone_gbs, "frac": rq_alone_gbs / load_peaks()["hbm_gbs"], "steps": n_alone,
-                    "note": "the same launches without the GEMMs between them"}
-
-    # ---- the same step with the codes packed b bits each (container 0), for the record: fewer steps
-    packed = None
-    if args.container != 0 and not args.no_packed and world == 1:
-        packed = run_packed_leg(args, wl, layers, xs, dev, B, M)
+    res = run_workload(args, wl, B, W, D, dist, dev, rank, local_rank, world, peaks, full=True)
+    leg = res.pop("leg")
 
     # ---- end to end through dvdq_qlinear with HOST buffers (pinned), copies inside the timed region
     e2e = None
     if not args.no_e2e:
-        e2e = run_e2e(args, wl, layers, xs, dev, B, dist, world)
+        e2e = run_e2e(args, wl, leg, dev, B, dist, world)
+    del leg
+
+    # ---- the other configurations, one after the other (per-layer stages and rooflines only)
+    extra = None
+    if args.all_workloads and world == 1:
+        import dataclasses
+        extra = {}
+        todo = [(n, w, 0) for n, w in W.WORKLOADS.items() if n not in (wl.name, "tiny")]
+        # the HunyuanVideo shapes at both bit widths (the headline runs the seeded 25 % mask)
+        todo += [("hunyuan_all_A4", W.WORKLOADS["hunyuan"], 4), ("hunyuan_all_A6", W.WORKLOADS["hunyuan"], 6)]
+        for name, w2, bits in todo:
+            if bits:
+                w2 = dataclasses.replace(w2, layers=tuple(dataclasses.replace(l, bits=bits) for l in w2.layers))
+            torch.cuda.empty_cache()
+            r = run_workload(args, w2, B, W, D, dist, dev, rank, local_rank, world, peaks, full=False)
+            r.pop("leg")
+            r.pop("ceiling")
+            r["config"] = config_of(w2, args)["workload"]
+            extra[name] = r
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    # the ncu counters were taken on the default workload (hunyuan, its own bit widths, per-token scales)
-    captured = wl.name == "hunyuan" and wl.M == 65536 and args.bits == 0 and args.scale_group == 0 and args.container == 8
     line = {
-        "metric": METRIC, "value": value, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "metric": METRIC, "value": res["value"], "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": res["ms_per_step"], "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "i8", "data": "synthetic", "config": config_of(wl, args),
-        "roofline": {"kernel": ("qgemm_ss_kernel" if args.container == 8 and args.scale_group == 0 else "qgemm_kernel") + " (tcgen05.mma kind::i8)", "bound": "tensor", "achieved": gemm_tops,
-                     "peak": int8_peak, "unit": "TOPS", "frac": gemm_tops / int8_peak,
-                     "peak_source": f"{peaks['source']}: bf16_tflops_sustained x {INT8_OVER_BF16} (nominal int8:bf16)",
-                     "frac_of_nominal_4500": gemm_tops / NOMINAL_INT8_TOPS,
-                     "avg_launch_ms": sum(gm_ms) / len(gm_ms), "traffic": QGEMM_DRAM_TRAFFIC_PER_LAUNCH if captured else None},
-        "roofline_rotate_quantize": {"kernel": "rq_kernel", "bound": "hbm", "achieved": rq_gbs,
-                                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": rq_gbs / peaks["hbm_gbs"],
-                                     "peak_source": peaks["source"], "frac_of_nominal_8000": rq_gbs / 8000.0,
-                                     "avg_launch_ms": sum(rq_ms) / len(rq_ms), "traffic": RQ_DRAM_TRAFFIC_PER_LAUNCH if captured else None,
-                                     "alone": rq_alone},
-        "stages": stages,
-        "packed_codes": packed,
-        "e2e": e2e,
-        "gpu_launches": 2 * len(layers) * args.steps,
-        "clocks": clocks,
+        "roofline": res["roofline"], "roofline_rotate_quantize": res["roofline_rotate_quantize"],
+        "int8_ceiling": res["ceiling"], "stages": res["stages"], "other_layout": res.get("other_layout"),
+        "e2e": e2e, "gpu_launches": res["gpu_launches"], "clocks": res["clocks"],
     }
+    if extra is not None:
+        line["workloads"] = extra
     if not args.no_cpu_baseline and world == 1:
         dt, ops, threads = oracle_sample(wl, args.ref_tokens, scale_group=args.scale_group)
         line["cpu_baseline"] = {"value": ops / dt / 1e12, "unit": "TOPS", "cores": threads, "kind": "oracle",
@@ -351,62 +463,20 @@ def run_cuda(args, wl):
         dist.destroy_process_group()
 
 
-# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/; None
-# until a capture of the corresponding kernel exists.
-QGEMM_DRAM_TRAFFIC_PER_LAUNCH = 1.15e9   # bytes: 16384-token capture x 4 (traffic grows with M), mean of the 4 layers
-RQ_DRAM_TRAFFIC_PER_LAUNCH = 0.94e9
-
-
-def run_packed_leg(args, wl, layers, xs, dev, B, M):
-    """The step with activation codes packed b bits each (the layout the GEMM widens in shared and
-    tensor memory), timed on max(5, steps / 5) steps after 3 warm-up steps.  Same inputs, same outputs."""
-    packed_layers = []
-    for L in layers:
-        layer = L["layer"]
-        q = B.ActQuant(layer.bits, layer.rot_block, args.scale_group, 0)
-        codes = torch.empty(B.dvdq_act_codes_bytes_q(M, layer.K, q), dtype=torch.uint8, device=dev)
-        packed_layers.append((layer, q, codes, L))
-    n_steps = max(5, args.steps // 5)
-    ev = [[[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in packed_layers] for _ in range(n_steps)]
-
-    def step(events=None):
-        for li, (layer, q, codes, L) in enumerate(packed_layers):
-            if events is not None:
-                events[li][0].record()
-            B.dvdq_rotate_quantize(xs[layer.K], q, codes, L["scales"], L["sums"])
-            if events is not None:
-                events[li][1].record()
-            B.dvdq_qgemm(codes, L["scales"], L["sums"], M, q, L["w"], L["bias"], layer.act, L["Y"])
-            if events is not None:
-                events[li][2].record()
-
-    for _ in range(3):
-        step()
-    torch.cuda.synchronize()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for s in range(n_steps):
-        step(ev[s])
-    t1.record()
-    torch.cuda.synchronize()
-    ms = t0.elapsed_time(t1) / n_steps
-    rq_ms = sum(ev[s][li][0].elapsed_time(ev[s][li][1]) for s in range(n_steps) for li in range(len(packed_layers))) / n_steps
-    gm_ms = sum(ev[s][li][1].elapsed_time(ev[s][li][2]) for s in range(n_steps) for li in range(len(packed_layers))) / n_steps
-    ops = sum(layer_ops(M, l) for l, _, _, _ in packed_layers)
-    nbytes = sum(rq_bytes(M, l, args.scale_group, 0) for l, _, _, _ in packed_layers)
-    return {"value": ops / (ms * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": ms, "steps": n_steps,
-            "qgemm_tops": ops / (gm_ms * 1e-3) / 1e12, "rq_gbs": nbytes / (rq_ms * 1e-3) / 1e9}
-
-
-def run_e2e(args, wl, layers, xs, dev, B, dist, world):
+def run_e2e(args, wl, leg, dev, B, dist, world):
     """Same metric through the user-facing call dvdq_qlinear, with the layer input copied from
     pinned host memory and the layer output copied back to pinned host memory inside every step.
     Three streams (copy-in, compute, copy-out) and two device input buffers let the PCIe copies of
-    neighbouring layers overlap the kernels; every byte still crosses the bus inside the timed region."""
+    neighbouring layers overlap the kernels; every byte still crosses the bus inside the timed region.
+    (In the chain workload every layer's input is copied in like the others': the host holds it.)"""
     M = wl.M
+    layers = leg.layers
     maxK = max(L["layer"].K for L in layers)
     maxN = max(L["layer"].N for L in layers)
-    host_x = {K: x.to("cpu").pin_memory() for K, x in xs.items()}
+    host_x = {}
+    for L in layers:
+        if L["layer"].K not in host_x:
+            host_x[L["layer"].K] = L["x"].to("cpu").pin_memory()
     host_y = [torch.empty(M, maxN, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
     dev_x = [torch.empty(M, maxK, dtype=torch.bfloat16, device=dev) for _ in range(2)]
     ws = torch.empty(max(B.dvdq_qlinear_workspace_bytes(M, L["layer"].K, L["q"]) for L in layers), dtype=torch.uint8, device=dev)
@@ -475,22 +545,28 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="hunyuan")
+    ap.add_argument("--workload", default="hunyuan",
+                    help="tiny, wan1p3b, hunyuan (default, the headline), wan14b, ffn_chain; 'all' = the headline plus a "
+                         "'workloads' block with the per-layer figures of every other configuration")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--ref-tokens", type=int, default=384, help="token sample timed on the CPU oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--tokens", type=int, default=0, help="override the workload's token count (profiling runs)")
-    ap.add_argument("--container", type=int, default=8,
-                    help="8: one int8 per activation code (default, the faster GEMM); 0: codes packed b bits each")
-    ap.add_argument("--no-packed", action="store_true", help="skip the extra leg that times the packed layout")
+    ap.add_argument("--container", type=int, default=0,
+                    help="0 (default): activation codes packed b bits each, widened inside the GEMM; "
+                         "8: one int8 per code, read by the GEMM as they are")
+    ap.add_argument("--no-other-layout", "--no-packed", dest="no_other_layout", action="store_true",
+                    help="skip the extra leg that times the other code layout")
     ap.add_argument("--no-alone", action="store_true", help="skip the extra leg that times rotate-quantize on its own")
+    ap.add_argument("--no-ceiling", action="store_true", help="skip the int8 issue-loop ceiling (the roofline then falls back to 2 x bf16)")
     ap.add_argument("--scale-group", type=int, default=0,
-                    help="0: one activation scale per token; 1024: one per token and block of 1024 channels")
+                    help="0: one activation scale per token; 128, 256, 1024: one per token and group of that many channels")
     ap.add_argument("--bits", type=int, default=0, help="override the activation bit width of every layer (4, 6 or 8)")
     args = ap.parse_args()
     from paper_2505_18663_b200 import workloads as W
-    wl = W.WORKLOADS[args.workload]
+    args.all_workloads = args.workload == "all"
+    wl = W.WORKLOADS["hunyuan" if args.all_workloads else args.workload]
     if args.tokens > 0:
         import dataclasses
         wl = dataclasses.replace(wl, M=args.tokens)

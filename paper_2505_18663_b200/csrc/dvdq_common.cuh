@@ -163,14 +163,12 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
 }
 
 // Before a buffer that this thread has READ is handed back to whoever overwrites it (a TMA copy
-// armed by the arrive that follows): a CTA-scope fence, which waits until the thread's loads have
-// delivered.  An mbarrier arrive is not a shared-memory access in the load pipeline: without the
-// fence it could be performed while a load issued before it was still waiting, and the refill
-// landed first -- seen as one stale 32-byte piece of an operand row in about one kernel in two
-// at 65536 tokens, never in small cases.
-__device__ __forceinline__ void fence_loads_done() { asm volatile("fence.acq_rel.cta;" ::: "memory"); }
-
-// The hand-back is also tied to the loaded data itself: the arrive's address is formed from a word of
+// armed by the arrive that follows), the loads must have DELIVERED.  An mbarrier arrive is not an
+// access of the load pipeline, and the instructions that consume the loaded registers may be
+// scheduled after it: the refill then lands before a straggling load has read the stage (seen as a
+// warp's worth of stale operand rows in one k-block, at full size only, and far more often when
+// the epilogue keeps the schedulers busy).  A CTA-scope fence before the arrive made that rare but
+// not impossible.  What closes it is a data dependency: the arrive's address is formed from a word of
 // every load (ANDed with a zero the compiler cannot see through, so the address does not change),
 // and an instruction cannot issue before its operands have been delivered.
 __device__ __forceinline__ uint32_t runtime_zero() {

@@ -8,6 +8,7 @@
 #include "pack.cuh"
 #include "qgemm.cuh"
 #include "qgemm_ss.cuh"
+#include "qgemm_fat.cuh"
 #include "rotate_quantize.cuh"
 #include "weights.cuh"
 #include "diag.cuh"

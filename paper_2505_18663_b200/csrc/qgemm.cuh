@@ -224,18 +224,29 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 // accumulator covers KBG k-blocks (a power of two, or the whole of K): with KBG = 1
                 // the two blocks of a trip go to different accumulators.
                 int kin = 0;  // k-blocks issued into the accumulator in use
+                if constexpr (!BLK) {
+                    acquire();  // one accumulator per tile
+                    if (!ok) break;
+                }
                 for (int kb = 0; ok && kb < KB; kb += 2) {
                     uint32_t acc_h[2];
                     bool first_h[2], last_h[2];
+                    if constexpr (BLK) {
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        first_h[h] = kin == 0;
-                        if (first_h[h]) acquire();
-                        acc_h[h] = acc;
-                        last_h[h] = ++kin == KBG;
-                        if (last_h[h]) kin = 0;
+                        for (int h = 0; h < 2; ++h) {
+                            first_h[h] = kin == 0;
+                            if (first_h[h]) acquire();
+                            acc_h[h] = acc;
+                            last_h[h] = ++kin == KBG;
+                            if (last_h[h]) kin = 0;
+                        }
+                        if (!ok) break;
+                    } else {
+                        acc_h[0] = acc_h[1] = acc;
+                        first_h[0] = kb == 0;
+                        first_h[1] = last_h[0] = false;
+                        last_h[1] = kb + 2 >= KB;
                     }
-                    if (!ok) break;
                     if (!mbar_wait_warp(wd_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     if (!mbar_wait_warp(wd_full(st + 1), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     tc_fence_after();
@@ -542,7 +553,6 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 }
                 // the codes are widened in registers before the stage of tensor memory is known to be free
                 loaded &= rt_zero;
-                fence_loads_done();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_after_loads(pk_empty(pst), loaded);
                 if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
@@ -585,7 +595,6 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 for (int jw = 0; jw < 4; ++jw) { e[it][jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[it][jw] = w[jw] & 0xF0F0F0F0u; }
             }
             loaded &= rt_zero;
-            fence_loads_done();
             __syncwarp();
             if (lane == 0) mbar_arrive_after_loads(wp_empty(pst), loaded);  // the packed rows are in registers
             if (!mbar_wait(wd_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
@@ -732,8 +741,9 @@ static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const
                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
                                    int32_t* acc_out, int64_t ldacc, cudaStream_t st);
 
-static dvdq_status launch_qgemm_ss_blk(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
-                                       const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, cudaStream_t st);
+// qgemm_fat.cuh: the same with block-wise activation scales
+static dvdq_status launch_qgemm_blk(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, cudaStream_t st);
 
 inline dvdq_status launch_qgemm(const void* codes, const float* scales, const int32_t* sums, int64_t M,
                                 const dvdq_act_quant& q, const dvdq_weights& w, const void* bias, int act,
@@ -745,7 +755,7 @@ inline dvdq_status launch_qgemm(const void* codes, const float* scales, const in
     const int spr = q.scale_group != 0 ? (int)(w.K / q.scale_group) : 1;  // code sums (and scales) per token
     const int sb = storage_bits(q);
     if (sb == 8 && !raw && q.scale_group != 0)
-        return launch_qgemm_ss_blk(codes, scales, sums, spr, M, w, bias, act, Y, ldy, st);
+        return launch_qgemm_blk(codes, scales, sums, spr, M, w, bias, act, Y, ldy, st);
     if (sb == 8 && (raw || q.scale_group == 0))
         return raw ? launch_qgemm_ss<true>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
                    : launch_qgemm_ss<false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);

@@ -1,0 +1,423 @@
+// The GEMM for block-wise activation scales with the codes kept one int8 each (Sec. 3.2, last
+// paragraph: one scale per token and per group of 128, 256 or 1024 rotated channels):
+//
+//   y_in = bf16( Delta_n * ( sum_g s_ig * acc_ing  -  (z_n - 8) * T_i ) + bias_n ),
+//   acc_ing = sum_{k in group g} c_ik (u_nk - 8)   exact int32,    T_i = sum_g s_ig * S_ig.
+//
+// Same mainloop as qgemm_ss_kernel (a CTA pair owns 256 tokens x 256 channels, both operands of
+// tcgen05.mma.cta_group::2.kind::i8 in shared memory, two 256-column int32 accumulators that
+// alternate between scale groups).  What a short group changes is the epilogue's share: every
+// group's accumulator has to be read, converted and added into an fp32 running sum, two
+// instructions per output element and group against the tensor core's G multiply-adds.  Tensor
+// memory is full with the two accumulators, so the running sum lives in REGISTERS: eight epilogue
+// warps, one row and 128 columns per thread, with the register file re-divided between the roles
+// (setmaxnreg: the loaders and the widening warps give registers up, the epilogue warps take them).
+// Roles are aligned to groups of four warps, as that instruction requires:
+//   warps 0-3    TMA producer of activation tiles | MMA issuer (leader CTA) | "rows landed"
+//                forwarder | TMA producer of packed weight rows
+//   warps 4-11   widen weight codes into the operand stages (two groups, alternate k-blocks)
+//   warps 12-19  epilogue: warp w reads tensor-memory lanes 32 * (w % 4).., columns 128 * ((w - 12) / 4)..
+// Every wait is bounded, as in qgemm.cuh.
+#pragma once
+
+#include "qgemm_ss.cuh"
+
+namespace dvdq {
+
+constexpr int kFatThreads = 20 * 32;
+constexpr int kFatFirstWWarp = 4, kFatFirstEpilogueWarp = 12;
+// setmaxnreg moves registers between the warps of ONE CTA: what the epilogue warps take must have
+// been given up by the others, out of the CTA's allocation at launch (threads x the kernel's
+// register count), or the taking warps wait for ever.  The host checks the sum against the compiled
+// register count before every first launch (fat_kernel_registers_fit) and refuses to launch otherwise.
+constexpr int kFatRegsLoader = 40, kFatRegsWiden = 48, kFatRegsEpilogue = 168;
+constexpr int kFatRegsTotal = 128 * kFatRegsLoader + 256 * kFatRegsWiden + 256 * kFatRegsEpilogue;
+static_assert(kFatRegsTotal <= kFatThreads * 96, "the CTA's register allocation at 96 registers per thread");
+
+template <int N>
+__device__ __forceinline__ void regs_take() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N>
+__device__ __forceinline__ void regs_give() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFatThreads, 1)
+qgemm_blk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+                 const __grid_constant__ CUtensorMap tmY, const float* __restrict__ scales,
+                 const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
+                 const __nv_bfloat16* __restrict__ bias, int M, int N, int K, int act, int spr) {
+    using S = SsSmem<false>;
+    constexpr int BN = S::BN, BNh = S::BNh;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    const int num_n = (N + BN - 1) / BN, num_m = (M + 2 * kBM - 1) / (2 * kBM);
+    const int num_tiles = num_m * num_n;
+    const int KB = K / kBK;   // even: K is a multiple of 256
+    const int NG = spr;       // scale groups per token
+    const int KBG = KB / NG;  // k-blocks per group: 1, 2 or 8
+
+    const uint32_t bar0 = sbase + S::kBarOff;
+    auto a_full = [&](int s) { return bar0 + 8u * s; };
+    auto a_ready = [&](int s) { return bar0 + 8u * (kSsAStages + s); };
+    auto a_empty = [&](int s) { return bar0 + 8u * (2 * kSsAStages + s); };
+    const uint32_t barw = bar0 + 8u * (3 * kSsAStages);
+    auto ops_full = [&](int s) { return barw + 8u * s; };
+    auto ops_empty = [&](int s) { return barw + 8u * (kSsStages + s); };
+    auto acc_full = [&](int s) { return barw + 8u * (2 * kSsStages + s); };
+    auto acc_empty = [&](int s) { return barw + 8u * (2 * kSsStages + 2 + s); };
+    const uint32_t drain_bar = barw + 8u * (2 * kSsStages + 4);
+    auto wp_full = [&](int s) { return drain_bar + 8u * (1 + s); };
+    auto wp_empty = [&](int s) { return drain_bar + 8u * (1 + kSsWPackedStages + s); };
+    volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + S::kMiscOff);  // [0] tmem base, [1] abort
+    volatile uint32_t* abort_flag = misc + 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kSsAStages; ++s) { mbar_init(a_full(s), 1); mbar_init(a_ready(s), 2); mbar_init(a_empty(s), 1); }
+        for (int s = 0; s < kSsStages; ++s) { mbar_init(ops_full(s), 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
+        for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * 8); }
+        mbar_init(drain_bar, 1);
+        for (int s = 0; s < kSsWPackedStages; ++s) { mbar_init(wp_full(s), 1); mbar_init(wp_empty(s), kSsWWarps / kUnpackGroups); }
+        misc[1] = 0u;
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(sbase + S::kMiscOff, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    const uint32_t tmem_base = misc[0];
+
+    if (warp < kFatFirstWWarp) {
+        regs_give<kFatRegsLoader>();
+        if (warp == 0) {
+            // ------------------------------------------------------------ TMA producer, activation rows
+            if (lane == 0) {
+                tma_prefetch_desc(&tmA);
+                uint32_t st = 0, ph = 0, issued = 0;
+                bool ok = true;
+                for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                    const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
+                    for (int kb = 0; ok && kb < KB; ++kb) {
+                        if (!mbar_wait(a_empty(st), ph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                        mbar_arrive_expect_tx(a_full(st), S::kA);
+                        tma_load_2d(sbase + S::kAOff + st * S::kA, &tmA, a_full(st), kb * kBK, m0);
+                        ++issued;
+                        if (++st == kSsAStages) { st = 0; ph ^= 1u; }
+                    }
+                }
+                if (!ok) {  // giving up: let copies already in flight land before the CTA exits (bounded)
+                    const uint32_t n_out = issued < (uint32_t)kSsAStages ? issued : (uint32_t)kSsAStages;
+                    for (uint32_t i = 0; i < n_out; ++i) {
+                        const uint32_t s = (st + kSsAStages - 1 - i) % kSsAStages;
+                        const uint32_t p = (s < st) ? ph : (ph ^ 1u);
+                        for (int it = 0; it < (1 << 16) && !mbar_try_wait(a_full(s), p); ++it) {}
+                    }
+                }
+            }
+            __syncwarp();
+        } else if (warp == 3) {
+            // ------------------------------------------------------------ TMA producer, packed weight rows
+            if (lane == 0) {
+                tma_prefetch_desc(&tmW);
+                uint32_t wst = 0, wph = 0, wissued = 0;
+                bool ok = true;
+                for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                    const int n0 = (tile % num_n) * BN + (int)rank * BNh;
+                    for (int kb = 0; ok && kb < KB; ++kb) {
+                        if (!mbar_wait(wp_empty(wst), wph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
+                        mbar_arrive_expect_tx(wp_full(wst), S::kWPacked);
+                        tma_load_2d(sbase + S::kWPackedOff + wst * S::kWPacked, &tmW, wp_full(wst), kb * (kBK / 2), n0);
+                        ++wissued;
+                        if (++wst == kSsWPackedStages) { wst = 0; wph ^= 1u; }
+                    }
+                }
+                if (!ok) {
+                    const uint32_t w_out = wissued < (uint32_t)kSsWPackedStages ? wissued : (uint32_t)kSsWPackedStages;
+                    for (uint32_t i = 0; i < w_out; ++i) {
+                        const uint32_t s = (wst + kSsWPackedStages - 1 - i) % kSsWPackedStages;
+                        const uint32_t p = (s < wst) ? wph : (wph ^ 1u);
+                        for (int it = 0; it < (1 << 16) && !mbar_try_wait(wp_full(s), p); ++it) {}
+                    }
+                }
+            }
+            __syncwarp();
+        } else if (warp == 1) {
+            // ------------------------------------------------------------ MMA issuer (leader CTA only)
+            // An accumulator is acquired only when its first k-block is due.  Groups of two or more
+            // k-blocks go two k-blocks per trip (every cycle between two issues is a bubble in the MMA
+            // stream, and pairing halves the waits and votes); groups of one go a k-block at a time,
+            // so that the epilogue of a group overlaps the next group's MMAs.
+            if (rank == 0) {
+                constexpr uint32_t idesc = umma_idesc_s8s8s32(2 * kBM, BN);
+                uint32_t st = 0, ph = 0, sa = 0, pa = 0, lt = 0, acc = 0;
+                bool ok = true;
+                const int step = KBG >= 2 ? 2 : 1;
+                for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                    int kin = 0;
+                    for (int kb = 0; ok && kb < KB; kb += step) {
+                        const bool first = kin == 0;
+                        if (first) {
+                            acc = lt & 1u;
+                            if (!mbar_wait_warp(acc_empty(acc), ((lt >> 1) & 1u) ^ 1u, abort_flag, kWaitAccEmpty)) { ok = false; break; }
+                            ++lt;
+                        }
+                        kin += step;
+                        const bool last = kin == KBG;
+                        if (last) kin = 0;
+                        const uint32_t sa1 = sa + 1 == kSsAStages ? 0u : sa + 1, pa1 = sa + 1 == kSsAStages ? pa ^ 1u : pa;
+                        if (!mbar_wait_warp(a_ready(sa), pa, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                        if (!mbar_wait_warp(ops_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
+                        if (step == 2) {
+                            if (!mbar_wait_warp(a_ready(sa1), pa1, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                            if (!mbar_wait_warp(ops_full(st + 1), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
+                        }
+                        tc_fence_after();
+                        if (elect_one()) {
+                            const uint32_t d_tmem = tmem_base + acc * BN;
+                            for (int h = 0; h < step; ++h) {
+                                const uint32_t sah = h ? sa1 : sa;
+                                const uint64_t adesc = umma_desc_sw128_kmajor(sbase + S::kAOff + sah * S::kA);
+                                const uint64_t bdesc = umma_desc_sw128_kmajor(sbase + S::kWOff + (st + h) * S::kW);
+#pragma unroll
+                                for (int k = 0; k < kBK / 32; ++k)
+                                    tc_mma_i8_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (first && h == 0 && k == 0) ? 0u : 1u);
+                                tc_commit_pair(ops_empty(st + h), 3);
+                                tc_commit_pair(a_empty(sah), 3);
+                            }
+                            if (last) tc_commit_pair(acc_full(acc), 3);
+                        }
+                        __syncwarp();
+                        st += step;
+                        if (st == kSsStages) { st = 0; ph ^= 1u; }
+                        if (step == 2) { sa = sa1; pa = pa1; }
+                        if (++sa == kSsAStages) { sa = 0; pa ^= 1u; }
+                    }
+                }
+                if (elect_one()) tc_commit_pair(drain_bar, 1);
+                __syncwarp();
+                mbar_wait(drain_bar, 0u, abort_flag, kWaitDrain);
+            }
+            __syncwarp();
+        } else {
+            // ------------------------------------------------------------ "activation rows landed" -> leader
+            uint32_t st = 0, ph = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                for (int kb = 0; kb < KB; ++kb) {
+                    if (!mbar_wait_warp(a_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                    if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(st), 0));
+                    __syncwarp();
+                    if (++st == kSsAStages) { st = 0; ph ^= 1u; }
+                }
+            }
+        }
+    } else if (warp < kFatFirstEpilogueWarp) {
+        regs_give<kFatRegsWiden>();
+        // ------------------------------------------------------------ widen weight codes -> shared memory
+        const uint32_t grp = (uint32_t)(warp - kFatFirstWWarp) >> 2;
+        const int u = (threadIdx.x - kFatFirstWWarp * 32) & 127;  // thread of its group of four warps
+        uint32_t j = 0;
+        bool ok = true;
+        const uint32_t rt_zero = runtime_zero();
+        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+            for (int kb = 0; kb < KB; ++kb) {
+                const uint32_t jj = j++;
+                if (jj % kUnpackGroups != grp) continue;
+                const uint32_t pst = jj % kSsWPackedStages, pph = (jj / kSsWPackedStages) & 1u;
+                const uint32_t wst = jj % kSsStages, wph = (jj / kSsStages) & 1u;
+                if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                const uint32_t pw = sbase + S::kWPackedOff + pst * S::kWPacked;
+                const uint32_t wdW = sbase + S::kWOff + wst * S::kW;
+                // BNh rows x 4 chunks of 32 nibbles, stored as (u - 8): the packed rows go into registers
+                // before the operand stage is known to be free, and are widened on their way out
+                constexpr int kPieces = (BNh * 4) / 128;
+                uint4 p[kPieces];
+                uint32_t loaded = 0u;
+#pragma unroll
+                for (int it = 0; it < kPieces; ++it) {
+                    const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                    p[it] = lds128(pw + row * (kBK / 2) + ck * 16);
+                    loaded ^= p[it].w;
+                }
+                loaded &= rt_zero;
+                __syncwarp();
+                if (lane == 0) mbar_arrive_after_loads(wp_empty(pst), loaded);  // the packed rows are in registers
+                if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int it = 0; it < kPieces; ++it) {
+                    const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                    const uint32_t drow = wdW + (row >> 3) * 1024 + (row & 7) * 128;
+                    sts128(drow + (((2 * ck) ^ (row & 7)) << 4), (p[it].x << 4) & 0xF0F0F0F0u, p[it].x & 0xF0F0F0F0u,
+                           (p[it].y << 4) & 0xF0F0F0F0u, p[it].y & 0xF0F0F0F0u);
+                    sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), (p[it].z << 4) & 0xF0F0F0F0u, p[it].z & 0xF0F0F0F0u,
+                           (p[it].w << 4) & 0xF0F0F0F0u, p[it].w & 0xF0F0F0F0u);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(wst), 0));
+            }
+        }
+    } else {
+        regs_take<kFatRegsEpilogue>();
+        // ------------------------------------------------------------ epilogue: running sum over groups in registers
+        const int q = warp & 3;                                   // tensor-memory lane quarter this warp may read
+        const int half = (warp - kFatFirstEpilogueWarp) >> 2;     // which 128 of the tile's 256 columns
+        const int ew = 4 * half + q;
+        constexpr int CW = BN / 2;                                 // columns per thread
+        const uint32_t c_delta = sbase + S::kConstOff + ew * (3 * CW * 4);
+        const uint32_t c_zc = c_delta + CW * 4;                    // (z_n - 8) as a float: exact, |.| <= 8
+        const uint32_t c_bias = c_zc + CW * 4;
+        const uint32_t stg0 = sbase + S::kStageOutOff + ew * (32 * 64);  // 32 rows x 32 bf16
+        constexpr int kShift = 4;  // the widened weights are 16 x (u - 8)
+        if (lane == 0) tma_prefetch_desc(&tmY);
+        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+        uint32_t lt = 0;
+        bool ok = true;
+        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+            const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM, n0 = (tile % num_n) * BN + half * CW;
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < CW / 32; ++i) {
+                const int c = lane + 32 * i, n = n0 + c;
+                const bool okn = n < N;
+                sts32f(c_delta + 4 * c, okn ? __ldg(delta + n) : 0.f);
+                sts32f(c_zc + 4 * c, okn ? (float)__ldg(zc + n) : 0.f);
+                sts32f(c_bias + 4 * c, (okn && bias != nullptr) ? __bfloat162float(bias[n]) : 0.f);
+            }
+            __syncwarp();
+            const int row = m0 + q * 32 + lane;
+            const bool row_ok = row < M;
+            const float* srow = scales + (int64_t)(row_ok ? row : 0) * NG;
+            const int32_t* Srow = sums + (int64_t)(row_ok ? row : 0) * NG;
+            // the zero-point term of all groups at once: T_i = sum_g s_ig S_ig (each S_ig is exact in fp32)
+            float T = 0.f;
+            for (int g = 0; g < NG; ++g) T = fmaf(__ldg(srow + g), (float)__ldg(Srow + g), T);
+            if (!row_ok) T = 0.f;
+            uint64_t run[CW / 2];  // fp32 pairs: columns 2i and 2i + 1
+#pragma unroll
+            for (int t = 0; t < CW / 2; ++t) run[t] = f2_pack(0.f, 0.f);
+            float s_next = row_ok ? __ldg(srow) : 0.f;
+            for (int g = 0; g < NG; ++g, ++lt) {
+                const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
+                const float s_k = s_next * (1.0f / (float)(1 << kShift));
+                const uint64_t s2 = f2_pack(s_k, s_k);
+                if (g + 1 < NG) s_next = row_ok ? __ldg(srow + g + 1) : 0.f;  // its latency hides behind this group
+                if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) { ok = false; break; }
+                tc_fence_after();
+                // 16 columns at a time, the next load in flight while these are added up
+                const uint32_t col0 = tmem_base + a * BN + half * CW + lane_addr;
+                uint32_t ra[16], rb[16];
+                tmem_ld_32x16(col0, ra);
+#pragma unroll
+                for (int c = 0; c < CW / 16; c += 2) {
+                    tmem_ld_wait();
+                    tmem_ld_32x16(col0 + (c + 1) * 16, rb);
+#pragma unroll
+                    for (int t = 0; t < 16; t += 2)
+                        run[c * 8 + t / 2] = f2_fma(f2_pack((float)(int32_t)ra[t], (float)(int32_t)ra[t + 1]), s2, run[c * 8 + t / 2]);
+                    tmem_ld_wait();
+                    if (c + 2 < CW / 16) tmem_ld_32x16(col0 + (c + 2) * 16, ra);
+#pragma unroll
+                    for (int t = 0; t < 16; t += 2)
+                        run[(c + 1) * 8 + t / 2] = f2_fma(f2_pack((float)(int32_t)rb[t], (float)(int32_t)rb[t + 1]), s2, run[(c + 1) * 8 + t / 2]);
+                }
+                // the accumulator is in registers: the MMA warp may have it back
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty(a), 0));
+            }
+            if (!ok) break;
+            // ---- after the last group: dequantize, round, stage 32 columns per TMA store
+#pragma unroll
+            for (int c = 0; c < CW / 32; ++c) {
+                if (lane == 0) tma_store_wait_read<0>();
+                __syncwarp();
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                    const float4 d0 = lds128f(c_delta + 4 * (c * 32 + j)), d1 = lds128f(c_delta + 4 * (c * 32 + j + 4));
+                    const float4 z0 = lds128f(c_zc + 4 * (c * 32 + j)), z1 = lds128f(c_zc + 4 * (c * 32 + j + 4));
+                    const float4 b0 = lds128f(c_bias + 4 * (c * 32 + j)), b1 = lds128f(c_bias + 4 * (c * 32 + j + 4));
+                    const float dl[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
+                    const float zz[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
+                    const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                    uint32_t pk[4];
+#pragma unroll
+                    for (int t = 0; t < 8; t += 2) {
+                        float r0, r1;
+                        f2_unpack(run[(c * 32 + j + t) / 2], r0, r1);
+                        float y0 = fmaf(fmaf(-zz[t], T, r0), dl[t], bb[t]);
+                        float y1 = fmaf(fmaf(-zz[t + 1], T, r1), dl[t + 1], bb[t + 1]);
+                        if (act == 1) {
+                            y0 = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(y0)));
+                            y1 = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(y1)));
+                        }
+                        __nv_bfloat162 b2 = __floats2bfloat162_rn(y0, y1);
+                        pk[t >> 1] = *reinterpret_cast<uint32_t*>(&b2);
+                    }
+                    // 64-byte rows, 16-byte chunk index XORed with (row / 2) % 4: the layout a 64B-swizzled TMA store reads
+                    const int ch = (j >> 3) ^ ((lane >> 1) & 3);
+                    sts128(stg0 + lane * 64 + ch * 16, pk[0], pk[1], pk[2], pk[3]);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                const int nb = n0 + c * 32;
+                if (lane == 0 && nb < N && m0 + q * 32 < M) {
+                    tma_store_2d(&tmY, stg0, nb, m0 + q * 32);
+                    tma_store_commit();
+                }
+            }
+        }
+        if (lane == 0) tma_store_wait_all();
+        __syncwarp();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the peer may read this CTA's shared and tensor memory until it is done too
+    tc_fence_after();
+    if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+// ------------------------------------------------------------------ host side
+
+// True if the registers the kernel's roles ask for fit into what the CTA is given at launch.
+template <typename Kern>
+static bool fat_kernel_registers_fit(Kern kern) {
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, kern) != cudaSuccess) return false;
+    return kFatRegsTotal <= kFatThreads * fa.numRegs && fa.numRegs >= kFatRegsWiden && fa.numRegs <= kFatRegsEpilogue;
+}
+
+static dvdq_status launch_qgemm_blk(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, cudaStream_t st) {
+    using S = SsSmem<false>;
+    const int64_t K = w.K, N = w.N;
+    const BlobLayout L = blob_layout(N, K);
+    const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
+    CUtensorMap tmA, tmW, tmY;
+    if (!make_byte_map(&tmA, codes, (uint64_t)K, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B)) return DVDQ_ERR_CUDA;
+    if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, S::BNh,
+                       CU_TENSOR_MAP_SWIZZLE_NONE))
+        return DVDQ_ERR_CUDA;
+    if (!make_out_map32(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)) return DVDQ_ERR_CUDA;
+    if (!fat_kernel_registers_fit(qgemm_blk_kernel)) return DVDQ_ERR_CUDA;
+    static PerDevice<int> cache;
+    const int max_pairs = resident_pairs(cache, qgemm_blk_kernel, kFatThreads, S::kTotal);
+    if (max_pairs == 0) return DVDQ_ERR_CUDA;
+    const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + S::BN - 1) / S::BN);
+    const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
+    qgemm_blk_kernel<<<2 * pairs, kFatThreads, S::kTotal, st>>>(tmA, tmW, tmY, scales, sums,
+                                                                reinterpret_cast<const float*>(blob + L.delta_offset),
+                                                                reinterpret_cast<const int32_t*>(blob + L.zc_offset),
+                                                                static_cast<const __nv_bfloat16*>(bias), (int)M, (int)N, (int)K, act, spr);
+    return cuda_status(cudaGetLastError());
+}
+
+}  // namespace dvdq

@@ -206,18 +206,29 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 // Two k-blocks per trip.  An accumulator covers KBG k-blocks (a power of two, or the
                 // whole of K): with KBG = 1 the two blocks of a trip go to different accumulators.
                 int kin = 0;  // k-blocks issued into the accumulator in use
+                if constexpr (!BLK) {
+                    acquire();  // one accumulator per tile
+                    if (!ok) break;
+                }
                 for (int kb = 0; ok && kb < KB; kb += 2) {
                     uint32_t acc_h[2];
                     bool first_h[2], last_h[2];
+                    if constexpr (BLK) {
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        first_h[h] = kin == 0;
-                        if (first_h[h]) acquire();
-                        acc_h[h] = acc;
-                        last_h[h] = ++kin == KBG;
-                        if (last_h[h]) kin = 0;
+                        for (int h = 0; h < 2; ++h) {
+                            first_h[h] = kin == 0;
+                            if (first_h[h]) acquire();
+                            acc_h[h] = acc;
+                            last_h[h] = ++kin == KBG;
+                            if (last_h[h]) kin = 0;
+                        }
+                        if (!ok) break;
+                    } else {
+                        acc_h[0] = acc_h[1] = acc;
+                        first_h[0] = kb == 0;
+                        first_h[1] = last_h[0] = false;
+                        last_h[1] = kb + 2 >= KB;
                     }
-                    if (!ok) break;
                     // the activation ring may have an odd number of stages: its second stage of the trip can wrap
                     const uint32_t sa1 = sa + 1 == kSsAStages ? 0u : sa + 1, pa1 = sa + 1 == kSsAStages ? pa ^ 1u : pa;
                     if (!mbar_wait_warp(a_ready(sa), pa, abort_flag, kWaitPackedFull)) { ok = false; break; }
@@ -511,7 +522,6 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 for (int jw = 0; jw < 4; ++jw) { e[it][jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[it][jw] = w[jw] & 0xF0F0F0F0u; }
             }
             loaded &= rt_zero;
-            fence_loads_done();
             __syncwarp();
             if (lane == 0) mbar_arrive_after_loads(wp_empty(pst), loaded);  // the packed rows are in registers
             if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
@@ -609,12 +619,6 @@ static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const
     const bool wide_epilogue = w.K <= 2048 || (act != 0 && w.K <= 6144);
     return wide_epilogue ? launch_qgemm_ss_t<RAW, 8, false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
                          : launch_qgemm_ss_t<RAW, 4, false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
-}
-
-// Block-wise activation scales (scale_group = 1024), bf16 output.
-static dvdq_status launch_qgemm_ss_blk(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
-                                       const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, cudaStream_t st) {
-    return launch_qgemm_ss_t<false, 8, true>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, nullptr, 0, st);
 }
 
 }  // namespace dvdq
