@@ -203,6 +203,29 @@ dvdq_status dvdq_qgemm(const void* codes, const float* scales, const int32_t* co
                        const void* bias_bf16, int32_t act, void* Y_bf16, int64_t ldy,
                        void* cuda_stream);
 
+/* ---- (2) of one layer fused with (1) of the next: Eq. 10 applied layer after layer --------
+ *
+ * Where one quantized layer feeds another (Y of this layer is X of the next, Eq. 10 for both),
+ * the bf16 output need not exist: this call runs dvdq_qgemm's contraction and epilogue
+ * arithmetic (same roundings: bf16, optional tanh-GELU, bf16 again) and then, inside the same
+ * kernel, the next layer's activation transform on those bf16 values: x~ = y R with
+ * R = I (x) H_256 / 16, one absmax scale per token and per 256 rotated channels, codes
+ * c = round_half_even(x~ / s).  It writes what dvdq_rotate_quantize would write for Y:
+ *
+ *   q           this layer's quantizer: scale_group = 0 and container_bits = 8 (or bits = 8)
+ *   q_next      the next layer's: rot_block = 256, scale_group = 256, container_bits = 8,
+ *               bits 4, 6 or 8; the next layer's weights must be rotated with B = 256
+ *   codes_next      [M, N] one int8 per code (dvdq_act_codes_bytes_q(M, N, q_next) bytes)
+ *   scales_next     [M, N / 256] fp32,  code_sums_next [M, N / 256] int32
+ *   Y_bf16_or_null  if not NULL, the bf16 output [M, N] (row pitch ldy) is written as well
+ * N % 256 == 0 (a 256-wide tile of the GEMM owns whole rotation blocks and scale groups of its
+ * rows, which is what makes the fusion possible).  Other options give DVDQ_ERR_UNSUPPORTED. */
+dvdq_status dvdq_qgemm_fused_rq(const void* codes, const float* scales, const int32_t* code_sums,
+                                int64_t M, const dvdq_act_quant* q, const dvdq_weights* w /* host */,
+                                const void* bias_bf16, int32_t act, const dvdq_act_quant* q_next,
+                                void* codes_next, float* scales_next, int32_t* code_sums_next,
+                                void* Y_bf16_or_null, int64_t ldy, void* cuda_stream);
+
 /* ---- (1)+(2): one quantized linear layer ------------------------------------------
  * workspace: dvdq_qlinear_workspace_bytes(M, K, q) bytes, 256-byte aligned. */
 dvdq_status dvdq_qlinear(const void* X_bf16, int64_t M, int64_t ldx, const dvdq_act_quant* q,

@@ -22,7 +22,7 @@ OK, ERR_NULL, ERR_SHAPE, ERR_BITS, ERR_ROT_BLOCK, ERR_ALIGN, ERR_WORKSPACE, ERR_
 EXPORTS = [
     "dvdq_status_string", "dvdq_version", "dvdq_act_codes_bytes", "dvdq_act_codes_bytes_q", "dvdq_act_scales_count", "dvdq_weight_blob_bytes",
     "dvdq_qlinear_workspace_bytes", "dvdq_rotate_quantize", "dvdq_pack_weights", "dvdq_qgemm",
-    "dvdq_qlinear", "dvdq_qlinear_static", "dvdq_qgemm_int32", "dvdq_pack_act_codes", "dvdq_unpack_act_codes",
+    "dvdq_qlinear", "dvdq_qlinear_static", "dvdq_qgemm_fused_rq", "dvdq_qgemm_int32", "dvdq_pack_act_codes", "dvdq_unpack_act_codes",
     "dvdq_unpack_weights", "dvdq_last_device_status",
     "dvdq_rotate_weights", "dvdq_quantize_weights_symmetric", "dvdq_int8_mma_ceiling", "dvdq_debug_wait_timeout",
     "dvdq_bgr_quantize", "dvdq_gbs_l1_terms", "dvdq_gbs_init", "dvdq_gbs_next_bits", "dvdq_gbs_observe",
@@ -91,6 +91,7 @@ def load():
         "dvdq_qlinear": (C.c_int, [p, i64, i64, aq, wp, p, i32, p, i64, p, sz, p]),
         "dvdq_qlinear_static": (C.c_int, [p, i64, i64, aq, wp, p, i32, p, i64, p]),
         "dvdq_qgemm_int32": (C.c_int, [p, p, i64, aq, wp, p, i64, p]),
+        "dvdq_qgemm_fused_rq": (C.c_int, [p, p, p, i64, aq, wp, p, i32, aq, p, p, p, p, i64, p]),
         "dvdq_pack_act_codes": (C.c_int, [p, i64, i64, aq, p, p, p]),
         "dvdq_unpack_act_codes": (C.c_int, [p, i64, i64, aq, p, p]),
         "dvdq_unpack_weights": (C.c_int, [wp, p, p, p, p]),
@@ -202,6 +203,21 @@ def dvdq_qgemm(codes: torch.Tensor, scales: torch.Tensor, code_sums: torch.Tenso
                              _ptr(code_sums, torch.int32, "code_sums"), M, C.byref(q), C.byref(w),
                              _ptr(bias, torch.bfloat16, "bias"), act, _ptr(Y, torch.bfloat16, "Y"), ldy,
                              _stream(stream)), "dvdq_qgemm")
+
+
+def dvdq_qgemm_fused_rq(codes: torch.Tensor, scales: torch.Tensor, code_sums: torch.Tensor, M: int, q: ActQuant,
+                        w: Weights, bias: Optional[torch.Tensor], act: int, q_next: ActQuant, codes_next: torch.Tensor,
+                        scales_next: torch.Tensor, code_sums_next: torch.Tensor, Y: Optional[torch.Tensor] = None,
+                        stream=None) -> None:
+    """dvdq_qgemm whose epilogue writes the next layer's codes / scales / code sums
+    (rot_block = scale_group = 256, one int8 per code) instead of bf16; Y, if given, also gets the bf16 output."""
+    ldy = _row_major(Y, "Y") if Y is not None else 0
+    _check(load().dvdq_qgemm_fused_rq(_ptr(codes, torch.uint8, "codes"), _ptr(scales, torch.float32, "scales"),
+                                      _ptr(code_sums, torch.int32, "code_sums"), M, C.byref(q), C.byref(w),
+                                      _ptr(bias, torch.bfloat16, "bias"), act, C.byref(q_next),
+                                      _ptr(codes_next, torch.uint8, "codes_next"), _ptr(scales_next, torch.float32, "scales_next"),
+                                      _ptr(code_sums_next, torch.int32, "code_sums_next"), _ptr(Y, torch.bfloat16, "Y"), ldy,
+                                      _stream(stream)), "dvdq_qgemm_fused_rq")
 
 
 def dvdq_qlinear(X: torch.Tensor, q: ActQuant, w: Weights, bias: Optional[torch.Tensor], act: int,

@@ -245,6 +245,36 @@ dvdq_status dvdq_qgemm(const void* codes, const float* scales, const int32_t* co
     return launch_qgemm(codes, scales, code_sums, M, *q, *w, bias, act, Y, ldy, nullptr, 0, (cudaStream_t)stream);
 }
 
+dvdq_status dvdq_qgemm_fused_rq(const void* codes, const float* scales, const int32_t* code_sums, int64_t M,
+                                const dvdq_act_quant* q, const dvdq_weights* w, const void* bias, int32_t act,
+                                const dvdq_act_quant* q_next, void* codes_next, float* scales_next, int32_t* code_sums_next,
+                                void* Y_or_null, int64_t ldy, void* stream) {
+    dvdq_status s = check_gemm_args(codes, code_sums, M, q, w);
+    if (s != DVDQ_OK) return s;
+    if (act != 0 && act != 1) return DVDQ_ERR_UNSUPPORTED;
+    // this layer: per-token scales, codes one int8 each; the next layer: N input channels in whole
+    // 256-blocks, rotation block = scale group = 256 (what one 256-wide tile owns), codes one int8 each
+    if (q->scale_group != 0 || storage_bits(*q) != 8) return DVDQ_ERR_UNSUPPORTED;
+    if (!q_next) return DVDQ_ERR_NULL;
+    if (w->N % 256 != 0 || validate_k(w->N) != DVDQ_OK) return DVDQ_ERR_SHAPE;
+    if ((s = validate_act_quant(q_next, w->N)) != DVDQ_OK) return s;
+    if (q_next->rot_block != 256 || q_next->scale_group != 256 || q_next->container_bits != 8) return DVDQ_ERR_UNSUPPORTED;
+    if (Y_or_null && (ldy < w->N || ldy % 8 != 0)) return DVDQ_ERR_SHAPE;
+    if (M == 0) return DVDQ_OK;
+    if (!scales || !codes_next || !scales_next || !code_sums_next) return DVDQ_ERR_NULL;
+    if (!aligned(scales, 4) || !aligned(codes_next, 16) || !aligned(scales_next, 4) || !aligned(code_sums_next, 4) ||
+        (Y_or_null && !aligned(Y_or_null, 16)) || (bias && !aligned(bias, 2)))
+        return DVDQ_ERR_ALIGN;
+    FusedOut fo;
+    fo.codes = static_cast<uint8_t*>(codes_next);
+    fo.scales = scales_next;
+    fo.sums = code_sums_next;
+    fo.y_dbg = static_cast<__nv_bfloat16*>(Y_or_null);
+    fo.ldy = ldy;
+    fo.bits = q_next->bits;
+    return launch_qgemm_fused(codes, scales, code_sums, M, *w, bias, act, fo, (cudaStream_t)stream);
+}
+
 dvdq_status dvdq_qgemm_int32(const void* codes, const int32_t* code_sums, int64_t M, const dvdq_act_quant* q,
                              const dvdq_weights* w, int32_t* acc_out, int64_t ldacc, void* stream) {
     dvdq_status s = check_gemm_args(codes, code_sums, M, q, w);

@@ -18,6 +18,14 @@
 //   warps 4-11   widen weight codes into the operand stages (two groups, alternate k-blocks)
 //   warps 12-19  epilogue: warp w reads tensor-memory lanes 32 * (w % 4).., columns 128 * ((w - 12) / 4)..
 // Every wait is bounded, as in qgemm.cuh.
+//
+// The same skeleton carries the FUSED variant (kFatFuse): a layer with per-token input scales whose
+// epilogue does not write bf16 but applies the NEXT layer's activation transform (Eq. 10 for the
+// layer that consumes this output): rotate by H_256, one absmax scale per token and 256 channels,
+// round to codes, one int8 each.  A 256-wide tile holds whole rotation blocks and whole scale
+// groups of its rows, so nothing leaves the tile: a thread owns one row and 128 columns, does the
+// butterflies of seven index bits in registers, and meets the thread that owns the row's other
+// 128 columns through the (already drained) accumulator columns in tensor memory for the eighth.
 #pragma once
 
 #include "qgemm_ss.cuh"
@@ -39,11 +47,26 @@ __device__ __forceinline__ void regs_take() { asm volatile("setmaxnreg.inc.sync.
 template <int N>
 __device__ __forceinline__ void regs_give() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
 
+constexpr int kFatBlk = 0, kFatFuse = 1;
+
+// What the fused epilogue writes: the next layer's codes (one int8 each, row pitch N bytes),
+// scales and code sums [M, N / 256], and, if y_dbg is not null, the bf16 layer output it never
+// needs itself (for tests).
+struct FusedOut {
+    uint8_t* codes;
+    float* scales;
+    int32_t* sums;
+    __nv_bfloat16* y_dbg;
+    int64_t ldy;
+    int bits;
+};
+
+template <int MODE>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFatThreads, 1)
-qgemm_blk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                  const __grid_constant__ CUtensorMap tmY, const float* __restrict__ scales,
                  const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
-                 const __nv_bfloat16* __restrict__ bias, int M, int N, int K, int act, int spr) {
+                 const __nv_bfloat16* __restrict__ bias, int M, int N, int K, int act, int spr, const FusedOut fo) {
     using S = SsSmem<false>;
     constexpr int BN = S::BN, BNh = S::BNh;
     extern __shared__ uint8_t smem_raw[];
@@ -266,6 +289,7 @@ qgemm_blk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
     } else {
         regs_take<kFatRegsEpilogue>();
+        if constexpr (MODE == kFatBlk) {
         // ------------------------------------------------------------ epilogue: running sum over groups in registers
         const int q = warp & 3;                                   // tensor-memory lane quarter this warp may read
         const int half = (warp - kFatFirstEpilogueWarp) >> 2;     // which 128 of the tile's 256 columns
@@ -376,6 +400,158 @@ qgemm_blk_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         if (lane == 0) tma_store_wait_all();
         __syncwarp();
+    
+        } else {
+        // ------------------------------------------------------------ epilogue: the next layer's rotate-quantize
+        const int q = warp & 3;
+        const int half = (warp - kFatFirstEpilogueWarp) >> 2;
+        const int ew = 4 * half + q;
+        constexpr int CW = BN / 2;
+        const uint32_t c_delta = sbase + S::kConstOff + ew * (3 * CW * 4);
+        const uint32_t c_zc = c_delta + CW * 4;
+        const uint32_t c_bias = c_zc + CW * 4;
+        // exchange slots of the thread pairs (the staging buffers of the bf16 path are not used here)
+        float* x_max = reinterpret_cast<float*>(smem + S::kStageOutOff) + ew * 32;
+        int* x_sum = reinterpret_cast<int*>(smem + S::kStageOutOff + 8 * 32 * 4) + ew * 32;
+        const int pw = (ew ^ 4) - ew;  // the partner's slots are pw * 32 entries away
+        constexpr int kShift = 4;
+        constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23
+        const float qmax = (float)((1 << (fo.bits - 1)) - 1);
+        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+        const int gpr = N / BN;  // scale groups per token in the output
+        uint32_t lt = 0;
+        for (int tile = pair; tile < num_tiles; tile += num_pairs, ++lt) {
+            const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
+            const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM, nt = tile % num_n, n0 = nt * BN + half * CW;
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < CW / 32; ++i) {
+                const int c = lane + 32 * i, n = n0 + c;
+                sts32f(c_delta + 4 * c, __ldg(delta + n));
+                sts32f(c_zc + 4 * c, (float)__ldg(zc + n));
+                sts32f(c_bias + 4 * c, bias != nullptr ? __bfloat162float(bias[n]) : 0.f);
+            }
+            __syncwarp();
+            const int row = m0 + q * 32 + lane;
+            const bool row_ok = row < M;
+            const float s_i = row_ok ? scales[row] : 0.f;
+            const float S_f = row_ok ? (float)sums[row] : 0.f;
+            const float s_k = s_i * (1.0f / (float)(1 << kShift)), nS_k = -S_f * (float)(1 << kShift);
+            if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) break;
+            tc_fence_after();
+            const uint32_t own = tmem_base + a * BN + half * CW + lane_addr, theirs = tmem_base + a * BN + (half ^ 1) * CW + lane_addr;
+            // ---- this layer's output, as the bf16 values the next layer is defined on; the butterfly
+            // of index bit 0 on the way into the pairs (2i, 2i + 1)
+            uint64_t v[CW / 2];
+#pragma unroll
+            for (int c = 0; c < CW / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32(own + c * 32, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    const float4 dl = lds128f(c_delta + 4 * (c * 32 + j)), zz = lds128f(c_zc + 4 * (c * 32 + j)), bb = lds128f(c_bias + 4 * (c * 32 + j));
+                    const float d4[4] = {dl.x, dl.y, dl.z, dl.w}, z4[4] = {zz.x, zz.y, zz.z, zz.w}, b4[4] = {bb.x, bb.y, bb.z, bb.w};
+                    float y[4];
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        y[t] = fmaf(fmaf(z4[t], nS_k, (float)(int32_t)r[j + t]), d4[t] * s_k, b4[t]);
+                        y[t] = __bfloat162float(__float2bfloat16_rn(y[t]));
+                        if (act == 1) y[t] = __bfloat162float(__float2bfloat16_rn(gelu_tanh_f32(y[t])));
+                    }
+                    if (fo.y_dbg != nullptr && row_ok) {
+                        __nv_bfloat162 p0 = __floats2bfloat162_rn(y[0], y[1]), p1 = __floats2bfloat162_rn(y[2], y[3]);
+                        *reinterpret_cast<uint2*>(fo.y_dbg + (int64_t)row * fo.ldy + n0 + c * 32 + j) =
+                            make_uint2(*reinterpret_cast<uint32_t*>(&p0), *reinterpret_cast<uint32_t*>(&p1));
+                    }
+                    v[(c * 32 + j) / 2] = f2_pack(y[0] + y[1], y[0] - y[1]);
+                    v[(c * 32 + j) / 2 + 1] = f2_pack(y[2] + y[3], y[2] - y[3]);
+                }
+            }
+            // ---- index bits 1..6: butterflies between register pairs
+#pragma unroll
+            for (int st = 1; st < CW / 2; st <<= 1)
+#pragma unroll
+                for (int i = 0; i < CW / 2; ++i)
+                    if ((i & st) == 0) f2_butterfly(v[i], v[i + st]);
+            // ---- index bit 7: the two threads of a row swap their halves through the accumulator's
+            // columns (every value of it is in registers by now) and take sum or difference
+#pragma unroll
+            for (int c = 0; c < CW / 32; ++c) {
+                uint32_t r[32];
+#pragma unroll
+                for (int t = 0; t < 16; ++t) {
+                    float lo, hi;
+                    f2_unpack(v[c * 16 + t], lo, hi);
+                    r[2 * t] = __float_as_uint(lo);
+                    r[2 * t + 1] = __float_as_uint(hi);
+                }
+                tmem_st_32x32(own + c * 32, r);
+            }
+            tmem_st_wait();
+            tc_fence_before();
+            asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory");  // the two warps of this lane quarter
+            tc_fence_after();
+            const uint64_t sgn = half ? f2_pack(-1.f, -1.f) : f2_pack(1.f, 1.f);
+#pragma unroll
+            for (int c = 0; c < CW / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32(theirs + c * 32, r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int t = 0; t < 16; ++t)  // half 0: own + theirs; half 1: theirs - own
+                    v[c * 16 + t] = f2_fma(v[c * 16 + t], sgn, f2_pack(__uint_as_float(r[2 * t]), __uint_as_float(r[2 * t + 1])));
+            }
+            // both halves are read: the MMA warp may have the accumulator back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty(a), 0));
+            // ---- absmax of the 256 rotated channels (of the un-normalised transform)
+            float amax = 0.f;
+#pragma unroll
+            for (int i = 0; i < CW / 2; ++i) {
+                float lo, hi;
+                f2_unpack(v[i], lo, hi);
+                amax = fmaxf(amax, fmaxf(fabsf(lo), fabsf(hi)));
+            }
+            x_max[lane] = amax;
+            asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory");
+            amax = fmaxf(amax, x_max[pw * 32 + lane]);
+            const float inv = amax > 0.f ? qmax / amax : 0.f;
+            const uint64_t inv2 = f2_pack(inv, inv), magic2 = f2_pack(kMagic, kMagic);
+            // ---- quantize and store: per 8 channels the four even ones, then the four odd ones
+            uint8_t* crow = fo.codes + (int64_t)row * N + n0;
+            int lsum = 0;
+#pragma unroll
+            for (int k16 = 0; k16 < CW / 16; ++k16) {
+                uint32_t w[4];
+#pragma unroll
+                for (int k8 = 0; k8 < 2; ++k8) {
+                    uint32_t b[8];
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        float lo, hi;
+                        f2_unpack(f2_fma(v[k16 * 8 + k8 * 4 + t], inv2, magic2), lo, hi);
+                        b[2 * t] = __float_as_uint(lo);
+                        b[2 * t + 1] = __float_as_uint(hi);
+                    }
+                    const uint32_t E = __byte_perm(__byte_perm(b[0], b[2], 0x0040), __byte_perm(b[4], b[6], 0x0040), 0x5410);
+                    const uint32_t O = __byte_perm(__byte_perm(b[1], b[3], 0x0040), __byte_perm(b[5], b[7], 0x0040), 0x5410);
+                    lsum = __dp4a((int)E, 0x01010101, lsum);
+                    lsum = __dp4a((int)O, 0x01010101, lsum);
+                    w[2 * k8] = E;
+                    w[2 * k8 + 1] = O;
+                }
+                if (row_ok) *reinterpret_cast<uint4*>(crow + k16 * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            x_sum[lane] = lsum;
+            asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory");
+            if (half == 0 && row_ok) {
+                fo.scales[(int64_t)row * gpr + nt] = (amax * (1.0f / 16.0f)) / qmax;  // s = (absmax / sqrt(256)) / qmax
+                fo.sums[(int64_t)row * gpr + nt] = lsum + x_sum[pw * 32 + lane];
+            }
+        }
+        }
     }
 
     tc_fence_before();
@@ -407,16 +583,42 @@ static dvdq_status launch_qgemm_blk(const void* codes, const float* scales, cons
                        CU_TENSOR_MAP_SWIZZLE_NONE))
         return DVDQ_ERR_CUDA;
     if (!make_out_map32(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)) return DVDQ_ERR_CUDA;
-    if (!fat_kernel_registers_fit(qgemm_blk_kernel)) return DVDQ_ERR_CUDA;
+    auto kern = qgemm_fat_kernel<kFatBlk>;
+    if (!fat_kernel_registers_fit(kern)) return DVDQ_ERR_CUDA;
     static PerDevice<int> cache;
-    const int max_pairs = resident_pairs(cache, qgemm_blk_kernel, kFatThreads, S::kTotal);
+    const int max_pairs = resident_pairs(cache, kern, kFatThreads, S::kTotal);
     if (max_pairs == 0) return DVDQ_ERR_CUDA;
     const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + S::BN - 1) / S::BN);
     const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
-    qgemm_blk_kernel<<<2 * pairs, kFatThreads, S::kTotal, st>>>(tmA, tmW, tmY, scales, sums,
-                                                                reinterpret_cast<const float*>(blob + L.delta_offset),
-                                                                reinterpret_cast<const int32_t*>(blob + L.zc_offset),
-                                                                static_cast<const __nv_bfloat16*>(bias), (int)M, (int)N, (int)K, act, spr);
+    kern<<<2 * pairs, kFatThreads, S::kTotal, st>>>(tmA, tmW, tmY, scales, sums, reinterpret_cast<const float*>(blob + L.delta_offset),
+                                                    reinterpret_cast<const int32_t*>(blob + L.zc_offset),
+                                                    static_cast<const __nv_bfloat16*>(bias), (int)M, (int)N, (int)K, act, spr, FusedOut{});
+    return cuda_status(cudaGetLastError());
+}
+
+// The layer (per-token input scales, codes one int8 each) whose epilogue writes the next layer's
+// codes, scales and code sums for rot_block = scale_group = 256 instead of bf16.
+static dvdq_status launch_qgemm_fused(const void* codes, const float* scales, const int32_t* sums, int64_t M,
+                                      const dvdq_weights& w, const void* bias, int act, const FusedOut& fo, cudaStream_t st) {
+    using S = SsSmem<false>;
+    const int64_t K = w.K, N = w.N;
+    const BlobLayout L = blob_layout(N, K);
+    const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
+    CUtensorMap tmA, tmW;
+    if (!make_byte_map(&tmA, codes, (uint64_t)K, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B)) return DVDQ_ERR_CUDA;
+    if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, S::BNh,
+                       CU_TENSOR_MAP_SWIZZLE_NONE))
+        return DVDQ_ERR_CUDA;
+    auto kern = qgemm_fat_kernel<kFatFuse>;
+    if (!fat_kernel_registers_fit(kern)) return DVDQ_ERR_CUDA;
+    static PerDevice<int> cache;
+    const int max_pairs = resident_pairs(cache, kern, kFatThreads, S::kTotal);
+    if (max_pairs == 0) return DVDQ_ERR_CUDA;
+    const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * (N / S::BN);
+    const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
+    kern<<<2 * pairs, kFatThreads, S::kTotal, st>>>(tmA, tmW, tmA /* unused */, scales, sums, reinterpret_cast<const float*>(blob + L.delta_offset),
+                                                    reinterpret_cast<const int32_t*>(blob + L.zc_offset),
+                                                    static_cast<const __nv_bfloat16*>(bias), (int)M, (int)N, (int)K, act, 1, fo);
     return cuda_status(cudaGetLastError());
 }
 
