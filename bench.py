@@ -188,6 +188,7 @@ def config_of(wl, args):
             "l2_policy": "inputs larger than L2 (every layer streams >= 400 MB)",
             "act_codes": ("one int8 per code" if args.container else "packed, b bits per code"),
             "act_scales": (f"one per token and block of {args.scale_group} channels" if args.scale_group else "one per token"),
+            "fused": bool(getattr(args, "fuse", False) and wl.chain),
             "parallelism": f"dp{args.gpus} (token-sharded replicas, no collective)"}
 
 
@@ -204,8 +205,11 @@ class Leg:
     and the GEMM for every layer (what dvdq_qlinear runs), optionally with CUDA events around
     every launch."""
 
-    def __init__(self, B, W, wl, args, container, dev, rank, shared=None):
+    def __init__(self, B, W, wl, args, container, dev, rank, shared=None, fuse=False):
         self.B, self.wl, self.container, self.scale_group = B, wl, container, args.scale_group
+        self.fuse = fuse and wl.chain   # every layer but the last writes the next layer's codes instead of bf16
+        if self.fuse and (container != 8 or args.scale_group != 0):
+            raise SystemExit("--fuse needs --container 8 and per-token scales on the first layer")
         M = self.M = wl.M
         if shared is None:
             xs = {}
@@ -217,7 +221,8 @@ class Leg:
             for i, layer in enumerate(wl.layers):
                 u, d, z = W.make_weight_codes(layer, seed=i, device=dev)
                 blob = torch.empty(B.dvdq_weight_blob_bytes(layer.N, layer.K), dtype=torch.uint8, device=dev)
-                weights.append((B.dvdq_pack_weights(u, d, z, layer.rot_block, blob), blob, W.make_bias(wl, layer, device=dev)))
+                rot = 256 if (self.fuse and i > 0) else layer.rot_block   # recorded in the blob: what the activations are rotated with
+                weights.append((B.dvdq_pack_weights(u, d, z, rot, blob), blob, W.make_bias(wl, layer, device=dev)))
                 del u
             Ys = [torch.empty(M, layer.N, dtype=torch.bfloat16, device=dev) for layer in wl.layers]
             shared = dict(xs=xs, weights=weights, Ys=Ys)
@@ -225,6 +230,8 @@ class Leg:
         self.layers = []
         for i, layer in enumerate(wl.layers):
             q = B.ActQuant(layer.bits, layer.rot_block, args.scale_group, container)
+            if self.fuse and i > 0:
+                q = B.ActQuant(layer.bits, 256, 256, 8)   # what the fused epilogue of the layer before produces
             n_scales = B.dvdq_act_scales_count(M, layer.K, q)
             if n_scales == 0:
                 raise SystemExit(f"layer {layer.K}->{layer.N}: activation quantizer options not supported")
@@ -238,17 +245,27 @@ class Leg:
 
     def step(self, events=None, rq_only=False):
         B = self.B
+        n = len(self.layers)
         for li, L in enumerate(self.layers):
             if events is not None:
                 events[li][0].record()
-            B.dvdq_rotate_quantize(L["x"], L["q"], L["codes"], L["scales"], L["sums"])
+            if not (self.fuse and li > 0):
+                B.dvdq_rotate_quantize(L["x"], L["q"], L["codes"], L["scales"], L["sums"])
             if events is not None:
                 events[li][1].record()
             if rq_only:
                 continue
-            B.dvdq_qgemm(L["codes"], L["scales"], L["sums"], self.M, L["q"], L["w"], L["bias"], L["layer"].act, L["Y"])
+            if self.fuse and li + 1 < n:
+                nx = self.layers[li + 1]
+                B.dvdq_qgemm_fused_rq(L["codes"], L["scales"], L["sums"], self.M, L["q"], L["w"], L["bias"], L["layer"].act,
+                                      nx["q"], nx["codes"], nx["scales"], nx["sums"])
+            else:
+                B.dvdq_qgemm(L["codes"], L["scales"], L["sums"], self.M, L["q"], L["w"], L["bias"], L["layer"].act, L["Y"])
             if events is not None:
                 events[li][2].record()
+
+    def launches_per_step(self):
+        return 2 * len(self.layers) - (len(self.layers) - 1 if self.fuse else 0)
 
     def timed(self, steps, warmup, barrier, rq_only=False):
         """(ms per step, per-layer rq ms, per-layer GEMM ms) from CUDA events inside the timed region."""
@@ -295,8 +312,10 @@ def roofline_blocks(leg, ms_per_step, rq_ms, gm_ms, args, peaks, ceiling, timed_
     """The two roofline objects of a leg (GEMM: tensor-bound; rotate-quantize: HBM-bound) and its stages."""
     M, layers, sg, cont = leg.M, leg.layers, leg.scale_group, leg.container
     gemm_tops = sum(layer_ops(M, L["layer"]) for L in layers) / (sum(gm_ms) * 1e-3) / 1e12
-    alg = sum(rq_algorithmic_bytes(M, L["layer"], sg) for L in layers)
-    stored = sum(rq_stored_bytes(M, L["layer"], sg, cont) for L in layers)
+    has_rq = [not (leg.fuse and li > 0) for li in range(len(layers))]   # fused: only the first layer launches rotate-quantize
+    alg = sum(rq_algorithmic_bytes(M, L["layer"], sg) for L, h in zip(layers, has_rq) if h)
+    stored = sum(rq_stored_bytes(M, L["layer"], sg, cont) for L, h in zip(layers, has_rq) if h)
+    rq_ms = [t if h else 0.0 for t, h in zip(rq_ms, has_rq)]
     rq_gbs = alg / (sum(rq_ms) * 1e-3) / 1e9
     # which library figure a GEMM timed like this compares with: the burst one for a region well under a second
     bf16_kind = "bf16_tflops" if timed_s < 1.0 else "bf16_tflops_sustained"
@@ -315,13 +334,17 @@ def roofline_blocks(leg, ms_per_step, rq_ms, gm_ms, args, peaks, ceiling, timed_
                "frac_of_nominal_8000": rq_gbs / NOMINAL_HBM_GBS,
                "bytes": "algorithmic: 2K + K b/8 + 8 per token and scale group",
                "stored_bytes_gbs": stored / (sum(rq_ms) * 1e-3) / 1e9,
-               "avg_launch_ms": sum(rq_ms) / len(rq_ms), "traffic": RQ_DRAM_TRAFFIC_PER_LAUNCH.get(cont) if args.default_workload else None}
+               "avg_launch_ms": sum(rq_ms) / sum(has_rq), "traffic": RQ_DRAM_TRAFFIC_PER_LAUNCH.get(cont) if args.default_workload else None}
     stages = []
     for li, L in enumerate(layers):
         layer = L["layer"]
-        stages.append({"layer": f"{layer.K}->{layer.N} A{layer.bits} B{layer.rot_block}" + (" gelu" if layer.act else "") + (" bias" if layer.bias else ""),
-                       "rq_ms": rq_ms[li], "rq_gbs": rq_algorithmic_bytes(M, layer, sg) / (rq_ms[li] * 1e-3) / 1e9,
-                       "rq_frac_of_hbm": rq_algorithmic_bytes(M, layer, sg) / (rq_ms[li] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        rq_g = rq_algorithmic_bytes(M, layer, sg) / (rq_ms[li] * 1e-3) / 1e9 if has_rq[li] else None
+        stages.append({"layer": f"{layer.K}->{layer.N} A{layer.bits} B{L['q'].rot_block}" + (f" G{L['q'].scale_group}" if L['q'].scale_group else "")
+                       + (" gelu" if layer.act else "") + (" bias" if layer.bias else "")
+                       + (" [epilogue = next layer's rotate-quantize]" if leg.fuse and li + 1 < len(layers) else "")
+                       + (" [codes from the previous GEMM's epilogue]" if not has_rq[li] else ""),
+                       "rq_ms": rq_ms[li] if has_rq[li] else None, "rq_gbs": rq_g,
+                       "rq_frac_of_hbm": rq_g / peaks["hbm_gbs"] if has_rq[li] else None,
                        "qgemm_ms": gm_ms[li], "qgemm_tops": layer_ops(M, layer) / (gm_ms[li] * 1e-3) / 1e12,
                        "qgemm_frac_of_peak": layer_ops(M, layer) / (gm_ms[li] * 1e-3) / 1e12 / peak})
     return roof, rq_roof, stages
@@ -339,7 +362,7 @@ def run_workload(args, wl, B, W, D, dist, dev, rank, local_rank, world, peaks, f
         if status != B.OK:
             raise SystemExit(f"device status {status} ({B.status_string(status)}), wait id {detail}")
 
-    leg = Leg(B, W, wl, args, args.container, dev, rank)
+    leg = Leg(B, W, wl, args, args.container, dev, rank, fuse=args.fuse)
     M = wl.M
     warm = max(args.warmup, 3)
     leg.timed(1, warm - 1, barrier)   # warm-up (and first-use set-up) outside the sampled region
@@ -362,7 +385,7 @@ def run_workload(args, wl, B, W, D, dist, dev, rank, local_rank, world, peaks, f
     roof, rq_roof, stages = roofline_blocks(leg, ms_per_step, rq_ms, gm_ms, args, peaks, ceiling, timed_s)
 
     out = {"value": value, "ms_per_step": ms_per_step, "roofline": roof, "roofline_rotate_quantize": rq_roof, "stages": stages,
-           "clocks": clocks, "gpu_launches": 2 * len(leg.layers) * args.steps, "ceiling": ceiling, "leg": leg}
+           "clocks": clocks, "gpu_launches": leg.launches_per_step() * args.steps, "ceiling": ceiling, "leg": leg}
     if not full:
         return out
 
@@ -376,7 +399,7 @@ def run_workload(args, wl, B, W, D, dist, dev, rank, local_rank, world, peaks, f
                             "note": "the same launches without the GEMMs between them"}
 
     # ---- the same step with the other code layout, as a full block of its own
-    if not args.no_other_layout and world == 1:
+    if not args.no_other_layout and world == 1 and not leg.fuse:
         other = 8 if args.container == 0 else 0
         leg2 = Leg(B, W, wl, args, other, dev, rank, shared=leg.shared)
         n2 = max(5, min(args.steps, 50))
@@ -562,6 +585,9 @@ def main():
     ap.add_argument("--no-ceiling", action="store_true", help="skip the int8 issue-loop ceiling (the roofline then falls back to 2 x bf16)")
     ap.add_argument("--scale-group", type=int, default=0,
                     help="0: one activation scale per token; 128, 256, 1024: one per token and group of that many channels")
+    ap.add_argument("--fuse", action="store_true",
+                    help="chain workloads: every layer but the last writes the next layer's codes from its epilogue "
+                         "(dvdq_qgemm_fused_rq, rotation block = scale group = 256) instead of bf16; needs --container 8")
     ap.add_argument("--bits", type=int, default=0, help="override the activation bit width of every layer (4, 6 or 8)")
     args = ap.parse_args()
     from paper_2505_18663_b200 import workloads as W

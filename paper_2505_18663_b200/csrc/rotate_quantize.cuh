@@ -66,7 +66,12 @@ __device__ __forceinline__ uint32_t stage_a_entry(int m, int s) {
 // same way and written out after the next iteration's barrier.  The slots rotate over three sets:
 // a warp's whole iteration is a chain of dependent steps, so the exchange is kept as short as
 // it can be (an atomic, the barrier, one broadcast load).
-template <int LOG2B, int BITS, bool FULL, bool SUB>
+// MODE: the reach of a scale.  kRqToken: one per token, the token's warps meet (more than one span
+// per token).  kRqSpan1024: one per warp span (a token of one span, or scale groups of 1024).
+// kRqSub: groups of 256 or 128 channels inside the span.
+constexpr int kRqToken = 0, kRqSpan1024 = 1, kRqSub = 2;
+
+template <int LOG2B, int BITS, bool FULL, int MODE>
 __global__ void __maxnreg__(80)  // two CTAs of 12 warps per SM
 rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
           uint8_t* __restrict__ codes, float* __restrict__ scales, int32_t* __restrict__ sums,
@@ -77,14 +82,14 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
     constexpr bool kRot = LOG2B > 0;
     constexpr int kLog2Span = LOG2B > 10 ? 10 : LOG2B;  // butterflies a warp does on its own span
     constexpr int kCross = 1 << (LOG2B > 10 ? LOG2B - 10 : 0);  // spans per rotation block
-    const int blockwise = scale_group != 0;
+    constexpr bool SUB = MODE == kRqSub;
+    constexpr bool team = MODE == kRqToken;  // the token's warps exchange absmax and code sums
     // BITS is the width a code is STORED in; the quantizer's own width may be smaller (codes kept in bytes)
     const float qmax = (float)((1 << (code_bits - 1)) - 1);
     constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23: ulp 1, so the fma rounds to an integer
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int tl = warp / spans, sp = warp - tl * spans;
     const int g = lane >> 2, t = lane & 3;
-    const bool team = !blockwise && spans > 1;  // the token's warps exchange absmax and code sums
     if (team) {
         if (threadIdx.x < 3 * kRqMaxWarps) {
             (&s_max[0][0])[threadIdx.x] = 0u;
@@ -405,17 +410,10 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
             continue;
         }
         lsum = __reduce_add_sync(0xFFFFFFFFu, lsum);
-        if (blockwise) {
+        if (!team) {  // the span's own scale: a token of one span, or one scale per 1024 channels
             if (lane == 0) {
                 scales[(int64_t)token * spans + sp] = (amax * rs) / qmax;
                 sums[(int64_t)token * spans + sp] = lsum;
-            }
-            continue;
-        }
-        if (!team) {  // a single span per token
-            if (lane == 0) {
-                scales[token] = (amax * rs) / qmax;
-                sums[token] = lsum;
             }
             continue;
         }
@@ -442,7 +440,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
     }
 }
 
-template <int LOG2B, int BITS, bool FULL, bool SUB>
+template <int LOG2B, int BITS, bool FULL, int MODE>
 static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t ldx, void* codes, float* scales,
                                     int32_t* sums, int scale_group, int code_bits, cudaStream_t st) {
     const int spans = (int)((K + kRqSpan - 1) / kRqSpan);
@@ -456,7 +454,7 @@ static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t
     const size_t smem = (size_t)warps * 256 * sizeof(float4);
     const int64_t groups = (M + tpc - 1) / tpc;
     if (M > 0x7FFFFF00ll || ldx > 0x7FFFFFFFll || groups * tpc > 0x7FFFFFFFll) return DVDQ_ERR_SHAPE;
-    auto kern = rq_kernel<LOG2B, BITS, FULL, SUB>;
+    auto kern = rq_kernel<LOG2B, BITS, FULL, MODE>;
     struct Setup {
         int sm_count;
         int blocks_per_sm[kRqMaxWarps + 1];
@@ -481,7 +479,7 @@ static dvdq_status launch_rq_kernel(const void* X, int64_t M, int64_t K, int64_t
     return cuda_status(cudaGetLastError());
 }
 
-template <int BITS, bool SUB>
+template <int BITS, int MODE>
 static dvdq_status launch_rq_bits(const void* X, int64_t M, int64_t K, int64_t ldx, int rot_block, void* codes,
                                   float* scales, int32_t* sums, int scale_group, int code_bits, cudaStream_t st) {
     int log2b = 0;
@@ -489,8 +487,8 @@ static dvdq_status launch_rq_bits(const void* X, int64_t M, int64_t K, int64_t l
     const bool full = K % kRqSpan == 0;
 #define DVDQ_RQ_CASE(L)                                                                              \
     case L:                                                                                          \
-        return full ? launch_rq_kernel<L, BITS, true, SUB>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st)  \
-                    : launch_rq_kernel<L, BITS, false, SUB>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st);
+        return full ? launch_rq_kernel<L, BITS, true, MODE>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st)  \
+                    : launch_rq_kernel<L, BITS, false, MODE>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st);
     switch (log2b) {
         DVDQ_RQ_CASE(0)
         DVDQ_RQ_CASE(6)
@@ -499,9 +497,9 @@ static dvdq_status launch_rq_bits(const void* X, int64_t M, int64_t K, int64_t l
         DVDQ_RQ_CASE(9)
         DVDQ_RQ_CASE(10)
         case 11:  // blocks of 2048 and 4096 channels are whole spans: K is a multiple of 1024
-            return full ? launch_rq_kernel<11, BITS, true, SUB>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st) : DVDQ_ERR_ROT_BLOCK;
+            return full ? launch_rq_kernel<11, BITS, true, MODE>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st) : DVDQ_ERR_ROT_BLOCK;
         case 12:
-            return full ? launch_rq_kernel<12, BITS, true, SUB>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st) : DVDQ_ERR_ROT_BLOCK;
+            return full ? launch_rq_kernel<12, BITS, true, MODE>(X, M, K, ldx, codes, scales, sums, scale_group, code_bits, st) : DVDQ_ERR_ROT_BLOCK;
         default:
             return DVDQ_ERR_ROT_BLOCK;
     }
@@ -512,11 +510,13 @@ inline dvdq_status launch_rotate_quantize(const void* X, int64_t M, int64_t K, i
                                           void* codes, float* scales, int32_t* sums, cudaStream_t st) {
     if (M == 0) return DVDQ_OK;
     const int sb = storage_bits(q);
-    const bool sub = q.scale_group != 0 && q.scale_group < kRqSpan;
-#define DVDQ_RQ_BITS(B)                                                                                                  \
-    if (sb == B)                                                                                                         \
-        return sub ? launch_rq_bits<B, true>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group, q.bits, st)  \
-                   : launch_rq_bits<B, false>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group, q.bits, st);
+    const int mode = (q.scale_group != 0 && q.scale_group < kRqSpan) ? kRqSub : (q.scale_group == 0 && K > kRqSpan) ? kRqToken : kRqSpan1024;
+#define DVDQ_RQ_BITS(B)                                                                                                       \
+    if (sb == B) {                                                                                                            \
+        if (mode == kRqSub) return launch_rq_bits<B, kRqSub>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group, q.bits, st);        \
+        if (mode == kRqToken) return launch_rq_bits<B, kRqToken>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group, q.bits, st);    \
+        return launch_rq_bits<B, kRqSpan1024>(X, M, K, ldx, q.rot_block, codes, scales, sums, q.scale_group, q.bits, st);                       \
+    }
     DVDQ_RQ_BITS(4)
     DVDQ_RQ_BITS(6)
     DVDQ_RQ_BITS(8)
