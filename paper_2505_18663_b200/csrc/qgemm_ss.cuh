@@ -40,11 +40,8 @@ constexpr int kSsFirstEpilogueWarp2 = kSsWProducerWarp + 1;  // a multiple of 4:
 static_assert(kSsFirstEpilogueWarp2 % 4 == 0, "lane quarters");
 static_assert(kSsStages % 2 == 0, "the MMA warp takes the weight stages in pairs");
 
-// BLK: block-wise activation scales (tile of 128 channels: two int32 accumulators and an fp32
-// running sum share tensor memory, as in qgemm.cuh).
-template <bool BLK>
 struct SsSmem {
-    static constexpr int BN = BLK ? 128 : kSsBN, BNh = BN / 2;
+    static constexpr int BN = kSsBN, BNh = BN / 2;
     static constexpr int kA = kBM * kBK;              // activation tile of one k-block (int8, swizzled)
     static constexpr int kW = BNh * kBK;              // widened weight half-tile
     static constexpr int kWPacked = BNh * kBK / 2;    // packed weight half-tile (64-byte rows)
@@ -54,7 +51,7 @@ struct SsSmem {
     static constexpr int kStageOutOff = kWPackedOff + kSsWPackedStages * kWPacked;  // 1024-byte aligned
     // 16 KB of staging and 12 KB of constants whether four or eight epilogue warps share them: one
     // buffer of 32 rows x 64 (or 32) bf16 each, and delta / zero-point rest / bias of 256 (or 128) columns
-    static constexpr int kStageOutBytes = (BLK ? 16 : 4) * 32 * 128;  // block-wise: eight warps, two buffers each
+    static constexpr int kStageOutBytes = 4 * 32 * 128;
     static constexpr int kConstOff = kStageOutOff + kStageOutBytes;
     static constexpr int kConstBytes = 4 * 3 * BN * 4;
     static constexpr int kBarOff = kConstOff + kConstBytes;
@@ -76,16 +73,15 @@ __device__ __forceinline__ void tc_mma_i8_ss_pair(uint32_t d_tmem, uint64_t a_de
         : "memory");
 }
 
-template <bool RAW, int EW, bool BLK>
+template <bool RAW, int EW>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((EW == 8 ? kSsFirstEpilogueWarp2 + 4 : kSsFirstEpilogueWarp2) * 32, 1)
 qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
                 const __grid_constant__ CUtensorMap tmY, const float* __restrict__ scales,
                 const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
                 const __nv_bfloat16* __restrict__ bias, int32_t* __restrict__ acc_out, int64_t ldacc,
                 int M, int N, int K, int act, int spr) {
-    using S = SsSmem<BLK>;
+    using S = SsSmem;
     constexpr int BN = S::BN, BNh = S::BNh;
-    static_assert(!(BLK && RAW), "block-wise scales: bf16 output only");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -96,10 +92,6 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int num_n = (N + BN - 1) / BN, num_m = (M + 2 * kBM - 1) / (2 * kBM);
     const int num_tiles = num_m * num_n;
     const int KB = 2 * ((K + 2 * kBK - 1) / (2 * kBK));  // even; a k-block past K reads zeros
-    // one accumulator per tile, or (block-wise scales) one per tile and scale group: spr groups of
-    // 128, 256 or 1024 codes per token, i.e. 1, 2 or 8 k-blocks per accumulator (K is a multiple of 256)
-    const int NG = BLK ? spr : 1;
-    const int KBG = BLK ? KB / spr : KB;  // k-blocks per accumulator
 
     const uint32_t bar0 = sbase + S::kBarOff;
     auto a_full = [&](int s) { return bar0 + 8u * s; };                          // this CTA's TMA copy of the stage
@@ -192,43 +184,15 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (rank == 0) {
             constexpr uint32_t idesc = umma_idesc_s8s8s32(2 * kBM, BN);
-            uint32_t st = 0, ph = 0, sa = 0, pa = 0, lt = 0;  // lt: accumulators started so far
-            uint32_t acc = 0;                                  // the accumulator in use (0 or 1)
+            uint32_t st = 0, ph = 0, sa = 0, pa = 0, lt = 0;
             bool ok = true;
-            // Starts the next accumulator once the epilogue has drained its previous contents.
-            auto acquire = [&]() {
-                acc = lt & 1u;
-                if (!mbar_wait_warp(acc_empty(acc), ((lt >> 1) & 1u) ^ 1u, abort_flag, kWaitAccEmpty)) ok = false;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs, ++lt) {
+                const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
+                if (!mbar_wait_warp(acc_empty(a), aph ^ 1u, abort_flag, kWaitAccEmpty)) { ok = false; break; }
                 tc_fence_after();
-                ++lt;
-            };
-            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-                // Two k-blocks per trip.  An accumulator covers KBG k-blocks (a power of two, or the
-                // whole of K): with KBG = 1 the two blocks of a trip go to different accumulators.
-                int kin = 0;  // k-blocks issued into the accumulator in use
-                if constexpr (!BLK) {
-                    acquire();  // one accumulator per tile
-                    if (!ok) break;
-                }
-                for (int kb = 0; ok && kb < KB; kb += 2) {
-                    uint32_t acc_h[2];
-                    bool first_h[2], last_h[2];
-                    if constexpr (BLK) {
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            first_h[h] = kin == 0;
-                            if (first_h[h]) acquire();
-                            acc_h[h] = acc;
-                            last_h[h] = ++kin == KBG;
-                            if (last_h[h]) kin = 0;
-                        }
-                        if (!ok) break;
-                    } else {
-                        acc_h[0] = acc_h[1] = acc;
-                        first_h[0] = kb == 0;
-                        first_h[1] = last_h[0] = false;
-                        last_h[1] = kb + 2 >= KB;
-                    }
+                const uint32_t d_tmem = tmem_base + a * BN;
+                // Two k-blocks per trip: every cycle between two issues is a bubble in the MMA stream
+                for (int kb = 0; kb < KB; kb += 2) {
                     // the activation ring may have an odd number of stages: its second stage of the trip can wrap
                     const uint32_t sa1 = sa + 1 == kSsAStages ? 0u : sa + 1, pa1 = sa + 1 == kSsAStages ? pa ^ 1u : pa;
                     if (!mbar_wait_warp(a_ready(sa), pa, abort_flag, kWaitPackedFull)) { ok = false; break; }
@@ -239,16 +203,15 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (elect_one()) {
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            const uint32_t d_tmem = tmem_base + acc_h[h] * BN;
                             const uint64_t adesc = umma_desc_sw128_kmajor(sbase + S::kAOff + (h ? sa1 : sa) * S::kA);
                             const uint64_t bdesc = umma_desc_sw128_kmajor(sbase + S::kWOff + (st + h) * S::kW);
 #pragma unroll
                             for (int k = 0; k < kBK / 32; ++k)  // +32 int8 along K = +2 in the 16-byte address field
-                                tc_mma_i8_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (first_h[h] && k == 0) ? 0u : 1u);
+                                tc_mma_i8_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | h | k) != 0 ? 1u : 0u);
                             tc_commit_pair(ops_empty(st + h), 3);
                             tc_commit_pair(a_empty(h ? sa1 : sa), 3);
-                            if (last_h[h]) tc_commit_pair(acc_full(acc_h[h]), 3);
                         }
+                        if (kb + 2 >= KB) tc_commit_pair(acc_full(a), 3);
                     }
                     __syncwarp();
                     st += 2;
@@ -269,113 +232,13 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const int half = warp >= kSsFirstEpilogueWarp2 ? 1 : 0;  // EW = 8: which 128 of the tile's 256 columns
         const int ew = 4 * half + q;
         constexpr int CW = BN / (EW / 4);           // columns per warp
-        constexpr int RB = (EW == 8 && !BLK) ? 64 : 128;  // bytes per row of the staging buffer = of a TMA store
+        constexpr int RB = EW == 8 ? 64 : 128;  // bytes per row of the staging buffer = of a TMA store
         const uint32_t c_delta = sbase + S::kConstOff + ew * (3 * CW * 4);  // shared addresses of float[CW] each
         const uint32_t c_zc = c_delta + CW * 4;    // (z_n - 8) as a float: exact, |.| <= 8
         const uint32_t c_bias = c_zc + CW * 4;
-        const uint32_t stg0 = sbase + S::kStageOutOff + ew * ((BLK ? 2 : 1) * 32 * RB);
+        const uint32_t stg0 = sbase + S::kStageOutOff + ew * (32 * RB);
         constexpr int kShift = 4;  // the widened weights are 16 x (u - 8)
         if (!RAW && lane == 0) tma_prefetch_desc(&tmY);
-        if constexpr (BLK) {
-            // Block-wise scales: every block of 1024 codes has its own int32 accumulator (the two
-            // accumulators alternate) and its own scale per token.  This warp keeps the running
-            // fp32 sum over blocks of its 32 rows and CW columns in tensor-memory columns [256, 384)
-            // -- lanes and columns only it touches -- and dequantizes after the last block.  acc_g here is the sum over the
-            // stored codes (u - 8); the rest of the zero point is one term per row:
-            //     y = Delta_n * (sum_g s_ig acc_g - (z_n - 8) T_i) + bias_n,  T_i = sum_g s_ig S_ig.
-            constexpr uint32_t kFloatCol = 2 * BN;
-            uint32_t lt = 0, nstore = 0;
-            for (int tile = pair; tile < num_tiles; tile += num_pairs) {
-                const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM, n0 = (tile % num_n) * BN + half * CW;
-                __syncwarp();
-#pragma unroll
-                for (int i = 0; i < CW / 32; ++i) {
-                    const int c = lane + 32 * i, n = n0 + c;
-                    const bool okn = n < N;
-                    sts32f(c_delta + 4 * c, okn ? __ldg(delta + n) : 0.f);
-                    sts32f(c_zc + 4 * c, okn ? (float)__ldg(zc + n) : 0.f);
-                    sts32f(c_bias + 4 * c, (okn && bias != nullptr) ? __bfloat162float(bias[n]) : 0.f);
-                }
-                __syncwarp();
-                const int row = m0 + q * 32 + lane;
-                const bool row_ok = row < M;
-                const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-                // the zero-point term of all blocks at once: T_i = sum_g s_ig S_ig (each S_ig is exact in fp32)
-                float T = 0.f;
-                if (row_ok)
-                    for (int g = 0; g < NG; ++g) T = fmaf(scales[(int64_t)row * NG + g], (float)sums[(int64_t)row * NG + g], T);
-                bool ok = true;
-                for (int g = 0; g < NG; ++g, ++lt) {
-                    const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
-                    const float s_k = (row_ok ? scales[(int64_t)row * NG + g] : 0.f) * (1.0f / (float)(1 << kShift));
-                    if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) { ok = false; break; }
-                    tc_fence_after();
-                    const bool last = g == NG - 1;
-#pragma unroll 1
-                    for (int hc = 0; hc < CW / 32; ++hc) {
-                        uint32_t r[32], f[32];
-                        tmem_ld_32x32(tmem_base + a * BN + half * CW + hc * 32 + lane_addr, r);
-                        if (g > 0) tmem_ld_32x32(tmem_base + kFloatCol + half * CW + hc * 32 + lane_addr, f);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int t = 0; t < 32; ++t)  // running sum of s_ig * acc_g (the raw accumulator is 2^kShift x the true one)
-                            f[t] = __float_as_uint(fmaf((float)(int32_t)r[t], s_k, g > 0 ? __uint_as_float(f[t]) : 0.f));
-                        if (!last) {
-                            tmem_st_32x32(tmem_base + kFloatCol + half * CW + hc * 32 + lane_addr, f);
-                            continue;
-                        }
-                        // last block: dequantize, round, stage 64 columns per TMA store
-                        if ((hc & 1) == 0) {
-                            if (lane == 0) tma_store_wait_read<1>();
-                            __syncwarp();
-                        }
-                        const uint32_t buf = stg0 + (nstore & 1u) * (32 * 128);
-#pragma unroll
-                        for (int j = 0; j < 32; j += 8) {
-                            const float4 d0 = lds128f(c_delta + 4 * (hc * 32 + j)), d1 = lds128f(c_delta + 4 * (hc * 32 + j + 4));
-                            const float4 z0 = lds128f(c_zc + 4 * (hc * 32 + j)), z1 = lds128f(c_zc + 4 * (hc * 32 + j + 4));
-                            const float4 b0 = lds128f(c_bias + 4 * (hc * 32 + j)), b1 = lds128f(c_bias + 4 * (hc * 32 + j + 4));
-                            const float dl[8] = {d0.x, d0.y, d0.z, d0.w, d1.x, d1.y, d1.z, d1.w};
-                            const float zz[8] = {z0.x, z0.y, z0.z, z0.w, z1.x, z1.y, z1.z, z1.w};
-                            const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-                            uint32_t pk[4];
-#pragma unroll
-                            for (int t = 0; t < 8; t += 2) {
-                                float y0 = fmaf(fmaf(-zz[t], T, __uint_as_float(f[j + t])), dl[t], bb[t]);
-                                float y1 = fmaf(fmaf(-zz[t + 1], T, __uint_as_float(f[j + t + 1])), dl[t + 1], bb[t + 1]);
-                                if (act == 1) {
-                                    y0 = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(y0)));
-                                    y1 = gelu_tanh_f32(__bfloat162float(__float2bfloat16_rn(y1)));
-                                }
-                                __nv_bfloat162 b2 = __floats2bfloat162_rn(y0, y1);
-                                pk[t >> 1] = *reinterpret_cast<uint32_t*>(&b2);
-                            }
-                            const int ch = (4 * (hc & 1) + (j >> 3)) ^ (lane & 7);
-                            sts128(buf + lane * 128 + ch * 16, pk[0], pk[1], pk[2], pk[3]);
-                        }
-                        if (hc & 1) {
-                            fence_proxy_async_smem();
-                            __syncwarp();
-                            const int nb = n0 + (hc >> 1) * 64;
-                            if (lane == 0 && nb < N && m0 + q * 32 < M) {
-                                tma_store_2d(&tmY, buf, nb, m0 + q * 32);
-                                tma_store_commit();
-                            }
-                            ++nstore;
-                        }
-                    }
-                    // the accumulator is read: the MMA warp may have it back before this warp's
-                    // running sums have landed (nobody else touches those columns)
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty(a), 0));
-                    if (!last) tmem_st_wait();
-                }
-                if (!ok) break;
-            }
-            if (lane == 0) tma_store_wait_all();
-            __syncwarp();
-        } else {
         uint32_t lt = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++lt) {
             const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
@@ -489,7 +352,6 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         if (!RAW && lane == 0) tma_store_wait_all();
         __syncwarp();
-        }
 
     } else if (warp < kSsFwdWarp) {
         // ------------------------------------------------------------ widen weight codes -> shared memory
@@ -575,11 +437,11 @@ inline bool make_out_map32(CUtensorMap* tm, const void* base, uint64_t cols, uin
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool RAW, int EW, bool BLK>
+template <bool RAW, int EW>
 static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
                                    int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
-    using S = SsSmem<BLK>;
+    using S = SsSmem;
     const int64_t K = w.K, N = w.N;
     const BlobLayout L = blob_layout(N, K);
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
@@ -591,12 +453,12 @@ static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, con
         return DVDQ_ERR_CUDA;
     if (RAW) {
         tmY = tmA;  // unused
-    } else if (!((EW == 8 && !BLK) ? make_out_map32(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)
+    } else if (!(EW == 8 ? make_out_map32(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)
                                    : make_out_map(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy))) {
         return DVDQ_ERR_CUDA;
     }
     constexpr int kThreads = (EW == 8 ? kSsFirstEpilogueWarp2 + 4 : kSsFirstEpilogueWarp2) * 32;
-    auto kern = qgemm_ss_kernel<RAW, EW, BLK>;
+    auto kern = qgemm_ss_kernel<RAW, EW>;
     static PerDevice<int> cache;
     const int max_pairs = resident_pairs(cache, kern, kThreads, S::kTotal);
     if (max_pairs == 0) return DVDQ_ERR_CUDA;
@@ -617,8 +479,8 @@ static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const
                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
                                    int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
     const bool wide_epilogue = w.K <= 2048 || (act != 0 && w.K <= 6144);
-    return wide_epilogue ? launch_qgemm_ss_t<RAW, 8, false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
-                         : launch_qgemm_ss_t<RAW, 4, false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
+    return wide_epilogue ? launch_qgemm_ss_t<RAW, 8>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
+                         : launch_qgemm_ss_t<RAW, 4>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
 }
 
 }  // namespace dvdq

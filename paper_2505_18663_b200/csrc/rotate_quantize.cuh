@@ -76,7 +76,7 @@ __global__ void __maxnreg__(80)  // two CTAs of 12 warps per SM
 rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
           uint8_t* __restrict__ codes, float* __restrict__ scales, int32_t* __restrict__ sums,
           int spans, int tokens_per_cta, int num_groups, int scale_group, int code_bits) {
-    extern __shared__ float4 s_turn[];  // 256 float4 per warp
+    extern __shared__ __align__(128) float4 s_turn[];  // 256 float4 per warp
     __shared__ unsigned s_max[3][kRqMaxWarps];  // [slot set][token of the CTA]: bits of the token absmax
     __shared__ int s_sum[3][kRqMaxWarps];       // sum of the token's codes
     constexpr bool kRot = LOG2B > 0;
@@ -134,12 +134,18 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
         wr[1] = (b34 + 4) * 8 + (low ^ 4);
     }
     const int rd = lane * 8 + (lane & 7);
+    // the same as 32-bit shared addresses: the buffer is 128-byte aligned, so the XOR of the read
+    // index is an XOR of the address, and every access is base + immediate or base ^ immediate
+    const uint32_t turn_a = smem_u32(turn);
+    const uint32_t wr_a[2] = {turn_a + 16u * wr[0], turn_a + 16u * wr[1]};
+    const uint32_t rd_a = turn_a + 16u * rd;
     const int row_bytes = (int)act_row_bytes(K, BITS);
     // byte offsets of the lane's first output word (+ 32 j, or + 64 j for 8-bit codes) and of its
     // first high-plane word (+ 16 j): everything else in the loop is one 32 x 32 -> 64 bit multiply-add
     const int st_b0 = BITS == 8 ? st_e0 : st_e0 >> 1;
     const int st_h0 = (K >> 1) + ((st_e0 >> 4) << 2);
-    const float rs = (LOG2B & 1) ? rsqrtf((float)(1 << LOG2B)) : 1.0f / (float)(1 << (LOG2B / 2));
+    // s = (absmax / sqrt(B)) / qmax as one multiplication by a constant (at most an ulp from the quotient)
+    const float rs = ((LOG2B & 1) ? rsqrtf((float)(1 << LOG2B)) : 1.0f / (float)(1 << (LOG2B / 2))) / qmax;
 
     auto load_span = [&](uint4 (&raw)[4], int group) {
         int token = group * tokens_per_cta + tl;
@@ -232,7 +238,8 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
                 }
 #pragma unroll
             for (int r0 = 0; r0 < 2; ++r0)
-                turn[wr[r0] + 64 * c] = make_float4(v[0][0][r0], v[0][1][r0], v[1][0][r0], v[1][1][r0]);
+                sts128(wr_a[r0] + 1024u * c, __float_as_uint(v[0][0][r0]), __float_as_uint(v[0][1][r0]), __float_as_uint(v[1][0][r0]),
+                       __float_as_uint(v[1][1][r0]));
         }
         __syncwarp();
         // The lane now stands for bits 5:3 (lane & 7) and bits 9:8 (lane >> 3);
@@ -242,7 +249,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
         for (int j = 0; j < 4; ++j)
 #pragma unroll
             for (int i0 = 0; i0 < 2; ++i0) {
-                const float4 f = turn[rd ^ (j | (i0 << 2))];
+                const float4 f = lds128f(rd_a ^ (16u * (j | (i0 << 2))));
                 W[j][i0][0] = f2_pack(f.x, f.y);
                 W[j][i0][1] = f2_pack(f.z, f.w);
             }
@@ -399,11 +406,11 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
             if ((lane & 7) == 0) {
                 const int g0 = sp * per_span + (lane >> 3) * (per_span >> 2);
                 if (FULL || g0 < gps) {
-                    scales[(int64_t)token * gps + g0] = (am[0] * rs) / qmax;
+                    scales[(int64_t)token * gps + g0] = am[0] * rs;
                     sums[(int64_t)token * gps + g0] = s0;
                 }
                 if (scale_group != 256 && (FULL || g0 + 1 < gps)) {
-                    scales[(int64_t)token * gps + g0 + 1] = (am[1] * rs) / qmax;
+                    scales[(int64_t)token * gps + g0 + 1] = am[1] * rs;
                     sums[(int64_t)token * gps + g0 + 1] = s1;
                 }
             }
@@ -412,7 +419,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
         lsum = __reduce_add_sync(0xFFFFFFFFu, lsum);
         if (!team) {  // the span's own scale: a token of one span, or one scale per 1024 channels
             if (lane == 0) {
-                scales[(int64_t)token * spans + sp] = (amax * rs) / qmax;
+                scales[(int64_t)token * spans + sp] = amax * rs;
                 sums[(int64_t)token * spans + sp] = lsum;
             }
             continue;
@@ -421,7 +428,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
             atomicAdd(&s_sum[cur][tl], lsum);
             // the previous iteration's token: its warps added their code sums before this iteration's barrier
             if (sp == 0 && prev_token >= 0) {
-                scales[prev_token] = (prev_amax * rs) / qmax;  // s_i = (absmax / sqrt(B)) / qmax
+                scales[prev_token] = prev_amax * rs;  // s_i = (absmax / sqrt(B)) / qmax
                 sums[prev_token] = s_sum[prv][tl];
             }
         }
@@ -435,7 +442,7 @@ rq_kernel(const __nv_bfloat16* __restrict__ X, int M, int K, int ldx,
     if (!team) return;
     asm volatile("bar.sync %0, %1;" ::"r"(1 + tl), "r"(spans * 32) : "memory");
     if (sp == 0 && lane == 0 && prev_token >= 0) {
-        scales[prev_token] = (prev_amax * rs) / qmax;
+        scales[prev_token] = prev_amax * rs;
         sums[prev_token] = s_sum[prv][tl];  // the last iteration's slots
     }
 }
