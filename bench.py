@@ -196,8 +196,9 @@ def config_of(wl, args):
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/, by code
 # layout (container_bits); None where no capture of that kernel in its present form exists.
-QGEMM_DRAM_TRAFFIC_PER_LAUNCH = {0: None, 8: None}
-RQ_DRAM_TRAFFIC_PER_LAUNCH = {0: None, 8: None}
+# (16384-token capture x 4: traffic grows with M; mean of the four launches of a step)
+QGEMM_DRAM_TRAFFIC_PER_LAUNCH = {0: 0.97e9, 8: 1.15e9}
+RQ_DRAM_TRAFFIC_PER_LAUNCH = {0: 0.83e9, 8: 0.94e9}
 
 
 class Leg:
