@@ -351,7 +351,7 @@ def roofline_blocks(leg, ms_per_step, rq_ms, gm_ms, args, peaks, ceiling, timed_
     return roof, rq_roof, stages
 
 
-def run_workload(args, wl, B, W, D, dist, dev, rank, local_rank, world, peaks, full):
+def run_workload(args, wl, B, W, D, dist, dev, rank, local_rank, world, peaks, full, ceiling=None):
     """Times one workload; `full` adds the legs of the headline line (other layout, alone, ceiling, e2e, oracle)."""
     def barrier():
         if dist is not None:
@@ -379,7 +379,6 @@ def run_workload(args, wl, B, W, D, dist, dev, rank, local_rank, world, peaks, f
     value = D.aggregate_rate(ops_per_step, ms_per_step, world) / 1e12
     timed_s = ms_per_step * args.steps * 1e-3
 
-    ceiling = None
     if full and not args.no_ceiling:
         ceiling = measure_int8_ceiling(B, min(2.0, max(0.1, timed_s)), local_rank)
         check_status()
@@ -387,30 +386,34 @@ def run_workload(args, wl, B, W, D, dist, dev, rank, local_rank, world, peaks, f
 
     out = {"value": value, "ms_per_step": ms_per_step, "roofline": roof, "roofline_rotate_quantize": rq_roof, "stages": stages,
            "clocks": clocks, "gpu_launches": leg.launches_per_step() * args.steps, "ceiling": ceiling, "leg": leg}
-    if not full:
-        return out
-
-    # ---- rotate-quantize on its own (no GEMM between the launches drawing the power budget down)
-    if not args.no_alone:
-        n_alone = max(5, args.steps // 2)
-        _, rq_alone_ms, _ = leg.timed(n_alone, 3, barrier, rq_only=True)
-        alg = sum(rq_algorithmic_bytes(M, L["layer"], args.scale_group) for L in leg.layers)
-        g = alg / (sum(rq_alone_ms) * 1e-3) / 1e9
-        rq_roof["alone"] = {"achieved": g, "frac": g / peaks["hbm_gbs"], "frac_of_nominal_8000": g / NOMINAL_HBM_GBS, "steps": n_alone,
-                            "note": "the same launches without the GEMMs between them"}
-
-    # ---- the same step with the other code layout, as a full block of its own
-    if not args.no_other_layout and world == 1 and not leg.fuse:
+    def other_layout_leg():
         other = 8 if args.container == 0 else 0
         leg2 = Leg(B, W, wl, args, other, dev, rank, shared=leg.shared)
         n2 = max(5, min(args.steps, 50))
         ms2, rq2, gm2 = leg2.timed(n2, 3, barrier)
         check_status()
         r2, rr2, st2 = roofline_blocks(leg2, ms2, rq2, gm2, args, peaks, ceiling, ms2 * n2 * 1e-3)
-        out["other_layout"] = {"act_codes": "one int8 per code" if other == 8 else "packed, b bits per code",
-                               "value": ops_per_step / (ms2 * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": ms2, "steps": n2,
-                               "roofline": r2, "roofline_rotate_quantize": rr2, "stages": st2}
-        del leg2
+        return {"act_codes": "one int8 per code" if other == 8 else "packed, b bits per code",
+                "value": ops_per_step / (ms2 * 1e-3) / 1e12, "unit": "TOPS", "ms_per_step": ms2, "steps": n2,
+                "roofline": r2, "roofline_rotate_quantize": rr2, "stages": st2}
+
+    if not full:
+        if not args.no_other_layout and world == 1 and not leg.fuse:
+            out["other_layout"] = other_layout_leg()
+        return out
+
+    # ---- rotate-quantize on its own (no GEMM between the launches drawing the power budget down)
+    if not args.no_alone:
+        n_alone = max(5, args.steps // 2)
+        _, rq_alone_ms, _ = leg.timed(n_alone, 3, barrier, rq_only=True)
+        alg = sum(rq_algorithmic_bytes(M, L["layer"], args.scale_group) for li, L in enumerate(leg.layers) if not (leg.fuse and li > 0))
+        g = alg / (sum(t for li, t in enumerate(rq_alone_ms) if not (leg.fuse and li > 0)) * 1e-3) / 1e9
+        rq_roof["alone"] = {"achieved": g, "frac": g / peaks["hbm_gbs"], "frac_of_nominal_8000": g / NOMINAL_HBM_GBS, "steps": n_alone,
+                            "note": "the same launches without the GEMMs between them"}
+
+    # ---- the same step with the other code layout, as a full block of its own
+    if not args.no_other_layout and world == 1 and not leg.fuse:
+        out["other_layout"] = other_layout_leg()
     return out
 
 
@@ -457,7 +460,7 @@ def run_cuda(args, wl):
             if bits:
                 w2 = dataclasses.replace(w2, layers=tuple(dataclasses.replace(l, bits=bits) for l in w2.layers))
             torch.cuda.empty_cache()
-            r = run_workload(args, w2, B, W, D, dist, dev, rank, local_rank, world, peaks, full=False)
+            r = run_workload(args, w2, B, W, D, dist, dev, rank, local_rank, world, peaks, full=False, ceiling=res["ceiling"])
             r.pop("leg")
             r.pop("ceiling")
             r["config"] = config_of(w2, args)["workload"]
