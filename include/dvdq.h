@@ -46,7 +46,7 @@ typedef enum {
     DVDQ_ERR_ARCH = 8,           /* current device is not sm_100 */
     DVDQ_ERR_CUDA = 9,           /* a CUDA runtime or driver call failed */
     DVDQ_ERR_DEVICE_TIMEOUT = 10,/* a kernel gave up on a bounded device-side wait */
-    DVDQ_ERR_UNSUPPORTED = 11    /* an option that is not built (scale_group other than 0 or 1024, unknown activation function) */
+    DVDQ_ERR_UNSUPPORTED = 11    /* an option that is not built (scale_group other than 0, 128, 256, 1024; unknown activation function) */
 } dvdq_status;
 
 /* Human-readable name of a status code (static storage, never NULL). */
@@ -58,13 +58,13 @@ const char* dvdq_status_string(dvdq_status s);
  *               [-128,127]; the b_high = 8 of Sec. 3.3's bit-width switching, i.e. the W4A8 steps).
  *               The quantizer is symmetric with qmax = 2^(b-1) - 1.
  *   rot_block   B, the order of the Hadamard blocks of the rotation
- *               R = I_{K/B} (x) H_B / sqrt(B); a power of two in [64, 1024] that
+ *               R = I_{K/B} (x) H_B / sqrt(B); a power of two in [64, 4096] that
  *               divides K.  0 means no rotation (R = I).
  *   scale_group granularity of Lambda: 0 = one absmax scale per token over all K channels;
- *               1024 = the block-wise variant of Sec. 3.2's last paragraph, one scale per token
- *               and per block of 1024 consecutive rotated channels (K % 1024 == 0; every block
- *               is quantized on its own, the GEMM rescales per block).  Other values give
- *               DVDQ_ERR_UNSUPPORTED.
+ *               G = 128, 256 or 1024 = the block-wise variant of Sec. 3.2's last paragraph, one
+ *               scale per token and per group of G consecutive rotated channels (whole k-blocks
+ *               of the GEMM; K % G == 0 and K % 256 == 0; every group is quantized on its own,
+ *               the GEMM rescales per group).  Other values give DVDQ_ERR_UNSUPPORTED.
  *   container_bits  how the codes are kept between the transform and the GEMM (the values are
  *               the same either way): 0 = packed, b bits per code; 8 = one int8 per code.
  *               int8 tensor cores are the narrowest integer ones on sm_100, so packed codes
@@ -101,7 +101,7 @@ typedef struct {
 size_t dvdq_act_codes_bytes(int64_t M, int64_t K, int32_t bits);
 /* The same for a quantizer description: M * K * (container_bits ? container_bits : bits) / 8. */
 size_t dvdq_act_codes_bytes_q(int64_t M, int64_t K, const dvdq_act_quant* q);
-/* Number of scales (and of code sums) of an [M, K] tensor: M, or M * K / 1024 block-wise. 0 on bad input. */
+/* Number of scales (and of code sums) of an [M, K] tensor: M, or M * K / scale_group block-wise. 0 on bad input. */
 size_t dvdq_act_scales_count(int64_t M, int64_t K, const dvdq_act_quant* q);
 /* Bytes of the device blob that dvdq_pack_weights() writes for an [N, K] matrix. 0 on bad input. */
 size_t dvdq_weight_blob_bytes(int64_t N, int64_t K);
@@ -116,9 +116,9 @@ size_t dvdq_qlinear_workspace_bytes(int64_t M, int64_t K, const dvdq_act_quant* 
  *   X_bf16         [M, K] bf16, row pitch ldx elements; 16-byte aligned, ldx % 8 == 0
  *   codes_out      dvdq_act_codes_bytes_q(M, K, q) bytes, 16-byte aligned (opaque layout)
  *   scales_out     [M] fp32, s_i  (0 for an all-zero token, whose codes are all 0);
- *                  block-wise: [M, K/1024], one scale per token and block
+ *                  block-wise: [M, K/scale_group], one scale per token and group
  *   code_sums_out  [M] int32, sum_k c_ik (used by the GEMM for the weight zero point);
- *                  block-wise: [M, K/1024], the sum over each block
+ *                  block-wise: [M, K/scale_group], the sum over each group
  * K % 64 == 0, K <= 16384.  M == 0 is a no-op.
  */
 dvdq_status dvdq_rotate_quantize(const void* X_bf16, int64_t M, int64_t K, int64_t ldx,

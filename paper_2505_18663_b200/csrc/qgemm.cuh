@@ -308,14 +308,20 @@ qgemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                 const int row = m0 + q * 32 + lane;
                 const bool row_ok = row < M;
                 const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-                // the zero-point term of all blocks at once: T_i = sum_g s_ig S_ig (each S_ig is exact in fp32)
+                // the zero-point term T_i = sum_g s_ig S_ig (each S_ig is exact in fp32) is added up group by
+                // group, from loads issued a group ahead
                 float T = 0.f;
-                if (row_ok)
-                    for (int g = 0; g < NG; ++g) T = fmaf(scales[(int64_t)row * NG + g], (float)sums[(int64_t)row * NG + g], T);
+                float s_next = row_ok ? __ldg(scales + (int64_t)row * NG) : 0.f;
+                float S_next = row_ok ? (float)__ldg(sums + (int64_t)row * NG) : 0.f;
                 bool ok = true;
                 for (int g = 0; g < NG; ++g, ++lt) {
                     const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
-                    const float s_k = (row_ok ? scales[(int64_t)row * NG + g] : 0.f) * (1.0f / (float)(1 << kShift));
+                    const float s_k = s_next * (1.0f / (float)(1 << kShift));
+                    T = fmaf(s_next, S_next, T);
+                    if (g + 1 < NG && row_ok) {
+                        s_next = __ldg(scales + (int64_t)row * NG + g + 1);
+                        S_next = (float)__ldg(sums + (int64_t)row * NG + g + 1);
+                    }
                     if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) { ok = false; break; }
                     tc_fence_after();
                     const bool last = g == NG - 1;

@@ -320,19 +320,23 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const bool row_ok = row < M;
             const float* srow = scales + (int64_t)(row_ok ? row : 0) * NG;
             const int32_t* Srow = sums + (int64_t)(row_ok ? row : 0) * NG;
-            // the zero-point term of all groups at once: T_i = sum_g s_ig S_ig (each S_ig is exact in fp32)
+            // the zero-point term T_i = sum_g s_ig S_ig (each S_ig is exact in fp32) is added up group by
+            // group, from loads issued a group ahead
             float T = 0.f;
-            for (int g = 0; g < NG; ++g) T = fmaf(__ldg(srow + g), (float)__ldg(Srow + g), T);
-            if (!row_ok) T = 0.f;
             uint64_t run[CW / 2];  // fp32 pairs: columns 2i and 2i + 1
 #pragma unroll
             for (int t = 0; t < CW / 2; ++t) run[t] = f2_pack(0.f, 0.f);
             float s_next = row_ok ? __ldg(srow) : 0.f;
+            float S_next = row_ok ? (float)__ldg(Srow) : 0.f;
             for (int g = 0; g < NG; ++g, ++lt) {
                 const uint32_t a = lt & 1u, aph = (lt >> 1) & 1u;
                 const float s_k = s_next * (1.0f / (float)(1 << kShift));
                 const uint64_t s2 = f2_pack(s_k, s_k);
-                if (g + 1 < NG) s_next = row_ok ? __ldg(srow + g + 1) : 0.f;  // its latency hides behind this group
+                T = fmaf(s_next, S_next, T);
+                if (g + 1 < NG) {  // the next group's scale and code sum: their latency hides behind this group
+                    s_next = row_ok ? __ldg(srow + g + 1) : 0.f;
+                    S_next = row_ok ? (float)__ldg(Srow + g + 1) : 0.f;
+                }
                 if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) { ok = false; break; }
                 tc_fence_after();
                 // 16 columns at a time, the next load in flight while these are added up

@@ -74,3 +74,42 @@ def test_int8_ceiling_runs_and_reports_its_work():
     assert 2000.0 < tops < 4700.0, tops
     with pytest.raises(B.DvdqError):
         B.dvdq_int8_mma_ceiling(0)
+
+
+def test_two_host_threads_share_the_library():
+    """The launch-time set-up is cached per device under a lock: two host threads that call the
+    library at the same time (own streams, own buffers) get the bits a single thread gets."""
+    import threading
+    wl = W.WORKLOADS["tiny"]
+    layer = wl.layers[0]
+    x = W.make_activations(wl, layer.K, device=DEV)
+    u, d, z = W.make_weight_codes(layer, seed=0, device=DEV)
+    blob = torch.empty(B.dvdq_weight_blob_bytes(layer.N, layer.K), dtype=torch.uint8, device=DEV)
+    w = B.dvdq_pack_weights(u, d, z, layer.rot_block, blob)
+    torch.cuda.synchronize()
+    results, errors = {}, []
+
+    def worker(idx, container):
+        try:
+            torch.cuda.set_device(0)
+            stream = torch.cuda.Stream()
+            q = B.ActQuant(layer.bits, layer.rot_block, 0, container)
+            ws = torch.empty(B.dvdq_qlinear_workspace_bytes(wl.M, layer.K, q), dtype=torch.uint8, device=DEV)
+            Y = torch.empty(wl.M, layer.N, dtype=torch.bfloat16, device=DEV)
+            for _ in range(20):
+                B.dvdq_qlinear(x, q, w, None, 0, Y, ws, stream=stream)
+            stream.synchronize()
+            results[idx] = Y
+        except Exception as e:   # surfaced by the assertion below
+            errors.append(e)
+
+    threads = [threading.Thread(target=worker, args=(i, 8 if i % 2 else 0)) for i in range(4)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    assert B.dvdq_last_device_status() == (B.OK, 0)
+    # both layouts give the same output; every thread got it
+    for i in range(1, 4):
+        assert torch.equal(results[0], results[i])
