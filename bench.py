@@ -456,9 +456,13 @@ def run_cuda(args, wl):
         todo = [(n, w, 0) for n, w in W.WORKLOADS.items() if n not in (wl.name, "tiny")]
         # the HunyuanVideo shapes at both bit widths (the headline runs the seeded 25 % mask)
         todo += [("hunyuan_all_A4", W.WORKLOADS["hunyuan"], 4), ("hunyuan_all_A6", W.WORKLOADS["hunyuan"], 6)]
+        # the K = 12288 layer with rotation blocks of 4096 channels (blocks that span four warps of the transform)
+        todo += [("hunyuan_B4096_for_K12288", W.WORKLOADS["hunyuan"], -4096)]
         for name, w2, bits in todo:
-            if bits:
+            if bits > 0:
                 w2 = dataclasses.replace(w2, layers=tuple(dataclasses.replace(l, bits=bits) for l in w2.layers))
+            elif bits < 0:
+                w2 = dataclasses.replace(w2, layers=tuple(dataclasses.replace(l, rot_block=-bits) if l.K % -bits == 0 else l for l in w2.layers))
             torch.cuda.empty_cache()
             r = run_workload(args, w2, B, W, D, dist, dev, rank, local_rank, world, peaks, full=False, ceiling=res["ceiling"])
             r.pop("leg")

@@ -37,6 +37,8 @@
 // all roles walk to the common exit, where the pair synchronises and tensor memory is released.
 #pragma once
 
+#include <stdlib.h>
+
 #include "dvdq_common.cuh"
 
 namespace dvdq {
@@ -747,6 +749,16 @@ static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const
                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
                                    int32_t* acc_out, int64_t ldacc, cudaStream_t st);
 
+template <bool RAW>
+static dvdq_status launch_qgemm_ps(int bits, const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+                                   const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
+                                   int32_t* acc_out, int64_t ldacc, cudaStream_t st);
+inline bool use_ps_kernel() {
+    static int v = -1;
+    if (v < 0) { const char* e = getenv("DVDQ_PS"); v = (e && e[0] == '0') ? 0 : 1; }
+    return v == 1;
+}
+
 // qgemm_fat.cuh: the same with block-wise activation scales
 static dvdq_status launch_qgemm_blk(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                     const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, cudaStream_t st);
@@ -765,6 +777,9 @@ inline dvdq_status launch_qgemm(const void* codes, const float* scales, const in
     if (sb == 8 && (raw || q.scale_group == 0))
         return raw ? launch_qgemm_ss<true>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
                    : launch_qgemm_ss<false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
+    if ((sb == 4 || sb == 6) && (raw || q.scale_group == 0) && use_ps_kernel())
+        return raw ? launch_qgemm_ps<true>(sb, codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
+                   : launch_qgemm_ps<false>(sb, codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
 #define DVDQ_GEMM_CASE(B)                                                                                          \
     if (sb == B) {                                                                                                 \
         if (raw) return launch_qgemm_t<B, true, false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st); \

@@ -67,7 +67,7 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmY, const float* __restrict__ scales,
                  const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
                  const __nv_bfloat16* __restrict__ bias, int M, int N, int K, int act, int spr, const FusedOut fo) {
-    using S = SsSmem;
+    using S = SsSmem<8>;
     constexpr int BN = S::BN, BNh = S::BNh;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -577,7 +577,7 @@ static bool fat_kernel_registers_fit(Kern kern) {
 
 static dvdq_status launch_qgemm_blk(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                     const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, cudaStream_t st) {
-    using S = SsSmem;
+    using S = SsSmem<8>;
     const int64_t K = w.K, N = w.N;
     const BlobLayout L = blob_layout(N, K);
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
@@ -604,7 +604,7 @@ static dvdq_status launch_qgemm_blk(const void* codes, const float* scales, cons
 // codes, scales and code sums for rot_block = scale_group = 256 instead of bf16.
 static dvdq_status launch_qgemm_fused(const void* codes, const float* scales, const int32_t* sums, int64_t M,
                                       const dvdq_weights& w, const void* bias, int act, const FusedOut& fo, cudaStream_t st) {
-    using S = SsSmem;
+    using S = SsSmem<8>;
     const int64_t K = w.K, N = w.N;
     const BlobLayout L = blob_layout(N, K);
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);

@@ -40,22 +40,37 @@ constexpr int kSsFirstEpilogueWarp2 = kSsWProducerWarp + 1;  // a multiple of 4:
 static_assert(kSsFirstEpilogueWarp2 % 4 == 0, "lane quarters");
 static_assert(kSsStages % 2 == 0, "the MMA warp takes the weight stages in pairs");
 
+constexpr int kSsFirstAWarp = kSsFirstEpilogueWarp2;  // packed activation codes: eight more warps widen them (no second set of epilogue warps then)
+constexpr int kSsAWarps = 8;
+
+// ABITS: how the activation codes arrive.  8: one int8 each, TMA writes the operand stages themselves.
+// 4 / 6: packed; TMA fills a ring of packed tiles and warps widen them into the operand stages, as
+// for the weights (a 4-bit code masked into the high half of a byte is 16 x code, a 6-bit code
+// moved to the top of a byte 4 x code; the factor is shifted out of the accumulator).
+template <int ABITS>
 struct SsSmem {
     static constexpr int BN = kSsBN, BNh = BN / 2;
+    static constexpr bool kPackedA = ABITS != 8;
+    static constexpr int kAStages = kPackedA ? kSsStages : kSsAStages;  // operand stages of the activation tile
     static constexpr int kA = kBM * kBK;              // activation tile of one k-block (int8, swizzled)
     static constexpr int kW = BNh * kBK;              // widened weight half-tile
     static constexpr int kWPacked = BNh * kBK / 2;    // packed weight half-tile (64-byte rows)
+    static constexpr int kALo = kPackedA ? kBM * kBK / 2 : 0;            // packed codes / low plane (64-byte rows)
+    static constexpr int kAHi = ABITS == 6 ? kBM * kBK / 4 : 0;          // high plane of 6-bit codes (32-byte rows)
+    static constexpr int kAPacked = kALo + kAHi;
+    static constexpr int kAPackedStages = !kPackedA ? 0 : (ABITS == 6 ? 3 : 4);  // what fits
     static constexpr int kAOff = 0;
-    static constexpr int kWOff = kAOff + kSsAStages * kA;
+    static constexpr int kWOff = kAOff + kAStages * kA;
     static constexpr int kWPackedOff = kWOff + kSsStages * kW;
-    static constexpr int kStageOutOff = kWPackedOff + kSsWPackedStages * kWPacked;  // 1024-byte aligned
+    static constexpr int kAPackedOff = kWPackedOff + kSsWPackedStages * kWPacked;
+    static constexpr int kStageOutOff = kAPackedOff + kAPackedStages * kAPacked;  // 1024-byte aligned
     // 16 KB of staging and 12 KB of constants whether four or eight epilogue warps share them: one
     // buffer of 32 rows x 64 (or 32) bf16 each, and delta / zero-point rest / bias of 256 (or 128) columns
     static constexpr int kStageOutBytes = 4 * 32 * 128;
     static constexpr int kConstOff = kStageOutOff + kStageOutBytes;
     static constexpr int kConstBytes = 4 * 3 * BN * 4;
     static constexpr int kBarOff = kConstOff + kConstBytes;
-    static constexpr int kNumBars = 3 * kSsAStages + 2 * kSsStages + 5 + 2 * kSsWPackedStages;
+    static constexpr int kNumBars = 3 * kAStages + 2 * kSsStages + 5 + 2 * kSsWPackedStages + 2 * kAPackedStages;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kTotal = kMiscOff + 16 + 1024;
     static_assert(kStageOutOff % 1024 == 0, "swizzled tiles need 1024-byte alignment");
@@ -73,15 +88,21 @@ __device__ __forceinline__ void tc_mma_i8_ss_pair(uint32_t d_tmem, uint64_t a_de
         : "memory");
 }
 
-template <bool RAW, int EW>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((EW == 8 ? kSsFirstEpilogueWarp2 + 4 : kSsFirstEpilogueWarp2) * 32, 1)
-qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+template <int ABITS>
+constexpr int ss_warps(int ew) { return ABITS != 8 ? kSsFirstAWarp + kSsAWarps : (ew == 8 ? kSsFirstEpilogueWarp2 + 4 : kSsFirstEpilogueWarp2); }
+
+template <int ABITS, bool RAW, int EW>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(ss_warps<ABITS>(EW) * 32, 1)
+qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmAhi, const __grid_constant__ CUtensorMap tmW,
                 const __grid_constant__ CUtensorMap tmY, const float* __restrict__ scales,
                 const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
                 const __nv_bfloat16* __restrict__ bias, int32_t* __restrict__ acc_out, int64_t ldacc,
                 int M, int N, int K, int act, int spr) {
-    using S = SsSmem;
+    using S = SsSmem<ABITS>;
     constexpr int BN = S::BN, BNh = S::BNh;
+    constexpr bool kPackedA = S::kPackedA;
+    constexpr int AST = S::kAStages, APS = S::kAPackedStages;
+    static_assert(!kPackedA || EW == 4, "packed activation codes: the second set of epilogue warps gives way to the widening warps");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -95,9 +116,9 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
     const uint32_t bar0 = sbase + S::kBarOff;
     auto a_full = [&](int s) { return bar0 + 8u * s; };                          // this CTA's TMA copy of the stage
-    auto a_ready = [&](int s) { return bar0 + 8u * (kSsAStages + s); };          // leader's copy: both CTAs' copies landed
-    auto a_empty = [&](int s) { return bar0 + 8u * (2 * kSsAStages + s); };      // one per CTA
-    const uint32_t barw = bar0 + 8u * (3 * kSsAStages);
+    auto a_ready = [&](int s) { return bar0 + 8u * (AST + s); };                 // leader's copy: both CTAs' rows of the stage are in place
+    auto a_empty = [&](int s) { return bar0 + 8u * (2 * AST + s); };             // one per CTA
+    const uint32_t barw = bar0 + 8u * (3 * AST);
     auto ops_full = [&](int s) { return barw + 8u * s; };                        // widened weights; leader's copy is used
     auto ops_empty = [&](int s) { return barw + 8u * (kSsStages + s); };         // one per CTA
     auto acc_full = [&](int s) { return barw + 8u * (2 * kSsStages + s); };      // one per CTA
@@ -105,11 +126,18 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t drain_bar = barw + 8u * (2 * kSsStages + 4);
     auto wp_full = [&](int s) { return drain_bar + 8u * (1 + s); };
     auto wp_empty = [&](int s) { return drain_bar + 8u * (1 + kSsWPackedStages + s); };
+    auto apk_full = [&](int s) { return drain_bar + 8u * (1 + 2 * kSsWPackedStages + s); };        // packed activation tiles (TMA)
+    auto apk_empty = [&](int s) { return drain_bar + 8u * (1 + 2 * kSsWPackedStages + APS + s); };
     volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + S::kMiscOff);  // [0] tmem base, [1] abort
     volatile uint32_t* abort_flag = misc + 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kSsAStages; ++s) { mbar_init(a_full(s), 1); mbar_init(a_ready(s), 2); mbar_init(a_empty(s), 1); }
+        for (int s = 0; s < AST; ++s) {
+            mbar_init(a_full(s), 1);
+            mbar_init(a_ready(s), kPackedA ? 2 * (kSsAWarps / kUnpackGroups) : 2);
+            mbar_init(a_empty(s), 1);
+        }
+        for (int s = 0; s < APS; ++s) { mbar_init(apk_full(s), 1); mbar_init(apk_empty(s), kSsAWarps / kUnpackGroups); }
         for (int s = 0; s < kSsStages; ++s) { mbar_init(ops_full(s), 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * EW); }
         mbar_init(drain_bar, 1);
@@ -131,25 +159,37 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         // ------------------------------------------------------------ TMA producer, activation rows
         if (lane == 0) {
             tma_prefetch_desc(&tmA);
+            if (ABITS == 6) tma_prefetch_desc(&tmAhi);
+            // one int8 per code: straight into the operand stages; packed codes: into the ring the widening warps read
+            constexpr int kRing = kPackedA ? APS : AST;
+            constexpr uint32_t kBytes = kPackedA ? S::kAPacked : S::kA;
+            auto ring_full = [&](int s) { return kPackedA ? apk_full(s) : a_full(s); };
+            auto ring_empty = [&](int s) { return kPackedA ? apk_empty(s) : a_empty(s); };
             uint32_t st = 0, ph = 0, issued = 0;
             bool ok = true;
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
                 for (int kb = 0; ok && kb < KB; ++kb) {
-                    if (!mbar_wait(a_empty(st), ph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-                    mbar_arrive_expect_tx(a_full(st), S::kA);
-                    tma_load_2d(sbase + S::kAOff + st * S::kA, &tmA, a_full(st), kb * kBK, m0);
+                    if (!mbar_wait(ring_empty(st), ph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                    mbar_arrive_expect_tx(ring_full(st), kBytes);
+                    if (kPackedA) {
+                        const uint32_t dst = sbase + S::kAPackedOff + st * S::kAPacked;
+                        tma_load_2d(dst, &tmA, ring_full(st), kb * (kBK / 2), m0);
+                        if (ABITS == 6) tma_load_2d(dst + S::kALo, &tmAhi, ring_full(st), kb * (kBK / 4), m0);
+                    } else {
+                        tma_load_2d(sbase + S::kAOff + st * S::kA, &tmA, ring_full(st), kb * kBK, m0);
+                    }
                     ++issued;
-                    if (++st == kSsAStages) { st = 0; ph ^= 1u; }
+                    if (++st == kRing) { st = 0; ph ^= 1u; }
                 }
             }
             if (!ok) {
                 // Giving up: let copies already in flight land before the CTA exits (bounded).
-                const uint32_t n_out = issued < (uint32_t)kSsAStages ? issued : (uint32_t)kSsAStages;
+                const uint32_t n_out = issued < (uint32_t)kRing ? issued : (uint32_t)kRing;
                 for (uint32_t i = 0; i < n_out; ++i) {
-                    const uint32_t s = (st + kSsAStages - 1 - i) % kSsAStages;
+                    const uint32_t s = (st + kRing - 1 - i) % kRing;
                     const uint32_t p = (s < st) ? ph : (ph ^ 1u);
-                    for (int it = 0; it < (1 << 16) && !mbar_try_wait(a_full(s), p); ++it) {}
+                    for (int it = 0; it < (1 << 16) && !mbar_try_wait(ring_full(s), p); ++it) {}
                 }
             }
         }
@@ -194,7 +234,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 // Two k-blocks per trip: every cycle between two issues is a bubble in the MMA stream
                 for (int kb = 0; kb < KB; kb += 2) {
                     // the activation ring may have an odd number of stages: its second stage of the trip can wrap
-                    const uint32_t sa1 = sa + 1 == kSsAStages ? 0u : sa + 1, pa1 = sa + 1 == kSsAStages ? pa ^ 1u : pa;
+                    const uint32_t sa1 = sa + 1 == AST ? 0u : sa + 1, pa1 = sa + 1 == AST ? pa ^ 1u : pa;
                     if (!mbar_wait_warp(a_ready(sa), pa, abort_flag, kWaitPackedFull)) { ok = false; break; }
                     if (!mbar_wait_warp(ops_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     if (!mbar_wait_warp(a_ready(sa1), pa1, abort_flag, kWaitPackedFull)) { ok = false; break; }
@@ -218,7 +258,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (st == kSsStages) { st = 0; ph ^= 1u; }
                     sa = sa1 + 1;
                     pa = pa1;
-                    if (sa == kSsAStages) { sa = 0; pa ^= 1u; }
+                    if (sa == AST) { sa = 0; pa ^= 1u; }
                 }
             }
             if (elect_one()) tc_commit_pair(drain_bar, 1);
@@ -226,7 +266,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             mbar_wait(drain_bar, 0u, abort_flag, kWaitDrain);
         }
         __syncwarp();
-    } else if (warp < kSsFirstWWarp || warp >= kSsFirstEpilogueWarp2) {
+    } else if (warp < kSsFirstWWarp || (!kPackedA && warp >= kSsFirstEpilogueWarp2)) {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;  // tensor-memory lane quarter this warp may read
         const int half = warp >= kSsFirstEpilogueWarp2 ? 1 : 0;  // EW = 8: which 128 of the tile's 256 columns
@@ -237,7 +277,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         const uint32_t c_zc = c_delta + CW * 4;    // (z_n - 8) as a float: exact, |.| <= 8
         const uint32_t c_bias = c_zc + CW * 4;
         const uint32_t stg0 = sbase + S::kStageOutOff + ew * (32 * RB);
-        constexpr int kShift = 4;  // the widened weights are 16 x (u - 8)
+        constexpr int kShift = ABITS == 4 ? 8 : ABITS == 6 ? 6 : 4;  // log2 of (A factor 16 / 4 / 1) x (W factor 16)
         if (!RAW && lane == 0) tma_prefetch_desc(&tmY);
         uint32_t lt = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++lt) {
@@ -402,14 +442,78 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
     } else if (warp == kSsFwdWarp) {
         // ------------------------------------------------------------ "activation rows landed" -> leader
-        uint32_t st = 0, ph = 0;
-        bool ok = true;
-        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-            for (int kb = 0; kb < KB; ++kb) {
-                if (!mbar_wait_warp(a_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(st), 0));
-                __syncwarp();
-                if (++st == kSsAStages) { st = 0; ph ^= 1u; }
+        // (codes in bytes only: a TMA copy completes on a barrier of its own CTA; widening warps arrive on the leader's themselves)
+        if constexpr (!kPackedA) {
+            uint32_t st = 0, ph = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                for (int kb = 0; kb < KB; ++kb) {
+                    if (!mbar_wait_warp(a_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                    if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(st), 0));
+                    __syncwarp();
+                    if (++st == AST) { st = 0; ph ^= 1u; }
+                }
+            }
+        }
+    } else if (kPackedA && warp >= kSsFirstAWarp) {
+        // ------------------------------------------------------------ widen activation codes -> shared memory
+        // The same job as the weight warps': this CTA's 128 token rows x 128 codes of a k-block, 16 bytes
+        // of packed low bits (and 8 bytes of high bits) per piece, into the K-major 128-byte-swizzled stage.
+        if constexpr (kPackedA) {
+            const uint32_t grp = (uint32_t)(warp - kSsFirstAWarp) >> 2;
+            const int u = (threadIdx.x - kSsFirstAWarp * 32) & 127;
+            uint32_t j = 0;
+            bool ok = true;
+            const uint32_t rt_zero = runtime_zero();
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                for (int kb = 0; kb < KB; ++kb) {
+                    const uint32_t jj = j++;
+                    if (jj % kUnpackGroups != grp) continue;
+                    const uint32_t pst = jj % APS, pph = (jj / APS) & 1u;
+                    const uint32_t wst = jj % AST, wph = (jj / AST) & 1u;
+                    if (!mbar_wait(apk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                    const uint32_t pa = sbase + S::kAPackedOff + pst * S::kAPacked;
+                    const uint32_t wd = sbase + S::kAOff + wst * S::kA;
+                    constexpr int kPieces = (kBM * 4) / 128;
+                    uint32_t e[kPieces][4], o[kPieces][4];
+                    uint32_t loaded = 0u;
+#pragma unroll
+                    for (int it = 0; it < kPieces; ++it) {
+                        const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                        const uint4 p = lds128(pa + row * (kBK / 2) + ck * 16);
+                        const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+                        loaded ^= p.w;
+                        if (ABITS == 4) {
+#pragma unroll
+                            for (int jw = 0; jw < 4; ++jw) { e[it][jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[it][jw] = w[jw] & 0xF0F0F0F0u; }
+                        } else {
+                            const uint2 hp = lds64(pa + S::kALo + row * (kBK / 4) + ck * 8);  // bits 5:4 of the piece's 32 codes
+                            const uint32_t hh[2] = {hp.x, hp.y};
+                            loaded ^= hp.y;
+#pragma unroll
+                            for (int jw = 0; jw < 4; ++jw) {
+                                const int a2 = 2 * (jw & 1);
+                                e[it][jw] = ((w[jw] << 2) & 0x3C3C3C3Cu) | ((hh[jw >> 1] << (6 - 2 * a2)) & 0xC0C0C0C0u);
+                                o[it][jw] = ((w[jw] >> 2) & 0x3C3C3C3Cu) | ((hh[jw >> 1] << (4 - 2 * a2)) & 0xC0C0C0C0u);
+                            }
+                        }
+                    }
+                    loaded &= rt_zero;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_after_loads(apk_empty(pst), loaded);  // the packed rows are in registers
+                    if (!mbar_wait(a_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int it = 0; it < kPieces; ++it) {
+                        const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                        const uint32_t drow = wd + (row >> 3) * 1024 + (row & 7) * 128;
+                        sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[it][0], o[it][0], e[it][1], o[it][1]);
+                        sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[it][2], o[it][2], e[it][3], o[it][3]);
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(wst), 0));
+                }
             }
         }
     }
@@ -437,34 +541,47 @@ inline bool make_out_map32(CUtensorMap* tm, const void* base, uint64_t cols, uin
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool RAW, int EW>
+template <int ABITS, bool RAW, int EW>
 static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
                                    int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
-    using S = SsSmem;
+    using S = SsSmem<ABITS>;
     const int64_t K = w.K, N = w.N;
     const BlobLayout L = blob_layout(N, K);
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
-    CUtensorMap tmA, tmW, tmY;
-    if (!make_byte_map(&tmA, codes, (uint64_t)K, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B))
-        return DVDQ_ERR_CUDA;
+    CUtensorMap tmA, tmAhi, tmW, tmY;
+    if (ABITS == 8) {
+        if (!make_byte_map(&tmA, codes, (uint64_t)K, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B)) return DVDQ_ERR_CUDA;
+        tmAhi = tmA;  // unused
+    } else {
+        // packed codes: 64-byte rows of low bits per k-block (and 32-byte rows of high bits), unswizzled, as the weights
+        const uint64_t pitch = (uint64_t)act_row_bytes(K, ABITS);
+        if (!make_byte_map(&tmA, codes, (uint64_t)K / 2, (uint64_t)M, pitch, kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_NONE)) return DVDQ_ERR_CUDA;
+        if (ABITS == 6) {
+            if (!make_byte_map(&tmAhi, static_cast<const uint8_t*>(codes) + K / 2, (uint64_t)K / 4, (uint64_t)M, pitch, kBK / 4, kBM,
+                               CU_TENSOR_MAP_SWIZZLE_NONE))
+                return DVDQ_ERR_CUDA;
+        } else {
+            tmAhi = tmA;  // unused
+        }
+    }
     if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, S::BNh,
                        CU_TENSOR_MAP_SWIZZLE_NONE))
         return DVDQ_ERR_CUDA;
     if (RAW) {
         tmY = tmA;  // unused
     } else if (!(EW == 8 ? make_out_map32(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)
-                                   : make_out_map(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy))) {
+                         : make_out_map(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy))) {
         return DVDQ_ERR_CUDA;
     }
-    constexpr int kThreads = (EW == 8 ? kSsFirstEpilogueWarp2 + 4 : kSsFirstEpilogueWarp2) * 32;
-    auto kern = qgemm_ss_kernel<RAW, EW>;
+    constexpr int kThreads = ss_warps<ABITS>(EW) * 32;
+    auto kern = qgemm_ss_kernel<ABITS, RAW, EW>;
     static PerDevice<int> cache;
     const int max_pairs = resident_pairs(cache, kern, kThreads, S::kTotal);
     if (max_pairs == 0) return DVDQ_ERR_CUDA;
     const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + S::BN - 1) / S::BN);
     const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
-    kern<<<2 * pairs, kThreads, S::kTotal, st>>>(tmA, tmW, tmY, scales, sums,
+    kern<<<2 * pairs, kThreads, S::kTotal, st>>>(tmA, tmAhi, tmW, tmY, scales, sums,
                                                    reinterpret_cast<const float*>(blob + L.delta_offset),
                                                    reinterpret_cast<const int32_t*>(blob + L.zc_offset),
                                                    static_cast<const __nv_bfloat16*>(bias), acc_out, ldacc, (int)M, (int)N, (int)K,
@@ -472,15 +589,25 @@ static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, con
     return cuda_status(cudaGetLastError());
 }
 
-// Eight epilogue warps where the epilogue would otherwise set the pace: a tile's mainloop is K / 128
-// k-blocks long, its epilogue always 256 columns, and a GELU about doubles the epilogue's work.
+// Codes in bytes: eight epilogue warps where the epilogue would otherwise set the pace: a tile's
+// mainloop is K / 128 k-blocks long, its epilogue always 256 columns, and a GELU about doubles the
+// epilogue's work.
 template <bool RAW>
 static dvdq_status launch_qgemm_ss(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
                                    int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
     const bool wide_epilogue = w.K <= 2048 || (act != 0 && w.K <= 6144);
-    return wide_epilogue ? launch_qgemm_ss_t<RAW, 8>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
-                         : launch_qgemm_ss_t<RAW, 4>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
+    return wide_epilogue ? launch_qgemm_ss_t<8, RAW, 8>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
+                         : launch_qgemm_ss_t<8, RAW, 4>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
+}
+
+// Packed 4- or 6-bit codes, widened into the shared-memory operand stages by warps.
+template <bool RAW>
+static dvdq_status launch_qgemm_ps(int bits, const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+                                   const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
+                                   int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
+    return bits == 4 ? launch_qgemm_ss_t<4, RAW, 4>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
+                     : launch_qgemm_ss_t<6, RAW, 4>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
 }
 
 }  // namespace dvdq
