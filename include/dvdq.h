@@ -212,7 +212,7 @@ dvdq_status dvdq_qgemm(const void* codes, const float* scales, const int32_t* co
  * R = I (x) H_256 / 16, one absmax scale per token and per 256 rotated channels, codes
  * c = round_half_even(x~ / s).  It writes what dvdq_rotate_quantize would write for Y:
  *
- *   q           this layer's quantizer: scale_group = 0 and container_bits = 8 (or bits = 8)
+ *   q           this layer's quantizer: scale_group = 0 (one scale per token); either code layout
  *   q_next      the next layer's: rot_block = 256, scale_group = 256, container_bits = 8,
  *               bits 4, 6 or 8; the next layer's weights must be rotated with B = 256
  *   codes_next      [M, N] one int8 per code (dvdq_act_codes_bytes_q(M, N, q_next) bytes)

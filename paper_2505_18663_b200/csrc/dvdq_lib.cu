@@ -252,9 +252,9 @@ dvdq_status dvdq_qgemm_fused_rq(const void* codes, const float* scales, const in
     dvdq_status s = check_gemm_args(codes, code_sums, M, q, w);
     if (s != DVDQ_OK) return s;
     if (act != 0 && act != 1) return DVDQ_ERR_UNSUPPORTED;
-    // this layer: per-token scales, codes one int8 each; the next layer: N input channels in whole
+    // this layer: per-token scales; the next layer: N input channels in whole
     // 256-blocks, rotation block = scale group = 256 (what one 256-wide tile owns), codes one int8 each
-    if (q->scale_group != 0 || storage_bits(*q) != 8) return DVDQ_ERR_UNSUPPORTED;
+    if (q->scale_group != 0) return DVDQ_ERR_UNSUPPORTED;
     if (!q_next) return DVDQ_ERR_NULL;
     if (w->N % 256 != 0 || validate_k(w->N) != DVDQ_OK) return DVDQ_ERR_SHAPE;
     if ((s = validate_act_quant(q_next, w->N)) != DVDQ_OK) return s;
@@ -272,7 +272,7 @@ dvdq_status dvdq_qgemm_fused_rq(const void* codes, const float* scales, const in
     fo.y_dbg = static_cast<__nv_bfloat16*>(Y_or_null);
     fo.ldy = ldy;
     fo.bits = q_next->bits;
-    return launch_qgemm_fused(codes, scales, code_sums, M, *w, bias, act, fo, (cudaStream_t)stream);
+    return launch_qgemm_fused(storage_bits(*q), codes, scales, code_sums, M, *w, bias, act, fo, (cudaStream_t)stream);
 }
 
 dvdq_status dvdq_qgemm_int32(const void* codes, const int32_t* code_sums, int64_t M, const dvdq_act_quant* q,

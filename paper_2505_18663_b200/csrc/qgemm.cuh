@@ -760,7 +760,7 @@ inline bool use_ps_kernel() {
 }
 
 // qgemm_fat.cuh: the same with block-wise activation scales
-static dvdq_status launch_qgemm_blk(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+static dvdq_status launch_qgemm_blk(int sb, const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                     const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, cudaStream_t st);
 
 inline dvdq_status launch_qgemm(const void* codes, const float* scales, const int32_t* sums, int64_t M,
@@ -772,8 +772,8 @@ inline dvdq_status launch_qgemm(const void* codes, const float* scales, const in
     const bool raw = acc_out != nullptr;
     const int spr = q.scale_group != 0 ? (int)(w.K / q.scale_group) : 1;  // code sums (and scales) per token
     const int sb = storage_bits(q);
-    if (sb == 8 && !raw && q.scale_group != 0)
-        return launch_qgemm_blk(codes, scales, sums, spr, M, w, bias, act, Y, ldy, st);
+    if (!raw && q.scale_group != 0)
+        return launch_qgemm_blk(sb, codes, scales, sums, spr, M, w, bias, act, Y, ldy, st);
     if (sb == 8 && (raw || q.scale_group == 0))
         return raw ? launch_qgemm_ss<true>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
                    : launch_qgemm_ss<false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);

@@ -61,14 +61,16 @@ struct FusedOut {
     int bits;
 };
 
-template <int MODE>
+template <int MODE, int ABITS>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFatThreads, 1)
-qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW,
+qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmAhi, const __grid_constant__ CUtensorMap tmW,
                  const __grid_constant__ CUtensorMap tmY, const float* __restrict__ scales,
                  const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
                  const __nv_bfloat16* __restrict__ bias, int M, int N, int K, int act, int spr, const FusedOut fo) {
-    using S = SsSmem<8>;
+    using S = SsSmem<ABITS>;
     constexpr int BN = S::BN, BNh = S::BNh;
+    constexpr bool kPackedA = S::kPackedA;  // packed activation codes: the widening warps widen both operands
+    constexpr int AST = S::kAStages, APS = S::kAPackedStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -84,9 +86,9 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     const uint32_t bar0 = sbase + S::kBarOff;
     auto a_full = [&](int s) { return bar0 + 8u * s; };
-    auto a_ready = [&](int s) { return bar0 + 8u * (kSsAStages + s); };
-    auto a_empty = [&](int s) { return bar0 + 8u * (2 * kSsAStages + s); };
-    const uint32_t barw = bar0 + 8u * (3 * kSsAStages);
+    auto a_ready = [&](int s) { return bar0 + 8u * (AST + s); };
+    auto a_empty = [&](int s) { return bar0 + 8u * (2 * AST + s); };
+    const uint32_t barw = bar0 + 8u * (3 * AST);
     auto ops_full = [&](int s) { return barw + 8u * s; };
     auto ops_empty = [&](int s) { return barw + 8u * (kSsStages + s); };
     auto acc_full = [&](int s) { return barw + 8u * (2 * kSsStages + s); };
@@ -94,11 +96,18 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t drain_bar = barw + 8u * (2 * kSsStages + 4);
     auto wp_full = [&](int s) { return drain_bar + 8u * (1 + s); };
     auto wp_empty = [&](int s) { return drain_bar + 8u * (1 + kSsWPackedStages + s); };
+    auto apk_full = [&](int s) { return drain_bar + 8u * (1 + 2 * kSsWPackedStages + s); };
+    auto apk_empty = [&](int s) { return drain_bar + 8u * (1 + 2 * kSsWPackedStages + APS + s); };
     volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + S::kMiscOff);  // [0] tmem base, [1] abort
     volatile uint32_t* abort_flag = misc + 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kSsAStages; ++s) { mbar_init(a_full(s), 1); mbar_init(a_ready(s), 2); mbar_init(a_empty(s), 1); }
+        for (int s = 0; s < AST; ++s) {
+            mbar_init(a_full(s), 1);
+            mbar_init(a_ready(s), kPackedA ? 2 * (kSsWWarps / kUnpackGroups) : 2);
+            mbar_init(a_empty(s), 1);
+        }
+        for (int s = 0; s < APS; ++s) { mbar_init(apk_full(s), 1); mbar_init(apk_empty(s), kSsWWarps / kUnpackGroups); }
         for (int s = 0; s < kSsStages; ++s) { mbar_init(ops_full(s), 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * 8); }
         mbar_init(drain_bar, 1);
@@ -122,24 +131,35 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // ------------------------------------------------------------ TMA producer, activation rows
             if (lane == 0) {
                 tma_prefetch_desc(&tmA);
+                if (ABITS == 6) tma_prefetch_desc(&tmAhi);
+                constexpr int kRing = kPackedA ? APS : AST;
+                constexpr uint32_t kBytes = kPackedA ? S::kAPacked : S::kA;
+                auto ring_full = [&](int s) { return kPackedA ? apk_full(s) : a_full(s); };
+                auto ring_empty = [&](int s) { return kPackedA ? apk_empty(s) : a_empty(s); };
                 uint32_t st = 0, ph = 0, issued = 0;
                 bool ok = true;
                 for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                     const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
                     for (int kb = 0; ok && kb < KB; ++kb) {
-                        if (!mbar_wait(a_empty(st), ph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-                        mbar_arrive_expect_tx(a_full(st), S::kA);
-                        tma_load_2d(sbase + S::kAOff + st * S::kA, &tmA, a_full(st), kb * kBK, m0);
+                        if (!mbar_wait(ring_empty(st), ph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                        mbar_arrive_expect_tx(ring_full(st), kBytes);
+                        if (kPackedA) {
+                            const uint32_t dst = sbase + S::kAPackedOff + st * S::kAPacked;
+                            tma_load_2d(dst, &tmA, ring_full(st), kb * (kBK / 2), m0);
+                            if (ABITS == 6) tma_load_2d(dst + S::kALo, &tmAhi, ring_full(st), kb * (kBK / 4), m0);
+                        } else {
+                            tma_load_2d(sbase + S::kAOff + st * S::kA, &tmA, ring_full(st), kb * kBK, m0);
+                        }
                         ++issued;
-                        if (++st == kSsAStages) { st = 0; ph ^= 1u; }
+                        if (++st == kRing) { st = 0; ph ^= 1u; }
                     }
                 }
                 if (!ok) {  // giving up: let copies already in flight land before the CTA exits (bounded)
-                    const uint32_t n_out = issued < (uint32_t)kSsAStages ? issued : (uint32_t)kSsAStages;
+                    const uint32_t n_out = issued < (uint32_t)kRing ? issued : (uint32_t)kRing;
                     for (uint32_t i = 0; i < n_out; ++i) {
-                        const uint32_t s = (st + kSsAStages - 1 - i) % kSsAStages;
+                        const uint32_t s = (st + kRing - 1 - i) % kRing;
                         const uint32_t p = (s < st) ? ph : (ph ^ 1u);
-                        for (int it = 0; it < (1 << 16) && !mbar_try_wait(a_full(s), p); ++it) {}
+                        for (int it = 0; it < (1 << 16) && !mbar_try_wait(ring_full(s), p); ++it) {}
                     }
                 }
             }
@@ -193,7 +213,7 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         kin += step;
                         const bool last = kin == KBG;
                         if (last) kin = 0;
-                        const uint32_t sa1 = sa + 1 == kSsAStages ? 0u : sa + 1, pa1 = sa + 1 == kSsAStages ? pa ^ 1u : pa;
+                        const uint32_t sa1 = sa + 1 == AST ? 0u : sa + 1, pa1 = sa + 1 == AST ? pa ^ 1u : pa;
                         if (!mbar_wait_warp(a_ready(sa), pa, abort_flag, kWaitPackedFull)) { ok = false; break; }
                         if (!mbar_wait_warp(ops_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                         if (step == 2) {
@@ -219,7 +239,7 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         st += step;
                         if (st == kSsStages) { st = 0; ph ^= 1u; }
                         if (step == 2) { sa = sa1; pa = pa1; }
-                        if (++sa == kSsAStages) { sa = 0; pa ^= 1u; }
+                        if (++sa == AST) { sa = 0; pa ^= 1u; }
                     }
                 }
                 if (elect_one()) tc_commit_pair(drain_bar, 1);
@@ -229,14 +249,17 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             __syncwarp();
         } else {
             // ------------------------------------------------------------ "activation rows landed" -> leader
-            uint32_t st = 0, ph = 0;
-            bool ok = true;
-            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-                for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_wait_warp(a_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                    if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(st), 0));
-                    __syncwarp();
-                    if (++st == kSsAStages) { st = 0; ph ^= 1u; }
+            // (codes in bytes only; packed codes are widened by warps that arrive on the leader's barrier themselves)
+            if constexpr (!kPackedA) {
+                uint32_t st = 0, ph = 0;
+                bool ok = true;
+                for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                    for (int kb = 0; kb < KB; ++kb) {
+                        if (!mbar_wait_warp(a_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                        if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(st), 0));
+                        __syncwarp();
+                        if (++st == AST) { st = 0; ph ^= 1u; }
+                    }
                 }
             }
         }
@@ -252,6 +275,57 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             for (int kb = 0; kb < KB; ++kb) {
                 const uint32_t jj = j++;
                 if (jj % kUnpackGroups != grp) continue;
+                if constexpr (kPackedA) {
+                    // this CTA's 128 token rows of the k-block first: the same job on the activation rings
+                    const uint32_t apst = jj % APS, apph = (jj / APS) & 1u;
+                    const uint32_t awst = jj % AST, awph = (jj / AST) & 1u;
+                    if (!mbar_wait(apk_full(apst), apph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                    const uint32_t pa = sbase + S::kAPackedOff + apst * S::kAPacked;
+                    const uint32_t wd = sbase + S::kAOff + awst * S::kA;
+                    constexpr int kAPieces = (kBM * 4) / 128;
+                    uint4 pl[kAPieces];
+                    uint2 ph2[kAPieces];
+                    uint32_t got = 0u;
+#pragma unroll
+                    for (int it = 0; it < kAPieces; ++it) {
+                        const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                        pl[it] = lds128(pa + row * (kBK / 2) + ck * 16);
+                        got ^= pl[it].w;
+                        if (ABITS == 6) {
+                            ph2[it] = lds64(pa + S::kALo + row * (kBK / 4) + ck * 8);
+                            got ^= ph2[it].y;
+                        }
+                    }
+                    got &= rt_zero;
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_after_loads(apk_empty(apst), got);
+                    if (!mbar_wait(a_empty(awst), awph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                    tc_fence_after();
+#pragma unroll
+                    for (int it = 0; it < kAPieces; ++it) {
+                        const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                        const uint32_t w[4] = {pl[it].x, pl[it].y, pl[it].z, pl[it].w};
+                        uint32_t e[4], o[4];
+#pragma unroll
+                        for (int jw = 0; jw < 4; ++jw) {
+                            if (ABITS == 4) {
+                                e[jw] = (w[jw] << 4) & 0xF0F0F0F0u;
+                                o[jw] = w[jw] & 0xF0F0F0F0u;
+                            } else {
+                                const uint32_t hh = (jw >> 1) ? ph2[it].y : ph2[it].x;
+                                const int a2 = 2 * (jw & 1);
+                                e[jw] = ((w[jw] << 2) & 0x3C3C3C3Cu) | ((hh << (6 - 2 * a2)) & 0xC0C0C0C0u);
+                                o[jw] = ((w[jw] >> 2) & 0x3C3C3C3Cu) | ((hh << (4 - 2 * a2)) & 0xC0C0C0C0u);
+                            }
+                        }
+                        const uint32_t drow = wd + (row >> 3) * 1024 + (row & 7) * 128;
+                        sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[0], o[0], e[1], o[1]);
+                        sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[2], o[2], e[3], o[3]);
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(awst), 0));
+                }
                 const uint32_t pst = jj % kSsWPackedStages, pph = (jj / kSsWPackedStages) & 1u;
                 const uint32_t wst = jj % kSsStages, wph = (jj / kSsStages) & 1u;
                 if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
@@ -299,7 +373,7 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint32_t c_zc = c_delta + CW * 4;                    // (z_n - 8) as a float: exact, |.| <= 8
         const uint32_t c_bias = c_zc + CW * 4;
         const uint32_t stg0 = sbase + S::kStageOutOff + ew * (32 * 64);  // 32 rows x 32 bf16
-        constexpr int kShift = 4;  // the widened weights are 16 x (u - 8)
+        constexpr int kShift = ABITS == 4 ? 8 : ABITS == 6 ? 6 : 4;  // log2 of (A factor 16 / 4 / 1) x (W factor 16)
         if (lane == 0) tma_prefetch_desc(&tmY);
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         uint32_t lt = 0;
@@ -418,7 +492,7 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         float* x_max = reinterpret_cast<float*>(smem + S::kStageOutOff) + ew * 32;
         int* x_sum = reinterpret_cast<int*>(smem + S::kStageOutOff + 8 * 32 * 4) + ew * 32;
         const int pw = (ew ^ 4) - ew;  // the partner's slots are pw * 32 entries away
-        constexpr int kShift = 4;
+        constexpr int kShift = ABITS == 4 ? 8 : ABITS == 6 ? 6 : 4;
         constexpr float kMagic = 12582912.0f;  // 1.5 * 2^23
         const float qmax = (float)((1 << (fo.bits - 1)) - 1);
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
@@ -575,55 +649,52 @@ static bool fat_kernel_registers_fit(Kern kern) {
     return kFatRegsTotal <= kFatThreads * fa.numRegs && fa.numRegs >= kFatRegsWiden && fa.numRegs <= kFatRegsEpilogue;
 }
 
-static dvdq_status launch_qgemm_blk(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
-                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, cudaStream_t st) {
-    using S = SsSmem<8>;
+template <int MODE, int ABITS>
+static dvdq_status launch_qgemm_fat_t(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+                                      const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, const FusedOut& fo,
+                                      cudaStream_t st) {
+    using S = SsSmem<ABITS>;
     const int64_t K = w.K, N = w.N;
     const BlobLayout L = blob_layout(N, K);
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
-    CUtensorMap tmA, tmW, tmY;
-    if (!make_byte_map(&tmA, codes, (uint64_t)K, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B)) return DVDQ_ERR_CUDA;
+    CUtensorMap tmA, tmAhi, tmW, tmY;
+    if (!make_act_maps<ABITS>(codes, M, K, &tmA, &tmAhi)) return DVDQ_ERR_CUDA;
     if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, S::BNh,
                        CU_TENSOR_MAP_SWIZZLE_NONE))
         return DVDQ_ERR_CUDA;
-    if (!make_out_map32(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)) return DVDQ_ERR_CUDA;
-    auto kern = qgemm_fat_kernel<kFatBlk>;
+    if (MODE == kFatFuse) {
+        tmY = tmA;  // unused: the fused epilogue stores codes, scales and sums itself
+    } else if (!make_out_map32(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)) {
+        return DVDQ_ERR_CUDA;
+    }
+    auto kern = qgemm_fat_kernel<MODE, ABITS>;
     if (!fat_kernel_registers_fit(kern)) return DVDQ_ERR_CUDA;
     static PerDevice<int> cache;
     const int max_pairs = resident_pairs(cache, kern, kFatThreads, S::kTotal);
     if (max_pairs == 0) return DVDQ_ERR_CUDA;
     const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + S::BN - 1) / S::BN);
     const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
-    kern<<<2 * pairs, kFatThreads, S::kTotal, st>>>(tmA, tmW, tmY, scales, sums, reinterpret_cast<const float*>(blob + L.delta_offset),
+    kern<<<2 * pairs, kFatThreads, S::kTotal, st>>>(tmA, tmAhi, tmW, tmY, scales, sums, reinterpret_cast<const float*>(blob + L.delta_offset),
                                                     reinterpret_cast<const int32_t*>(blob + L.zc_offset),
-                                                    static_cast<const __nv_bfloat16*>(bias), (int)M, (int)N, (int)K, act, spr, FusedOut{});
+                                                    static_cast<const __nv_bfloat16*>(bias), (int)M, (int)N, (int)K, act, spr, fo);
     return cuda_status(cudaGetLastError());
 }
 
-// The layer (per-token input scales, codes one int8 each) whose epilogue writes the next layer's
-// codes, scales and code sums for rot_block = scale_group = 256 instead of bf16.
-static dvdq_status launch_qgemm_fused(const void* codes, const float* scales, const int32_t* sums, int64_t M,
+// Block-wise activation scales, bf16 output; sb = bits a code is stored in (4, 6 or 8).
+static dvdq_status launch_qgemm_blk(int sb, const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, cudaStream_t st) {
+    if (sb == 4) return launch_qgemm_fat_t<kFatBlk, 4>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, FusedOut{}, st);
+    if (sb == 6) return launch_qgemm_fat_t<kFatBlk, 6>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, FusedOut{}, st);
+    return launch_qgemm_fat_t<kFatBlk, 8>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, FusedOut{}, st);
+}
+
+// The layer (per-token input scales) whose epilogue writes the next layer's codes, scales and code
+// sums for rot_block = scale_group = 256 instead of bf16.
+static dvdq_status launch_qgemm_fused(int sb, const void* codes, const float* scales, const int32_t* sums, int64_t M,
                                       const dvdq_weights& w, const void* bias, int act, const FusedOut& fo, cudaStream_t st) {
-    using S = SsSmem<8>;
-    const int64_t K = w.K, N = w.N;
-    const BlobLayout L = blob_layout(N, K);
-    const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
-    CUtensorMap tmA, tmW;
-    if (!make_byte_map(&tmA, codes, (uint64_t)K, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B)) return DVDQ_ERR_CUDA;
-    if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, S::BNh,
-                       CU_TENSOR_MAP_SWIZZLE_NONE))
-        return DVDQ_ERR_CUDA;
-    auto kern = qgemm_fat_kernel<kFatFuse>;
-    if (!fat_kernel_registers_fit(kern)) return DVDQ_ERR_CUDA;
-    static PerDevice<int> cache;
-    const int max_pairs = resident_pairs(cache, kern, kFatThreads, S::kTotal);
-    if (max_pairs == 0) return DVDQ_ERR_CUDA;
-    const int64_t tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * (N / S::BN);
-    const unsigned pairs = (unsigned)(tiles < max_pairs ? tiles : max_pairs);
-    kern<<<2 * pairs, kFatThreads, S::kTotal, st>>>(tmA, tmW, tmA /* unused */, scales, sums, reinterpret_cast<const float*>(blob + L.delta_offset),
-                                                    reinterpret_cast<const int32_t*>(blob + L.zc_offset),
-                                                    static_cast<const __nv_bfloat16*>(bias), (int)M, (int)N, (int)K, act, 1, fo);
-    return cuda_status(cudaGetLastError());
+    if (sb == 4) return launch_qgemm_fat_t<kFatFuse, 4>(codes, scales, sums, 1, M, w, bias, act, nullptr, 0, fo, st);
+    if (sb == 6) return launch_qgemm_fat_t<kFatFuse, 6>(codes, scales, sums, 1, M, w, bias, act, nullptr, 0, fo, st);
+    return launch_qgemm_fat_t<kFatFuse, 8>(codes, scales, sums, 1, M, w, bias, act, nullptr, 0, fo, st);
 }
 
 }  // namespace dvdq

@@ -541,6 +541,25 @@ inline bool make_out_map32(CUtensorMap* tm, const void* base, uint64_t cols, uin
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor maps of the activation codes: one int8 each -> tiles of 128 tokens x 128 bytes in the operand
+// layout (128-byte swizzle); packed -> 64-byte rows of low bits per k-block (and 32-byte rows of
+// high bits for 6-bit codes), unswizzled, as the weights.
+template <int ABITS>
+static bool make_act_maps(const void* codes, int64_t M, int64_t K, CUtensorMap* tmA, CUtensorMap* tmAhi) {
+    if (ABITS == 8) {
+        if (!make_byte_map(tmA, codes, (uint64_t)K, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B)) return false;
+        *tmAhi = *tmA;  // unused
+        return true;
+    }
+    const uint64_t pitch = (uint64_t)act_row_bytes(K, ABITS);
+    if (!make_byte_map(tmA, codes, (uint64_t)K / 2, (uint64_t)M, pitch, kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_NONE)) return false;
+    *tmAhi = *tmA;
+    if (ABITS == 6 && !make_byte_map(tmAhi, static_cast<const uint8_t*>(codes) + K / 2, (uint64_t)K / 4, (uint64_t)M, pitch, kBK / 4, kBM,
+                                     CU_TENSOR_MAP_SWIZZLE_NONE))
+        return false;
+    return true;
+}
+
 template <int ABITS, bool RAW, int EW>
 static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
@@ -550,21 +569,7 @@ static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, con
     const BlobLayout L = blob_layout(N, K);
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
     CUtensorMap tmA, tmAhi, tmW, tmY;
-    if (ABITS == 8) {
-        if (!make_byte_map(&tmA, codes, (uint64_t)K, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B)) return DVDQ_ERR_CUDA;
-        tmAhi = tmA;  // unused
-    } else {
-        // packed codes: 64-byte rows of low bits per k-block (and 32-byte rows of high bits), unswizzled, as the weights
-        const uint64_t pitch = (uint64_t)act_row_bytes(K, ABITS);
-        if (!make_byte_map(&tmA, codes, (uint64_t)K / 2, (uint64_t)M, pitch, kBK / 2, kBM, CU_TENSOR_MAP_SWIZZLE_NONE)) return DVDQ_ERR_CUDA;
-        if (ABITS == 6) {
-            if (!make_byte_map(&tmAhi, static_cast<const uint8_t*>(codes) + K / 2, (uint64_t)K / 4, (uint64_t)M, pitch, kBK / 4, kBM,
-                               CU_TENSOR_MAP_SWIZZLE_NONE))
-                return DVDQ_ERR_CUDA;
-        } else {
-            tmAhi = tmA;  // unused
-        }
-    }
+    if (!make_act_maps<ABITS>(codes, M, K, &tmA, &tmAhi)) return DVDQ_ERR_CUDA;
     if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, S::BNh,
                        CU_TENSOR_MAP_SWIZZLE_NONE))
         return DVDQ_ERR_CUDA;

@@ -24,10 +24,10 @@ def assert_device_ok():
     assert status == B.OK, f"device status {status} ({B.status_string(status)}), wait id {detail}"
 
 
-def first_stage(x_dev, bits, Bk):
-    """The first layer's own transform: per-token scales, codes one int8 each."""
+def first_stage(x_dev, bits, Bk, container=8):
+    """The first layer's own transform: per-token scales, codes one int8 each or packed."""
     M, K = x_dev.shape
-    q = B.ActQuant(bits, Bk, 0, 8)
+    q = B.ActQuant(bits, Bk, 0, container)
     codes = torch.empty(B.dvdq_act_codes_bytes_q(M, K, q), dtype=torch.uint8, device=DEV)
     scales = torch.empty(M, dtype=torch.float32, device=DEV)
     sums = torch.empty(M, dtype=torch.int32, device=DEV)
@@ -63,12 +63,13 @@ def check_against_oracle(y_bits, nat, scales, sums, bits_next):
     assert np.all(np.abs(nat.reshape(M, -1, G)).max(axis=2)[nz] == qmax)
 
 
+@pytest.mark.parametrize("container", [8, 0])
 @pytest.mark.parametrize("M,K,N,Bk,bits,act,use_bias,bits_next", [
     (200, 512, 512, 256, 4, 1, True, 6),      # a row tail, two column tiles, GELU + bias
     (513, 1024, 256, 1024, 6, 0, False, 4),   # three row tiles (one with a single row), one column tile
     (64, 256, 768, 64, 8, 1, False, 8),
 ])
-def test_fused_epilogue_matches_unfused_output_and_oracle_transform(M, K, N, Bk, bits, act, use_bias, bits_next):
+def test_fused_epilogue_matches_unfused_output_and_oracle_transform(M, K, N, Bk, bits, act, use_bias, bits_next, container):
     g = torch.Generator().manual_seed(M + K + N)
     x = torch.randn(M, K, generator=g)
     x[:, torch.randperm(K, generator=g)[:4]] *= 20.0
@@ -78,7 +79,7 @@ def test_fused_epilogue_matches_unfused_output_and_oracle_transform(M, K, N, Bk,
     u, d, z = orc.prepare_weights(to_bits(wb), Bk, "minmax")
     w, blob = gpu_pack_weights(u, d, z, Bk)
     bias = (torch.randn(N, generator=g) * 0.1).to(torch.bfloat16).to(DEV) if use_bias else None
-    q, codes, scales, sums = first_stage(x.to(DEV), bits, Bk)
+    q, codes, scales, sums = first_stage(x.to(DEV), bits, Bk, container)
     # the unfused layer on the same codes: its bf16 output is what the fused epilogue must reproduce, bit for bit
     Y_ref = torch.empty(M, N, dtype=torch.bfloat16, device=DEV)
     B.dvdq_qgemm(codes, scales, sums, M, q, w, bias, act, Y_ref)
@@ -151,9 +152,9 @@ def test_fused_options_are_validated():
         with pytest.raises(B.DvdqError) as e:
             B.dvdq_qgemm_fused_rq(codes, scales, sums, M, q, w, None, 0, bad, cn, sn, Sn)
         assert e.value.status in (B.ERR_UNSUPPORTED, B.ERR_SHAPE)
-    # the first layer must keep its codes in bytes with per-token scales
+    # the first layer must have per-token scales
     with pytest.raises(B.DvdqError) as e:
-        B.dvdq_qgemm_fused_rq(codes, scales, sums, M, B.ActQuant(4, 256, 0, 0), w, None, 0, B.ActQuant(6, 256, 256, 8), cn, sn, Sn)
+        B.dvdq_qgemm_fused_rq(codes, scales, sums, M, B.ActQuant(4, 256, 256, 8), w, None, 0, B.ActQuant(6, 256, 256, 8), cn, sn, Sn)
     assert e.value.status == B.ERR_UNSUPPORTED
 
 
