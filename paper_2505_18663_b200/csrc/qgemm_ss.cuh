@@ -1,30 +1,33 @@
-// The GEMM for activation codes that are stored one int8 per code (8-bit activations, or 4- and
-// 6-bit codes kept in byte containers): the same contraction and epilogue as qgemm.cuh,
+// The GEMM with one activation scale per token (Eq. 10):
 //
-//   acc_in = sum_k c_ik (u_nk - z_n),   y_in = bf16(acc_in * s_i * Delta_n + bias_n),
+//   acc_in = sum_k c_ik (u_nk - z_n),   y_in = bf16(acc_in * s_i * Delta_n + bias_n).
 //
-// but the activation operand needs no widening, so TMA puts it into shared memory in the layout
-// the tensor core reads (K-major rows of 128 bytes, 128-byte swizzle) and no warp ever touches
-// it.  With no activation stages in tensor memory both accumulators can be 256 columns wide:
-// a CTA pair owns a tile of 256 tokens x 256 channels, tcgen05.mma.cta_group::2.kind::i8
-// 256x256x32 with both operands from shared memory.  Only the 4-bit weights are still widened
-// by warps (each CTA its 128 of the 256 rows), as in qgemm.cuh.
+// A CTA pair owns a tile of 256 tokens x 256 channels: tcgen05.mma.cta_group::2.kind::i8
+// 256x256x32 with BOTH operands from shared memory (K-major rows of 128 bytes, 128-byte swizzle),
+// two 256-column int32 accumulators in tensor memory.  The 4-bit weights are widened to int8 by
+// warps (each CTA its 128 of the 256 rows).  The activation codes come in one of two ways (ABITS):
+//   8      one int8 per code (8-bit activations, or 4- / 6-bit codes kept in byte containers): TMA
+//          puts them into the operand stages as they are and no warp ever touches them;
+//   4, 6   packed: TMA fills a ring of packed tiles and eight more warps widen them into the
+//          operand stages, exactly as the weight warps do for their operand.
 //
-// Roles per CTA (16 or 20 warps):
-//   warp 0      TMA producer of the activation operand: this CTA's 128 token rows of a k-block
-//               straight into a ring of operand stages, deep enough to cover the copy's latency.
+// Roles per CTA (16, 20 or 24 warps):
+//   warp 0      TMA producer of the activation codes: this CTA's 128 token rows of a k-block,
+//               into the operand stages (ring of 6: the depth covers the copy's latency) or into
+//               the ring of packed tiles.
 //   warp 15     TMA producer of packed weight rows, into a ring for the widening warps.
 //   warp 1      (leader CTA) issues the MMAs; tcgen05.commit frees the stage in both CTAs.
-//   warps 2-5  epilogue (tcgen05.ld, zero-point term, scales, bias, GELU, bf16, TMA stores), one
+//   warps 2-5   epilogue (tcgen05.ld, zero-point term, scales, bias, GELU, bf16, TMA stores), one
 //               warp per tensor-memory lane quarter.
-//   warps 16-19 (EW = 8 only) a second epilogue warp per lane quarter; each then takes 128 of the
-//               256 columns.  With one warp per quarter the epilogue, not the MMA, sets the pace
-//               of layers with a short K or a GELU (+13..25 % there); where the mainloop sets it,
-//               the extra warps only compete with the widening warps (-2..7 %).  The host picks.
 //   warps 6-13  widen weight codes into the operand stage (two groups, alternate k-blocks).
-//   warp 14     tells the leader that this CTA's activation rows of a stage have landed (a TMA
-//               copy completes on a barrier of its own CTA).
-// Every wait is bounded, as in qgemm.cuh.
+//   warp 14     (codes in bytes) tells the leader that this CTA's activation rows of a stage have
+//               landed (a TMA copy completes on a barrier of its own CTA).
+//   warps 16-19 (codes in bytes, EW = 8 only) a second epilogue warp per lane quarter; each then
+//               takes 128 of the 256 columns.  With one warp per quarter the epilogue, not the MMA,
+//               sets the pace of layers with a short K or a GELU (+13..25 % there); where the
+//               mainloop sets it, the extra warps only compete with the widening warps (-2..7 %).
+//   warps 16-23 (packed codes) widen activation codes into the operand stage (two groups).
+// Every wait is bounded (mbar_wait).
 #pragma once
 
 #include "qgemm.cuh"
