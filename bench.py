@@ -198,7 +198,7 @@ def config_of(wl, args):
 # layout (container_bits); None where no capture of that kernel in its present form exists.
 # (16384-token capture x 4: traffic grows with M; mean of the four launches of a step)
 QGEMM_DRAM_TRAFFIC_PER_LAUNCH = {0: 0.97e9, 8: 1.15e9}
-RQ_DRAM_TRAFFIC_PER_LAUNCH = {0: 0.83e9, 8: 0.94e9}
+RQ_DRAM_TRAFFIC_PER_LAUNCH = {0: 0.82e9, 8: 0.94e9}
 
 
 class Leg:
@@ -320,7 +320,7 @@ def roofline_blocks(leg, ms_per_step, rq_ms, gm_ms, args, peaks, ceiling, timed_
     rq_gbs = alg / (sum(rq_ms) * 1e-3) / 1e9
     # which library figure a GEMM timed like this compares with: the burst one for a region well under a second
     bf16_kind = "bf16_tflops" if timed_s < 1.0 else "bf16_tflops_sustained"
-    gemm_kernel = "qgemm_ss_kernel" if cont == 8 else "qgemm_kernel"
+    gemm_kernel = "qgemm_ss_kernel<8>" if cont == 8 else "qgemm_ss_kernel<4|6>"
     peak = ceiling["tops"] if ceiling else peaks[bf16_kind] * INT8_OVER_BF16
     roof = {"kernel": gemm_kernel + " (tcgen05.mma kind::i8)", "bound": "tensor", "achieved": gemm_tops, "peak": peak, "unit": "TOPS",
             "frac": gemm_tops / peak,
