@@ -321,6 +321,8 @@ def roofline_blocks(leg, ms_per_step, rq_ms, gm_ms, args, peaks, ceiling, timed_
     # which library figure a GEMM timed like this compares with: the burst one for a region well under a second
     bf16_kind = "bf16_tflops" if timed_s < 1.0 else "bf16_tflops_sustained"
     gemm_kernel = "qgemm_ss_kernel<8>" if cont == 8 else "qgemm_ss_kernel<4|6>"
+    if sg or leg.fuse:
+        gemm_kernel = "qgemm_fat_kernel"
     peak = ceiling["tops"] if ceiling else peaks[bf16_kind] * INT8_OVER_BF16
     roof = {"kernel": gemm_kernel + " (tcgen05.mma kind::i8)", "bound": "tensor", "achieved": gemm_tops, "peak": peak, "unit": "TOPS",
             "frac": gemm_tops / peak,
