@@ -92,7 +92,7 @@ __device__ __forceinline__ void tc_mma_i8_ss_pair(uint32_t d_tmem, uint64_t a_de
 }
 
 template <int ABITS>
-constexpr int ss_warps(int ew) { return ABITS != 8 ? kSsFirstAWarp + kSsAWarps : (ew == 8 ? kSsFirstEpilogueWarp2 + 4 : kSsFirstEpilogueWarp2); }
+constexpr int ss_warps(int ew) { return ew == 8 ? kSsFirstEpilogueWarp2 + 4 : (ABITS != 8 ? kSsFirstAWarp + kSsAWarps : kSsFirstEpilogueWarp2); }
 
 template <int ABITS, bool RAW, int EW>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(ss_warps<ABITS>(EW) * 32, 1)
@@ -105,7 +105,9 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     constexpr int BN = S::BN, BNh = S::BNh;
     constexpr bool kPackedA = S::kPackedA;
     constexpr int AST = S::kAStages, APS = S::kAPackedStages;
-    static_assert(!kPackedA || EW == 4, "packed activation codes: the second set of epilogue warps gives way to the widening warps");
+    // packed codes with the second set of epilogue warps (layers whose epilogue sets the pace): the
+    // eight weight warps widen both operands of their k-block instead of eight more warps
+    constexpr bool kWidenBoth = kPackedA && EW == 8;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -269,7 +271,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             mbar_wait(drain_bar, 0u, abort_flag, kWaitDrain);
         }
         __syncwarp();
-    } else if (warp < kSsFirstWWarp || (!kPackedA && warp >= kSsFirstEpilogueWarp2)) {
+    } else if (warp < kSsFirstWWarp || (EW == 8 && warp >= kSsFirstEpilogueWarp2)) {
         // ------------------------------------------------------------ epilogue
         const int q = warp & 3;  // tensor-memory lane quarter this warp may read
         const int half = warp >= kSsFirstEpilogueWarp2 ? 1 : 0;  // EW = 8: which 128 of the tile's 256 columns
@@ -407,6 +409,57 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int kb = 0; kb < KB; ++kb) {
             const uint32_t jj = j++;
             if (jj % kUnpackGroups != grp) continue;
+            if constexpr (kWidenBoth) {
+                // this CTA's 128 token rows of the k-block first: the same job on the activation rings
+                const uint32_t apst = jj % APS, apph = (jj / APS) & 1u;
+                const uint32_t awst = jj % AST, awph = (jj / AST) & 1u;
+                if (!mbar_wait(apk_full(apst), apph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                const uint32_t pa = sbase + S::kAPackedOff + apst * S::kAPacked;
+                const uint32_t wd = sbase + S::kAOff + awst * S::kA;
+                constexpr int kAPieces = (kBM * 4) / 128;
+                uint4 pl[kAPieces];
+                uint2 ph2[kAPieces];
+                uint32_t got = 0u;
+#pragma unroll
+                for (int it = 0; it < kAPieces; ++it) {
+                    const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                    pl[it] = lds128(pa + row * (kBK / 2) + ck * 16);
+                    got ^= pl[it].w;
+                    if (ABITS == 6) {
+                        ph2[it] = lds64(pa + S::kALo + row * (kBK / 4) + ck * 8);
+                        got ^= ph2[it].y;
+                    }
+                }
+                got &= rt_zero;
+                __syncwarp();
+                if (lane == 0) mbar_arrive_after_loads(apk_empty(apst), got);
+                if (!mbar_wait(a_empty(awst), awph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int it = 0; it < kAPieces; ++it) {
+                    const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                    const uint32_t w[4] = {pl[it].x, pl[it].y, pl[it].z, pl[it].w};
+                    uint32_t e[4], o[4];
+#pragma unroll
+                    for (int jw = 0; jw < 4; ++jw) {
+                        if (ABITS == 4) {
+                            e[jw] = (w[jw] << 4) & 0xF0F0F0F0u;
+                            o[jw] = w[jw] & 0xF0F0F0F0u;
+                        } else {
+                            const uint32_t hh = (jw >> 1) ? ph2[it].y : ph2[it].x;
+                            const int a2 = 2 * (jw & 1);
+                            e[jw] = ((w[jw] << 2) & 0x3C3C3C3Cu) | ((hh << (6 - 2 * a2)) & 0xC0C0C0C0u);
+                            o[jw] = ((w[jw] >> 2) & 0x3C3C3C3Cu) | ((hh << (4 - 2 * a2)) & 0xC0C0C0C0u);
+                        }
+                    }
+                    const uint32_t drow = wd + (row >> 3) * 1024 + (row & 7) * 128;
+                    sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[0], o[0], e[1], o[1]);
+                    sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[2], o[2], e[3], o[3]);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(awst), 0));
+            }
             const uint32_t pst = jj % kSsWPackedStages, pph = (jj / kSsWPackedStages) & 1u;
             const uint32_t wst = jj % kSsStages, wph = (jj / kSsStages) & 1u;
             if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
@@ -458,11 +511,11 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
             }
         }
-    } else if (kPackedA && warp >= kSsFirstAWarp) {
+    } else if (kPackedA && EW == 4 && warp >= kSsFirstAWarp) {
         // ------------------------------------------------------------ widen activation codes -> shared memory
         // The same job as the weight warps': this CTA's 128 token rows x 128 codes of a k-block, 16 bytes
         // of packed low bits (and 8 bytes of high bits) per piece, into the K-major 128-byte-swizzled stage.
-        if constexpr (kPackedA) {
+        if constexpr (kPackedA && EW == 4) {
             const uint32_t grp = (uint32_t)(warp - kSsFirstAWarp) >> 2;
             const int u = (threadIdx.x - kSsFirstAWarp * 32) & 127;
             uint32_t j = 0;
@@ -614,8 +667,12 @@ template <bool RAW>
 static dvdq_status launch_qgemm_ps(int bits, const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
                                    int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
-    return bits == 4 ? launch_qgemm_ss_t<4, RAW, 4>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
-                     : launch_qgemm_ss_t<6, RAW, 4>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
+    const bool wide_epilogue = w.K <= 2048 || (act != 0 && w.K <= 6144);  // as for codes in bytes
+    if (bits == 4)
+        return wide_epilogue ? launch_qgemm_ss_t<4, RAW, 8>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
+                             : launch_qgemm_ss_t<4, RAW, 4>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
+    return wide_epilogue ? launch_qgemm_ss_t<6, RAW, 8>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st)
+                         : launch_qgemm_ss_t<6, RAW, 4>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
 }
 
 }  // namespace dvdq
