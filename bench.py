@@ -226,8 +226,13 @@ class Leg:
                 weights.append((B.dvdq_pack_weights(u, d, z, rot, blob), blob, W.make_bias(wl, layer, device=dev)))
                 del u
             Ys = [torch.empty(M, layer.N, dtype=torch.bfloat16, device=dev) for layer in wl.layers]
-            shared = dict(xs=xs, weights=weights, Ys=Ys)
+            # one scratch area for the int8 weight operand of whichever layer runs next (rewritten before every GEMM)
+            scratch = torch.empty(max(layer.N * layer.K for layer in wl.layers), dtype=torch.uint8, device=dev)
+            shared = dict(xs=xs, weights=weights, Ys=Ys, scratch=scratch)
         self.shared = shared
+        # where the GEMM's int8 weight operand comes from: widened inside the GEMM by every tile ("tile"), written
+        # into the scratch area before every GEMM launch ("launch", inside the timed region), or kept ("resident")
+        self.operand = args.weight_operand
         self.layers = []
         for i, layer in enumerate(wl.layers):
             q = B.ActQuant(layer.bits, layer.rot_block, args.scale_group, container)
@@ -239,6 +244,10 @@ class Leg:
             # in a chain every layer but the first reads the previous layer's output
             x = shared["Ys"][i - 1] if (wl.chain and i > 0) else shared["xs"][layer.K]
             w, _, bias = shared["weights"][i]
+            if self.operand == "resident":
+                keep = torch.empty(layer.N * layer.K, dtype=torch.uint8, device=dev)
+                w = B.dvdq_widen_weights(w, keep)
+                self.kept = getattr(self, "kept", []) + [keep]
             self.layers.append(dict(layer=layer, q=q, x=x, w=w, bias=bias, Y=shared["Ys"][i],
                                     codes=torch.empty(B.dvdq_act_codes_bytes_q(M, layer.K, q), dtype=torch.uint8, device=dev),
                                     scales=torch.empty(n_scales, dtype=torch.float32, device=dev),
@@ -256,17 +265,20 @@ class Leg:
                 events[li][1].record()
             if rq_only:
                 continue
+            w = L["w"]
+            if self.operand == "launch":
+                w = B.dvdq_widen_weights(w, self.shared["scratch"][:L["layer"].N * L["layer"].K])
             if self.fuse and li + 1 < n:
                 nx = self.layers[li + 1]
-                B.dvdq_qgemm_fused_rq(L["codes"], L["scales"], L["sums"], self.M, L["q"], L["w"], L["bias"], L["layer"].act,
+                B.dvdq_qgemm_fused_rq(L["codes"], L["scales"], L["sums"], self.M, L["q"], w, L["bias"], L["layer"].act,
                                       nx["q"], nx["codes"], nx["scales"], nx["sums"])
             else:
-                B.dvdq_qgemm(L["codes"], L["scales"], L["sums"], self.M, L["q"], L["w"], L["bias"], L["layer"].act, L["Y"])
+                B.dvdq_qgemm(L["codes"], L["scales"], L["sums"], self.M, L["q"], w, L["bias"], L["layer"].act, L["Y"])
             if events is not None:
                 events[li][2].record()
 
     def launches_per_step(self):
-        return 2 * len(self.layers) - (len(self.layers) - 1 if self.fuse else 0)
+        return 2 * len(self.layers) - (len(self.layers) - 1 if self.fuse else 0) + (len(self.layers) if self.operand == "launch" else 0)
 
     def timed(self, steps, warmup, barrier, rq_only=False):
         """(ms per step, per-layer rq ms, per-layer GEMM ms) from CUDA events inside the timed region."""
@@ -512,7 +524,9 @@ def run_e2e(args, wl, leg, dev, B, dist, world):
             host_x[L["layer"].K] = L["x"].to("cpu").pin_memory()
     host_y = [torch.empty(M, maxN, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
     dev_x = [torch.empty(M, maxK, dtype=torch.bfloat16, device=dev) for _ in range(2)]
-    ws = torch.empty(max(B.dvdq_qlinear_workspace_bytes(M, L["layer"].K, L["q"]) for L in layers), dtype=torch.uint8, device=dev)
+    # room for the int8 weight operand behind the codes: dvdq_qlinear then writes it once per call
+    extra = 0 if args.weight_operand == "tile" else max(B.dvdq_weight_operand_bytes(L["layer"].N, L["layer"].K) for L in layers) + 256
+    ws = torch.empty(max(B.dvdq_qlinear_workspace_bytes(M, L["layer"].K, L["q"]) for L in layers) + extra, dtype=torch.uint8, device=dev)
     h2d = sum(M * L["layer"].K * 2 for L in layers)
     d2h = sum(M * L["layer"].N * 2 for L in layers)
     s_in, s_run, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev), torch.cuda.Stream(dev)
@@ -598,6 +612,10 @@ def main():
     ap.add_argument("--fuse", action="store_true",
                     help="chain workloads: every layer but the last writes the next layer's codes from its epilogue "
                          "(dvdq_qgemm_fused_rq, rotation block = scale group = 256) instead of bf16; needs --container 8")
+    ap.add_argument("--weight-operand", default="launch", choices=["launch", "tile", "resident"],
+                    help="where the GEMM's int8 weight operand comes from: written into a scratch area by a widening "
+                         "kernel before every GEMM launch, inside the timed region (launch); widened inside the GEMM by "
+                         "every output tile (tile); or written once and kept, 8 more bits per weight (resident)")
     ap.add_argument("--bits", type=int, default=0, help="override the activation bit width of every layer (4, 6 or 8)")
     args = ap.parse_args()
     from paper_2505_18663_b200 import workloads as W

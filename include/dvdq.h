@@ -93,6 +93,8 @@ typedef struct {
     int32_t  k_layout;   /* storage order of the K axis shared with the activation codes */
     const void* blob;    /* device */
     uint64_t blob_bytes;
+    const void* operand; /* device, or NULL: the same codes one int8 each (dvdq_widen_weights) */
+    uint64_t operand_bytes;
 } dvdq_weights;
 
 /* ---- size queries (host only, no CUDA calls) ------------------------------------ */
@@ -105,6 +107,8 @@ size_t dvdq_act_codes_bytes_q(int64_t M, int64_t K, const dvdq_act_quant* q);
 size_t dvdq_act_scales_count(int64_t M, int64_t K, const dvdq_act_quant* q);
 /* Bytes of the device blob that dvdq_pack_weights() writes for an [N, K] matrix. 0 on bad input. */
 size_t dvdq_weight_blob_bytes(int64_t N, int64_t K);
+/* Bytes of the int8 copy of the codes that dvdq_widen_weights() writes for an [N, K] matrix: N * K. 0 on bad input. */
+size_t dvdq_weight_operand_bytes(int64_t N, int64_t K);
 /* Bytes of the workspace dvdq_qlinear() needs (codes, scales and code sums of X). 0 on bad input. */
 size_t dvdq_qlinear_workspace_bytes(int64_t M, int64_t K, const dvdq_act_quant* q);
 
@@ -140,6 +144,21 @@ dvdq_status dvdq_rotate_quantize(const void* X_bf16, int64_t M, int64_t K, int64
 dvdq_status dvdq_pack_weights(const uint8_t* Wq, const float* delta, const int32_t* zero,
                               int64_t N, int64_t K, int32_t rot_block,
                               void* blob_out, dvdq_weights* out /* host */, void* cuda_stream);
+
+/* ---- the weight operand of the GEMM, written once instead of once per tile: Sec. 3.1, Eq. 10 ----
+ *
+ * The tensor cores take int8 operands, so every GEMM widens the 4-bit codes (u - 8): by default
+ * inside the kernel, each output tile for itself.  This call does it once, into a buffer of the
+ * caller's: operand_out (device, dvdq_weight_operand_bytes(N, K) = N * K bytes, 256-byte
+ * aligned) receives one int8 per code, and *out is *w referring to that buffer as well.  GEMMs
+ * given `out` then read the operand with TMA and widen no weights; all results are bit-identical
+ * to those with `w`.  The blob stays the format of record (the
+ * scales, zero points and 4-bit codes are still read from it); the buffer may be a scratch area
+ * that is rewritten before every launch (one call per layer and step costs about 1 % of a GEMM
+ * over 65536 tokens) or kept for the life of the weights (at 8 more bits per weight).  w and out
+ * may be the same object.  dvdq_qgemm_int32 always reads the 4-bit codes. */
+dvdq_status dvdq_widen_weights(const dvdq_weights* w /* host */, void* operand_out, size_t operand_bytes,
+                               dvdq_weights* out /* host */, void* cuda_stream);
 
 /* ---- (0) offline weight rotation: Eq. 10, W^ = Quant(W H); Sec. 3.2 ------------------------
  *
@@ -227,7 +246,9 @@ dvdq_status dvdq_qgemm_fused_rq(const void* codes, const float* scales, const in
                                 void* Y_bf16_or_null, int64_t ldy, void* cuda_stream);
 
 /* ---- (1)+(2): one quantized linear layer ------------------------------------------
- * workspace: dvdq_qlinear_workspace_bytes(M, K, q) bytes, 256-byte aligned. */
+ * workspace: dvdq_qlinear_workspace_bytes(M, K, q) bytes, 256-byte aligned.  Given
+ * dvdq_weight_operand_bytes(N, K) + 256 bytes more (and M >= 1024, no operand in `w` already) the call writes the int8 weight operand behind the codes first, as
+ * dvdq_widen_weights would, and the GEMM reads it from there: same result bits, faster GEMM. */
 dvdq_status dvdq_qlinear(const void* X_bf16, int64_t M, int64_t ldx, const dvdq_act_quant* q,
                          const dvdq_weights* w /* host */, const void* bias_bf16, int32_t act,
                          void* Y_bf16, int64_t ldy, void* workspace, size_t workspace_bytes,

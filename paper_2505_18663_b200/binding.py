@@ -25,6 +25,7 @@ EXPORTS = [
     "dvdq_qlinear", "dvdq_qlinear_static", "dvdq_qgemm_fused_rq", "dvdq_qgemm_int32", "dvdq_pack_act_codes", "dvdq_unpack_act_codes",
     "dvdq_unpack_weights", "dvdq_last_device_status",
     "dvdq_rotate_weights", "dvdq_quantize_weights_symmetric", "dvdq_int8_mma_ceiling", "dvdq_debug_wait_timeout",
+    "dvdq_weight_operand_bytes", "dvdq_widen_weights",
     "dvdq_bgr_quantize", "dvdq_gbs_l1_terms", "dvdq_gbs_init", "dvdq_gbs_next_bits", "dvdq_gbs_observe",
 ]
 
@@ -46,7 +47,7 @@ class Weights(C.Structure):
     """dvdq_weights: host handle of a packed weight blob."""
     _fields_ = [("magic", C.c_uint32), ("version", C.c_uint32), ("N", C.c_int64), ("K", C.c_int64),
                 ("rot_block", C.c_int32), ("k_layout", C.c_int32), ("blob", C.c_void_p),
-                ("blob_bytes", C.c_uint64)]
+                ("blob_bytes", C.c_uint64), ("operand", C.c_void_p), ("operand_bytes", C.c_uint64)]
 
 
 class GbsState(C.Structure):
@@ -84,6 +85,8 @@ def load():
         "dvdq_act_codes_bytes_q": (sz, [i64, i64, aq]),
         "dvdq_act_scales_count": (sz, [i64, i64, aq]),
         "dvdq_weight_blob_bytes": (sz, [i64, i64]),
+        "dvdq_weight_operand_bytes": (sz, [i64, i64]),
+        "dvdq_widen_weights": (C.c_int, [wp, p, sz, wp, p]),
         "dvdq_qlinear_workspace_bytes": (sz, [i64, i64, aq]),
         "dvdq_rotate_quantize": (C.c_int, [p, i64, i64, i64, aq, p, p, p, p]),
         "dvdq_pack_weights": (C.c_int, [p, p, p, i64, i64, i32, p, wp, p]),
@@ -301,6 +304,19 @@ def dvdq_quantize_weights_symmetric(W: torch.Tensor, rot_block: int, blob: torch
                                                   _ptr(blob, torch.uint8, "blob"), C.byref(w), _stream(stream)),
            "dvdq_quantize_weights_symmetric")
     return w
+
+
+def dvdq_weight_operand_bytes(N: int, K: int) -> int:
+    return int(load().dvdq_weight_operand_bytes(N, K))
+
+
+def dvdq_widen_weights(w: Weights, operand: torch.Tensor, stream=None) -> Weights:
+    """Writes the 4-bit codes of `w` one int8 each into `operand` (uint8, >= N * K bytes) and returns
+    a handle that refers to both; GEMMs given it read the weight operand with TMA."""
+    out = Weights()
+    _check(load().dvdq_widen_weights(C.byref(w), _ptr(operand, torch.uint8, "operand"), operand.numel(), C.byref(out),
+                                     _stream(stream)), "dvdq_widen_weights")
+    return out
 
 
 def dvdq_int8_mma_ceiling(iters: int, stream=None) -> int:

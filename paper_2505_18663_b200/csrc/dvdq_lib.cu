@@ -59,6 +59,10 @@ dvdq_status validate_weights(const dvdq_weights* w) {
     if (w->blob_bytes != (uint64_t)blob_layout(w->N, w->K).total) return DVDQ_ERR_BLOB;
     if (w->k_layout != kKLayoutNatural) return DVDQ_ERR_BLOB;
     if (!aligned(w->blob, 256)) return DVDQ_ERR_ALIGN;
+    if (w->operand != nullptr) {
+        if (w->operand_bytes != (uint64_t)(w->N * w->K)) return DVDQ_ERR_BLOB;
+        if (!aligned(w->operand, 256)) return DVDQ_ERR_ALIGN;
+    }
     return DVDQ_OK;
 }
 
@@ -122,6 +126,11 @@ size_t dvdq_weight_blob_bytes(int64_t N, int64_t K) {
     return (size_t)blob_layout(N, K).total;
 }
 
+size_t dvdq_weight_operand_bytes(int64_t N, int64_t K) {
+    if (N <= 0 || N % 8 != 0 || validate_k(K) != DVDQ_OK) return 0;
+    return (size_t)(N * K);
+}
+
 size_t dvdq_qlinear_workspace_bytes(int64_t M, int64_t K, const dvdq_act_quant* q) {
     if (M < 0 || validate_k(K) != DVDQ_OK || validate_act_quant(q, K) != DVDQ_OK) return 0;
     return (size_t)workspace_plan(M, K, *q).total;
@@ -160,6 +169,8 @@ dvdq_status dvdq_pack_weights(const uint8_t* Wq, const float* delta, const int32
     out->k_layout = kKLayoutNatural;
     out->blob = blob_out;
     out->blob_bytes = (uint64_t)blob_layout(N, K).total;
+    out->operand = nullptr;
+    out->operand_bytes = 0;
     return DVDQ_OK;
 }
 
@@ -216,6 +227,28 @@ dvdq_status dvdq_quantize_weights_symmetric(const void* W, int64_t N, int64_t K,
     out->k_layout = kKLayoutNatural;
     out->blob = blob_out;
     out->blob_bytes = (uint64_t)blob_layout(N, K).total;
+    out->operand = nullptr;
+    out->operand_bytes = 0;
+    return DVDQ_OK;
+}
+
+dvdq_status dvdq_widen_weights(const dvdq_weights* w, void* operand_out, size_t operand_bytes, dvdq_weights* out, void* stream) {
+    if (!out) return DVDQ_ERR_NULL;
+    dvdq_weights in;
+    if (w) { in = *w; in.operand = nullptr; in.operand_bytes = 0; }
+    dvdq_status s = validate_weights(w ? &in : nullptr);
+    if (s != DVDQ_OK) return s;
+    if (!operand_out) return DVDQ_ERR_NULL;
+    if (operand_bytes < (size_t)(in.N * in.K)) return DVDQ_ERR_WORKSPACE;
+    if (!aligned(operand_out, 256)) return DVDQ_ERR_ALIGN;
+    if ((s = check_device_arch()) != DVDQ_OK) return s;
+    const int64_t pieces = in.N * (in.K / 32);
+    widen_weights_kernel<<<grid_for(pieces, 256), 256, 0, (cudaStream_t)stream>>>(
+        static_cast<const uint8_t*>(in.blob) + blob_layout(in.N, in.K).codes_offset, pieces, static_cast<uint8_t*>(operand_out));
+    if ((s = cuda_status(cudaGetLastError())) != DVDQ_OK) return s;
+    in.operand = operand_out;
+    in.operand_bytes = (uint64_t)(in.N * in.K);
+    *out = in;
     return DVDQ_OK;
 }
 
@@ -303,15 +336,31 @@ static dvdq_status check_qlinear_args(const void* X, int64_t M, int64_t ldx, con
     return check_device_arch();
 }
 
+constexpr int64_t kWidenOnceMinTokens = 1024;  // four rows of output tiles share one written operand
+
 static dvdq_status qlinear_on_workspace(const void* X, int64_t M, int64_t ldx, const dvdq_act_quant* q, const dvdq_weights* w,
-                                        const void* bias, int32_t act, void* Y, int64_t ldy, uint8_t* ws, void* stream) {
+                                        const void* bias, int32_t act, void* Y, int64_t ldy, uint8_t* ws, size_t ws_bytes,
+                                        void* stream) {
     const WorkspacePlan p = workspace_plan(M, w->K, *q);
     void* codes = ws + p.codes_off;
     float* scales = reinterpret_cast<float*>(ws + p.scales_off);
     int32_t* sums = reinterpret_cast<int32_t*>(ws + p.sums_off);
     dvdq_status s = launch_rotate_quantize(X, M, w->K, ldx, *q, codes, scales, sums, (cudaStream_t)stream);
     if (s != DVDQ_OK) return s;
-    return launch_qgemm(codes, scales, sums, M, *q, *w, bias, act, Y, ldy, nullptr, 0, (cudaStream_t)stream);
+    // Room behind the codes for the int8 weight operand, and enough token tiles to share it: written once
+    // per call instead of once per tile (same result bits).
+    dvdq_weights wide = *w;
+    const int64_t operand_off = align_up(p.total, 256);
+    if (w->operand == nullptr && M >= kWidenOnceMinTokens &&
+        ws_bytes >= (size_t)(operand_off + w->N * w->K)) {
+        const int64_t pieces = w->N * (w->K / 32);
+        widen_weights_kernel<<<grid_for(pieces, 256), 256, 0, (cudaStream_t)stream>>>(
+            static_cast<const uint8_t*>(w->blob) + blob_layout(w->N, w->K).codes_offset, pieces, ws + operand_off);
+        if ((s = cuda_status(cudaGetLastError())) != DVDQ_OK) return s;
+        wide.operand = ws + operand_off;
+        wide.operand_bytes = (uint64_t)(w->N * w->K);
+    }
+    return launch_qgemm(codes, scales, sums, M, *q, wide, bias, act, Y, ldy, nullptr, 0, (cudaStream_t)stream);
 }
 
 dvdq_status dvdq_qlinear(const void* X, int64_t M, int64_t ldx, const dvdq_act_quant* q, const dvdq_weights* w,
@@ -323,7 +372,7 @@ dvdq_status dvdq_qlinear(const void* X, int64_t M, int64_t ldx, const dvdq_act_q
     if (!workspace) return DVDQ_ERR_NULL;
     if (!aligned(workspace, 256)) return DVDQ_ERR_ALIGN;
     if (workspace_bytes < (size_t)workspace_plan(M, w->K, *q).total) return DVDQ_ERR_WORKSPACE;
-    return qlinear_on_workspace(X, M, ldx, q, w, bias, act, Y, ldy, static_cast<uint8_t*>(workspace), stream);
+    return qlinear_on_workspace(X, M, ldx, q, w, bias, act, Y, ldy, static_cast<uint8_t*>(workspace), workspace_bytes, stream);
 }
 
 // Scratch of dvdq_qlinear_static: part of the library image, so no allocation is ever needed.
@@ -341,7 +390,7 @@ dvdq_status dvdq_qlinear_static(const void* X, int64_t M, int64_t ldx, const dvd
         return cudaGetSymbolAddress(&ptr, g_static_scratch) == cudaSuccess && ptr != nullptr;
     });
     if (!ws) return DVDQ_ERR_CUDA;
-    return qlinear_on_workspace(X, M, ldx, q, w, bias, act, Y, ldy, static_cast<uint8_t*>(*ws), stream);
+    return qlinear_on_workspace(X, M, ldx, q, w, bias, act, Y, ldy, static_cast<uint8_t*>(*ws), (size_t)DVDQ_STATIC_SCRATCH_BYTES, stream);
 }
 
 dvdq_status dvdq_pack_act_codes(const int8_t* codes_nat, int64_t M, int64_t K, const dvdq_act_quant* q,

@@ -61,16 +61,16 @@ struct FusedOut {
     int bits;
 };
 
-template <int MODE, int ABITS>
+template <int MODE, int ABITS, bool WOP>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kFatThreads, 1)
 qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmAhi, const __grid_constant__ CUtensorMap tmW,
                  const __grid_constant__ CUtensorMap tmY, const float* __restrict__ scales,
                  const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
                  const __nv_bfloat16* __restrict__ bias, int M, int N, int K, int act, int spr, const FusedOut fo) {
-    using S = SsSmem<ABITS>;
+    using S = SsSmem<ABITS, WOP>;  // WOP: the weight operand is in global memory already and comes by TMA (see qgemm_ss.cuh)
     constexpr int BN = S::BN, BNh = S::BNh;
     constexpr bool kPackedA = S::kPackedA;  // packed activation codes: the widening warps widen both operands
-    constexpr int AST = S::kAStages, APS = S::kAPackedStages;
+    constexpr int AST = S::kAStages, APS = S::kAPackedStages, WST = S::kWStages, WPB = S::kWpBars;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -90,14 +90,14 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     auto a_empty = [&](int s) { return bar0 + 8u * (2 * AST + s); };
     const uint32_t barw = bar0 + 8u * (3 * AST);
     auto ops_full = [&](int s) { return barw + 8u * s; };
-    auto ops_empty = [&](int s) { return barw + 8u * (kSsStages + s); };
-    auto acc_full = [&](int s) { return barw + 8u * (2 * kSsStages + s); };
-    auto acc_empty = [&](int s) { return barw + 8u * (2 * kSsStages + 2 + s); };
-    const uint32_t drain_bar = barw + 8u * (2 * kSsStages + 4);
+    auto ops_empty = [&](int s) { return barw + 8u * (WST + s); };
+    auto acc_full = [&](int s) { return barw + 8u * (2 * WST + s); };
+    auto acc_empty = [&](int s) { return barw + 8u * (2 * WST + 2 + s); };
+    const uint32_t drain_bar = barw + 8u * (2 * WST + 4);
     auto wp_full = [&](int s) { return drain_bar + 8u * (1 + s); };
-    auto wp_empty = [&](int s) { return drain_bar + 8u * (1 + kSsWPackedStages + s); };
-    auto apk_full = [&](int s) { return drain_bar + 8u * (1 + 2 * kSsWPackedStages + s); };
-    auto apk_empty = [&](int s) { return drain_bar + 8u * (1 + 2 * kSsWPackedStages + APS + s); };
+    auto wp_empty = [&](int s) { return drain_bar + 8u * (1 + WPB + s); };
+    auto apk_full = [&](int s) { return drain_bar + 8u * (1 + 2 * WPB + s); };
+    auto apk_empty = [&](int s) { return drain_bar + 8u * (1 + 2 * WPB + APS + s); };
     volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + S::kMiscOff);  // [0] tmem base, [1] abort
     volatile uint32_t* abort_flag = misc + 1;
 
@@ -108,10 +108,10 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             mbar_init(a_empty(s), 1);
         }
         for (int s = 0; s < APS; ++s) { mbar_init(apk_full(s), 1); mbar_init(apk_empty(s), kSsWWarps / kUnpackGroups); }
-        for (int s = 0; s < kSsStages; ++s) { mbar_init(ops_full(s), 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
+        for (int s = 0; s < WST; ++s) { mbar_init(ops_full(s), WOP ? 2 : 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * 8); }
         mbar_init(drain_bar, 1);
-        for (int s = 0; s < kSsWPackedStages; ++s) { mbar_init(wp_full(s), 1); mbar_init(wp_empty(s), kSsWWarps / kUnpackGroups); }
+        for (int s = 0; s < WPB; ++s) { mbar_init(wp_full(s), 1); mbar_init(wp_empty(s), kSsWWarps / kUnpackGroups); }
         misc[1] = 0u;
         fence_mbar_init();
     }
@@ -125,6 +125,19 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = misc[0];
 
+    // WOP: "this CTA's weight rows of a stage have landed" -> leader (a TMA copy completes on a barrier of its own CTA)
+    auto forward_w = [&]() {
+        uint32_t st = 0, ph = 0;
+        bool ok = true;
+        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!mbar_wait_warp(wp_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(st), 0));
+                __syncwarp();
+                if (++st == WST) { st = 0; ph ^= 1u; }
+            }
+        }
+    };
     if (warp < kFatFirstWWarp) {
         regs_give<kFatRegsLoader>();
         if (warp == 0) {
@@ -173,17 +186,23 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                     const int n0 = (tile % num_n) * BN + (int)rank * BNh;
                     for (int kb = 0; ok && kb < KB; ++kb) {
-                        if (!mbar_wait(wp_empty(wst), wph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
-                        mbar_arrive_expect_tx(wp_full(wst), S::kWPacked);
-                        tma_load_2d(sbase + S::kWPackedOff + wst * S::kWPacked, &tmW, wp_full(wst), kb * (kBK / 2), n0);
+                        if (WOP) {  // straight into the operand stage, which the MMA's commit frees
+                            if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                            mbar_arrive_expect_tx(wp_full(wst), S::kW);
+                            tma_load_2d(sbase + S::kWOff + wst * S::kW, &tmW, wp_full(wst), kb * kBK, n0);
+                        } else {
+                            if (!mbar_wait(wp_empty(wst), wph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
+                            mbar_arrive_expect_tx(wp_full(wst), S::kWPacked);
+                            tma_load_2d(sbase + S::kWPackedOff + wst * S::kWPacked, &tmW, wp_full(wst), kb * (kBK / 2), n0);
+                        }
                         ++wissued;
-                        if (++wst == kSsWPackedStages) { wst = 0; wph ^= 1u; }
+                        if (++wst == WPB) { wst = 0; wph ^= 1u; }
                     }
                 }
                 if (!ok) {
-                    const uint32_t w_out = wissued < (uint32_t)kSsWPackedStages ? wissued : (uint32_t)kSsWPackedStages;
+                    const uint32_t w_out = wissued < (uint32_t)WPB ? wissued : (uint32_t)WPB;
                     for (uint32_t i = 0; i < w_out; ++i) {
-                        const uint32_t s = (wst + kSsWPackedStages - 1 - i) % kSsWPackedStages;
+                        const uint32_t s = (wst + WPB - 1 - i) % WPB;
                         const uint32_t p = (s < wst) ? wph : (wph ^ 1u);
                         for (int it = 0; it < (1 << 16) && !mbar_try_wait(wp_full(s), p); ++it) {}
                     }
@@ -237,7 +256,7 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         }
                         __syncwarp();
                         st += step;
-                        if (st == kSsStages) { st = 0; ph ^= 1u; }
+                        if (st == WST) { st = 0; ph ^= 1u; }
                         if (step == 2) { sa = sa1; pa = pa1; }
                         if (++sa == AST) { sa = 0; pa ^= 1u; }
                     }
@@ -261,10 +280,17 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         if (++st == AST) { st = 0; ph ^= 1u; }
                     }
                 }
+            } else if constexpr (WOP) {
+                forward_w();
             }
         }
     } else if (warp < kFatFirstEpilogueWarp) {
         regs_give<kFatRegsWiden>();
+        if constexpr (WOP && !kPackedA) {
+            // the weight operand comes by TMA and the activation codes are bytes: nothing to widen; the
+            // first of these warps forwards "weight rows landed", as warp 2 does for the activation rows
+            if (warp == kFatFirstWWarp) forward_w();
+        } else {
         // ------------------------------------------------------------ widen weight codes -> shared memory
         const uint32_t grp = (uint32_t)(warp - kFatFirstWWarp) >> 2;
         const int u = (threadIdx.x - kFatFirstWWarp * 32) & 127;  // thread of its group of four warps
@@ -326,8 +352,9 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(awst), 0));
                 }
-                const uint32_t pst = jj % kSsWPackedStages, pph = (jj / kSsWPackedStages) & 1u;
-                const uint32_t wst = jj % kSsStages, wph = (jj / kSsStages) & 1u;
+                if constexpr (!WOP) {
+                const uint32_t pst = jj % WPB, pph = (jj / WPB) & 1u;
+                const uint32_t wst = jj % WST, wph = (jj / WST) & 1u;
                 if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
                 const uint32_t pw = sbase + S::kWPackedOff + pst * S::kWPacked;
                 const uint32_t wdW = sbase + S::kWOff + wst * S::kW;
@@ -359,7 +386,9 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(wst), 0));
+                }
             }
+        }
         }
     } else {
         regs_take<kFatRegsEpilogue>();
@@ -649,25 +678,26 @@ static bool fat_kernel_registers_fit(Kern kern) {
     return kFatRegsTotal <= kFatThreads * fa.numRegs && fa.numRegs >= kFatRegsWiden && fa.numRegs <= kFatRegsEpilogue;
 }
 
-template <int MODE, int ABITS>
-static dvdq_status launch_qgemm_fat_t(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+template <int MODE, int ABITS, bool WOP>
+static dvdq_status launch_qgemm_fat_w(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                       const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, const FusedOut& fo,
                                       cudaStream_t st) {
-    using S = SsSmem<ABITS>;
+    using S = SsSmem<ABITS, WOP>;
     const int64_t K = w.K, N = w.N;
     const BlobLayout L = blob_layout(N, K);
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
     CUtensorMap tmA, tmAhi, tmW, tmY;
     if (!make_act_maps<ABITS>(codes, M, K, &tmA, &tmAhi)) return DVDQ_ERR_CUDA;
-    if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, S::BNh,
-                       CU_TENSOR_MAP_SWIZZLE_NONE))
+    if (WOP ? !make_byte_map(&tmW, w.operand, (uint64_t)K, (uint64_t)N, (uint64_t)K, kBK, S::BNh, CU_TENSOR_MAP_SWIZZLE_128B)
+            : !make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, S::BNh,
+                             CU_TENSOR_MAP_SWIZZLE_NONE))
         return DVDQ_ERR_CUDA;
     if (MODE == kFatFuse) {
         tmY = tmA;  // unused: the fused epilogue stores codes, scales and sums itself
     } else if (!make_out_map32(&tmY, Y, (uint64_t)N, (uint64_t)M, (uint64_t)ldy)) {
         return DVDQ_ERR_CUDA;
     }
-    auto kern = qgemm_fat_kernel<MODE, ABITS>;
+    auto kern = qgemm_fat_kernel<MODE, ABITS, WOP>;
     if (!fat_kernel_registers_fit(kern)) return DVDQ_ERR_CUDA;
     static PerDevice<int> cache;
     const int max_pairs = resident_pairs(cache, kern, kFatThreads, S::kTotal);
@@ -678,6 +708,14 @@ static dvdq_status launch_qgemm_fat_t(const void* codes, const float* scales, co
                                                     reinterpret_cast<const int32_t*>(blob + L.zc_offset),
                                                     static_cast<const __nv_bfloat16*>(bias), (int)M, (int)N, (int)K, act, spr, fo);
     return cuda_status(cudaGetLastError());
+}
+
+template <int MODE, int ABITS>
+static dvdq_status launch_qgemm_fat_t(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+                                      const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy, const FusedOut& fo,
+                                      cudaStream_t st) {
+    return w.operand != nullptr ? launch_qgemm_fat_w<MODE, ABITS, true>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, fo, st)
+                                : launch_qgemm_fat_w<MODE, ABITS, false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, fo, st);
 }
 
 // Block-wise activation scales, bf16 output; sb = bits a code is stored in (4, 6 or 8).

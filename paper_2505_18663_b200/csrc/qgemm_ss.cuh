@@ -50,11 +50,16 @@ constexpr int kSsAWarps = 8;
 // 4 / 6: packed; TMA fills a ring of packed tiles and warps widen them into the operand stages, as
 // for the weights (a 4-bit code masked into the high half of a byte is 16 x code, a 6-bit code
 // moved to the top of a byte 4 x code; the factor is shifted out of the accumulator).
-template <int ABITS>
+// WOP: the weight operand exists in global memory already (one int8 per code, in the operand's K
+// order): TMA writes the weight stages too and no warp widens weights.
+template <int ABITS, bool WOP = false>
 struct SsSmem {
     static constexpr int BN = kSsBN, BNh = BN / 2;
     static constexpr bool kPackedA = ABITS != 8;
     static constexpr int kAStages = kPackedA ? kSsStages : kSsAStages;  // operand stages of the activation tile
+    static constexpr int kWStages = WOP ? kSsAStages : kSsStages;       // operand stages of the weight half-tile
+    static constexpr int kWPackedStages = WOP ? 0 : kSsWPackedStages;   // ring of packed weight half-tiles
+    static constexpr int kWpBars = WOP ? kWStages : kSsWPackedStages;   // "this CTA's TMA copy of weight rows has landed"
     static constexpr int kA = kBM * kBK;              // activation tile of one k-block (int8, swizzled)
     static constexpr int kW = BNh * kBK;              // widened weight half-tile
     static constexpr int kWPacked = BNh * kBK / 2;    // packed weight half-tile (64-byte rows)
@@ -64,8 +69,8 @@ struct SsSmem {
     static constexpr int kAPackedStages = !kPackedA ? 0 : (ABITS == 6 ? 3 : 4);  // what fits
     static constexpr int kAOff = 0;
     static constexpr int kWOff = kAOff + kAStages * kA;
-    static constexpr int kWPackedOff = kWOff + kSsStages * kW;
-    static constexpr int kAPackedOff = kWPackedOff + kSsWPackedStages * kWPacked;
+    static constexpr int kWPackedOff = kWOff + kWStages * kW;
+    static constexpr int kAPackedOff = kWPackedOff + kWPackedStages * kWPacked;
     static constexpr int kStageOutOff = kAPackedOff + kAPackedStages * kAPacked;  // 1024-byte aligned
     // 16 KB of staging and 12 KB of constants whether four or eight epilogue warps share them: one
     // buffer of 32 rows x 64 (or 32) bf16 each, and delta / zero-point rest / bias of 256 (or 128) columns
@@ -73,7 +78,8 @@ struct SsSmem {
     static constexpr int kConstOff = kStageOutOff + kStageOutBytes;
     static constexpr int kConstBytes = 4 * 3 * BN * 4;
     static constexpr int kBarOff = kConstOff + kConstBytes;
-    static constexpr int kNumBars = 3 * kAStages + 2 * kSsStages + 5 + 2 * kSsWPackedStages + 2 * kAPackedStages;
+    static constexpr int kNumBars = 3 * kAStages + 2 * kWStages + 5 + 2 * kWpBars + 2 * kAPackedStages;
+    static_assert(kWStages % 2 == 0, "the MMA warp takes the weight stages in pairs");
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kTotal = kMiscOff + 16 + 1024;
     static_assert(kStageOutOff % 1024 == 0, "swizzled tiles need 1024-byte alignment");
@@ -94,17 +100,17 @@ __device__ __forceinline__ void tc_mma_i8_ss_pair(uint32_t d_tmem, uint64_t a_de
 template <int ABITS>
 constexpr int ss_warps(int ew) { return ew == 8 ? kSsFirstEpilogueWarp2 + 4 : (ABITS != 8 ? kSsFirstAWarp + kSsAWarps : kSsFirstEpilogueWarp2); }
 
-template <int ABITS, bool RAW, int EW>
+template <int ABITS, bool RAW, int EW, bool WOP>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(ss_warps<ABITS>(EW) * 32, 1)
 qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmAhi, const __grid_constant__ CUtensorMap tmW,
                 const __grid_constant__ CUtensorMap tmY, const float* __restrict__ scales,
                 const int32_t* __restrict__ sums, const float* __restrict__ delta, const int32_t* __restrict__ zc,
                 const __nv_bfloat16* __restrict__ bias, int32_t* __restrict__ acc_out, int64_t ldacc,
                 int M, int N, int K, int act, int spr) {
-    using S = SsSmem<ABITS>;
+    using S = SsSmem<ABITS, WOP>;
     constexpr int BN = S::BN, BNh = S::BNh;
     constexpr bool kPackedA = S::kPackedA;
-    constexpr int AST = S::kAStages, APS = S::kAPackedStages;
+    constexpr int AST = S::kAStages, APS = S::kAPackedStages, WST = S::kWStages, WPB = S::kWpBars;
     // packed codes with the second set of epilogue warps (layers whose epilogue sets the pace): the
     // eight weight warps widen both operands of their k-block instead of eight more warps
     constexpr bool kWidenBoth = kPackedA && EW == 8;
@@ -125,14 +131,14 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     auto a_empty = [&](int s) { return bar0 + 8u * (2 * AST + s); };             // one per CTA
     const uint32_t barw = bar0 + 8u * (3 * AST);
     auto ops_full = [&](int s) { return barw + 8u * s; };                        // widened weights; leader's copy is used
-    auto ops_empty = [&](int s) { return barw + 8u * (kSsStages + s); };         // one per CTA
-    auto acc_full = [&](int s) { return barw + 8u * (2 * kSsStages + s); };      // one per CTA
-    auto acc_empty = [&](int s) { return barw + 8u * (2 * kSsStages + 2 + s); }; // leader's copy
-    const uint32_t drain_bar = barw + 8u * (2 * kSsStages + 4);
-    auto wp_full = [&](int s) { return drain_bar + 8u * (1 + s); };
-    auto wp_empty = [&](int s) { return drain_bar + 8u * (1 + kSsWPackedStages + s); };
-    auto apk_full = [&](int s) { return drain_bar + 8u * (1 + 2 * kSsWPackedStages + s); };        // packed activation tiles (TMA)
-    auto apk_empty = [&](int s) { return drain_bar + 8u * (1 + 2 * kSsWPackedStages + APS + s); };
+    auto ops_empty = [&](int s) { return barw + 8u * (WST + s); };         // one per CTA
+    auto acc_full = [&](int s) { return barw + 8u * (2 * WST + s); };      // one per CTA
+    auto acc_empty = [&](int s) { return barw + 8u * (2 * WST + 2 + s); }; // leader's copy
+    const uint32_t drain_bar = barw + 8u * (2 * WST + 4);
+    auto wp_full = [&](int s) { return drain_bar + 8u * (1 + s); };        // this CTA's TMA copy of weight rows (packed ring, or the stage itself)
+    auto wp_empty = [&](int s) { return drain_bar + 8u * (1 + WPB + s); };
+    auto apk_full = [&](int s) { return drain_bar + 8u * (1 + 2 * WPB + s); };        // packed activation tiles (TMA)
+    auto apk_empty = [&](int s) { return drain_bar + 8u * (1 + 2 * WPB + APS + s); };
     volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + S::kMiscOff);  // [0] tmem base, [1] abort
     volatile uint32_t* abort_flag = misc + 1;
 
@@ -143,10 +149,10 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             mbar_init(a_empty(s), 1);
         }
         for (int s = 0; s < APS; ++s) { mbar_init(apk_full(s), 1); mbar_init(apk_empty(s), kSsAWarps / kUnpackGroups); }
-        for (int s = 0; s < kSsStages; ++s) { mbar_init(ops_full(s), 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
+        for (int s = 0; s < WST; ++s) { mbar_init(ops_full(s), WOP ? 2 : 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * EW); }
         mbar_init(drain_bar, 1);
-        for (int s = 0; s < kSsWPackedStages; ++s) { mbar_init(wp_full(s), 1); mbar_init(wp_empty(s), kSsWWarps / kUnpackGroups); }
+        for (int s = 0; s < WPB; ++s) { mbar_init(wp_full(s), 1); mbar_init(wp_empty(s), kSsWWarps / kUnpackGroups); }
         misc[1] = 0u;
         fence_mbar_init();
     }
@@ -160,6 +166,19 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = misc[0];
 
+    // WOP: "this CTA's weight rows of a stage have landed" -> leader (a TMA copy completes on a barrier of its own CTA)
+    auto forward_w = [&]() {
+        uint32_t st = 0, ph = 0;
+        bool ok = true;
+        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+            for (int kb = 0; kb < KB; ++kb) {
+                if (!mbar_wait_warp(wp_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(st), 0));
+                __syncwarp();
+                if (++st == WST) { st = 0; ph ^= 1u; }
+            }
+        }
+    };
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer, activation rows
         if (lane == 0) {
@@ -208,17 +227,23 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 const int n0 = (tile % num_n) * BN + (int)rank * BNh;
                 for (int kb = 0; ok && kb < KB; ++kb) {
-                    if (!mbar_wait(wp_empty(wst), wph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
-                    mbar_arrive_expect_tx(wp_full(wst), S::kWPacked);
-                    tma_load_2d(sbase + S::kWPackedOff + wst * S::kWPacked, &tmW, wp_full(wst), kb * (kBK / 2), n0);
+                    if (WOP) {  // straight into the operand stage, which the MMA's commit frees
+                        if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                        mbar_arrive_expect_tx(wp_full(wst), S::kW);
+                        tma_load_2d(sbase + S::kWOff + wst * S::kW, &tmW, wp_full(wst), kb * kBK, n0);
+                    } else {
+                        if (!mbar_wait(wp_empty(wst), wph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
+                        mbar_arrive_expect_tx(wp_full(wst), S::kWPacked);
+                        tma_load_2d(sbase + S::kWPackedOff + wst * S::kWPacked, &tmW, wp_full(wst), kb * (kBK / 2), n0);
+                    }
                     ++wissued;
-                    if (++wst == kSsWPackedStages) { wst = 0; wph ^= 1u; }
+                    if (++wst == WPB) { wst = 0; wph ^= 1u; }
                 }
             }
             if (!ok) {
-                const uint32_t w_out = wissued < (uint32_t)kSsWPackedStages ? wissued : (uint32_t)kSsWPackedStages;
+                const uint32_t w_out = wissued < (uint32_t)WPB ? wissued : (uint32_t)WPB;
                 for (uint32_t i = 0; i < w_out; ++i) {
-                    const uint32_t s = (wst + kSsWPackedStages - 1 - i) % kSsWPackedStages;
+                    const uint32_t s = (wst + WPB - 1 - i) % WPB;
                     const uint32_t p = (s < wst) ? wph : (wph ^ 1u);
                     for (int it = 0; it < (1 << 16) && !mbar_try_wait(wp_full(s), p); ++it) {}
                 }
@@ -260,7 +285,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     }
                     __syncwarp();
                     st += 2;
-                    if (st == kSsStages) { st = 0; ph ^= 1u; }
+                    if (st == WST) { st = 0; ph ^= 1u; }
                     sa = sa1 + 1;
                     pa = pa1;
                     if (sa == AST) { sa = 0; pa ^= 1u; }
@@ -398,6 +423,10 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         if (!RAW && lane == 0) tma_store_wait_all();
         __syncwarp();
 
+    } else if (WOP && !kWidenBoth && warp < kSsFwdWarp) {
+        // the weight operand comes by TMA: these warps have no work, but for one when the forwarding
+        // warp already forwards activation rows
+        if (!kPackedA && warp == kSsFirstWWarp) forward_w();
     } else if (warp < kSsFwdWarp) {
         // ------------------------------------------------------------ widen weight codes -> shared memory
         const uint32_t grp = (uint32_t)(warp - kSsFirstWWarp) >> 2;
@@ -460,8 +489,9 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(awst), 0));
             }
-            const uint32_t pst = jj % kSsWPackedStages, pph = (jj / kSsWPackedStages) & 1u;
-            const uint32_t wst = jj % kSsStages, wph = (jj / kSsStages) & 1u;
+            if constexpr (!WOP) {
+            const uint32_t pst = jj % WPB, pph = (jj / WPB) & 1u;
+            const uint32_t wst = jj % WST, wph = (jj / WST) & 1u;
             if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
             const uint32_t pw = sbase + S::kWPackedOff + pst * S::kWPacked;
             const uint32_t wdW = sbase + S::kWOff + wst * S::kW;
@@ -495,6 +525,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(wst), 0));
             }
+            }
         }
     } else if (warp == kSsFwdWarp) {
         // ------------------------------------------------------------ "activation rows landed" -> leader
@@ -510,6 +541,8 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (++st == AST) { st = 0; ph ^= 1u; }
                 }
             }
+        } else if constexpr (WOP) {
+            forward_w();
         }
     } else if (kPackedA && EW == 4 && warp >= kSsFirstAWarp) {
         // ------------------------------------------------------------ widen activation codes -> shared memory
@@ -616,18 +649,19 @@ static bool make_act_maps(const void* codes, int64_t M, int64_t K, CUtensorMap* 
     return true;
 }
 
-template <int ABITS, bool RAW, int EW>
-static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+template <int ABITS, bool RAW, int EW, bool WOP>
+static dvdq_status launch_qgemm_ss_w(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
                                    const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
                                    int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
-    using S = SsSmem<ABITS>;
+    using S = SsSmem<ABITS, WOP>;
     const int64_t K = w.K, N = w.N;
     const BlobLayout L = blob_layout(N, K);
     const uint8_t* blob = static_cast<const uint8_t*>(w.blob);
     CUtensorMap tmA, tmAhi, tmW, tmY;
     if (!make_act_maps<ABITS>(codes, M, K, &tmA, &tmAhi)) return DVDQ_ERR_CUDA;
-    if (!make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, S::BNh,
-                       CU_TENSOR_MAP_SWIZZLE_NONE))
+    if (WOP ? !make_byte_map(&tmW, w.operand, (uint64_t)K, (uint64_t)N, (uint64_t)K, kBK, S::BNh, CU_TENSOR_MAP_SWIZZLE_128B)
+            : !make_byte_map(&tmW, blob + L.codes_offset, (uint64_t)K / 2, (uint64_t)N, (uint64_t)K / 2, kBK / 2, S::BNh,
+                             CU_TENSOR_MAP_SWIZZLE_NONE))
         return DVDQ_ERR_CUDA;
     if (RAW) {
         tmY = tmA;  // unused
@@ -636,7 +670,7 @@ static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, con
         return DVDQ_ERR_CUDA;
     }
     constexpr int kThreads = ss_warps<ABITS>(EW) * 32;
-    auto kern = qgemm_ss_kernel<ABITS, RAW, EW>;
+    auto kern = qgemm_ss_kernel<ABITS, RAW, EW, WOP>;
     static PerDevice<int> cache;
     const int max_pairs = resident_pairs(cache, kern, kThreads, S::kTotal);
     if (max_pairs == 0) return DVDQ_ERR_CUDA;
@@ -648,6 +682,19 @@ static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, con
                                                    static_cast<const __nv_bfloat16*>(bias), acc_out, ldacc, (int)M, (int)N, (int)K,
                                                    act, spr);
     return cuda_status(cudaGetLastError());
+}
+
+// The weight operand as one int8 per code, where the handle has one (dvdq_widen_weights); the int32
+// output keeps to the 4-bit codes.
+template <int ABITS, bool RAW, int EW>
+static dvdq_status launch_qgemm_ss_t(const void* codes, const float* scales, const int32_t* sums, int spr, int64_t M,
+                                     const dvdq_weights& w, const void* bias, int act, void* Y, int64_t ldy,
+                                     int32_t* acc_out, int64_t ldacc, cudaStream_t st) {
+    if constexpr (!RAW) {
+        if (w.operand != nullptr)
+            return launch_qgemm_ss_w<ABITS, RAW, EW, true>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
+    }
+    return launch_qgemm_ss_w<ABITS, RAW, EW, false>(codes, scales, sums, spr, M, w, bias, act, Y, ldy, acc_out, ldacc, st);
 }
 
 // Codes in bytes: eight epilogue warps where the epilogue would otherwise set the pace: a tile's

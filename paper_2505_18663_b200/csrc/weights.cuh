@@ -82,6 +82,23 @@ __global__ void quantize_weights_symmetric_kernel(const __nv_bfloat16* __restric
     }
 }
 
+// The packed 4-bit codes of a blob as the GEMM's weight operand: one int8 per code holding 16 x (u - 8)
+// (the nibble in the high half of the byte), in the K order in which the GEMM's warps would write
+// them into a shared-memory stage: the 32 codes of a 16-byte piece become, word by word, the four
+// even-numbered codes then the four odd-numbered ones.  A thread per piece, grid-stride.
+__global__ void widen_weights_kernel(const uint8_t* __restrict__ packed, int64_t pieces, uint8_t* __restrict__ operand) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < pieces; i += (int64_t)gridDim.x * blockDim.x) {
+        const uint4 p = __ldg(reinterpret_cast<const uint4*>(packed) + i);
+        const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+        uint32_t e[4], o[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { e[j] = (w[j] << 4) & 0xF0F0F0F0u; o[j] = w[j] & 0xF0F0F0F0u; }
+        uint4* dst = reinterpret_cast<uint4*>(operand) + 2 * i;
+        dst[0] = make_uint4(e[0], o[0], e[1], o[1]);
+        dst[1] = make_uint4(e[2], o[2], e[3], o[3]);
+    }
+}
+
 // The opt-in of a weight kernel to a whole row of fp64 in shared memory, once per device.
 template <typename Kern>
 static bool weight_kernel_setup(PerDevice<int>& cache, Kern kern) {

@@ -145,6 +145,13 @@ def test_qgemm_blockwise_on_oracle_codes_and_scales(M, N, K, Bk, bits, mode, act
     # same integer inputs: what differs is fp32 against fp64 in the combination of at most forty
     # group terms -- a few ulp of fp32, far below the bf16 rounding, so nearly every output is equal
     assert np.mean(y != y_or) < 0.02
+    # the weight operand written once (dvdq_widen_weights) instead of widened tile by tile: the same bits
+    operand = torch.empty(N * K, dtype=torch.uint8, device=DEV)
+    Y2 = torch.zeros(M, N, dtype=torch.bfloat16, device=DEV)
+    B.dvdq_qgemm(packed, torch.from_numpy(np.ascontiguousarray(s32)).to(DEV), sums, M, q, B.dvdq_widen_weights(w, operand),
+                 bias.to(DEV), act, Y2)
+    assert_device_ok()
+    assert torch.equal(Y, Y2)
     # the int32 output does not depend on the scales: bit-exact against the whole-K integer GEMM
     acc = torch.zeros(M, N, dtype=torch.int32, device=DEV)
     B.dvdq_qgemm_int32(packed, sums, M, q, w, acc)

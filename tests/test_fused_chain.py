@@ -43,6 +43,12 @@ def run_fused(q, codes, scales, sums, M, w, bias, act, N, bits_next, with_y=True
     Y = torch.zeros(M, N, dtype=torch.bfloat16, device=DEV) if with_y else None
     B.dvdq_qgemm_fused_rq(codes, scales, sums, M, q, w, bias, act, qn, cn, sn, Sn, Y)
     assert_device_ok()
+    # the weight operand written once (dvdq_widen_weights) instead of widened tile by tile: the same bits
+    operand = torch.empty(w.N * w.K, dtype=torch.uint8, device=DEV)
+    cn2, sn2, Sn2 = torch.zeros_like(cn), torch.zeros_like(sn), torch.zeros_like(Sn)
+    B.dvdq_qgemm_fused_rq(codes, scales, sums, M, q, B.dvdq_widen_weights(w, operand), bias, act, qn, cn2, sn2, Sn2, None)
+    assert_device_ok()
+    assert torch.equal(cn, cn2) and torch.equal(sn, sn2) and torch.equal(Sn, Sn2)
     return qn, cn, sn.view(M, N // G), Sn.view(M, N // G), Y
 
 

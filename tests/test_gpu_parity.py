@@ -351,10 +351,18 @@ def test_full_size_layer_on_sampled_rows(workload, layer_idx, container):
     sums = torch.empty(M, dtype=torch.int32, device=DEV)
     Y = torch.empty(M, layer.N, dtype=torch.bfloat16, device=DEV)
     bias = W.make_bias(wl, layer, device=DEV)
-    # the two launches of a layer, as the benchmark issues them
+    # the three launches of a layer, as the benchmark issues them: the transform, the weight operand
+    # written into a scratch area, the GEMM that reads it
+    scratch = torch.empty(layer.N * layer.K, dtype=torch.uint8, device=DEV)
     B.dvdq_rotate_quantize(x, q, codes, scales, sums)
-    B.dvdq_qgemm(codes, scales, sums, M, q, w, bias, layer.act, Y)
+    B.dvdq_qgemm(codes, scales, sums, M, q, B.dvdq_widen_weights(w, scratch), bias, layer.act, Y)
     assert_device_ok()
+    # the GEMM that widens the weights itself, tile by tile, gives the same bits
+    Y_tile = torch.empty_like(Y)
+    B.dvdq_qgemm(codes, scales, sums, M, q, w, bias, layer.act, Y_tile)
+    assert_device_ok()
+    assert torch.equal(Y, Y_tile)
+    del Y_tile, scratch
     rows = W.sample_rows(M, 40, tile=256, seed=layer_idx)
     xs = x[rows.to(DEV)].cpu()
     un, dn, zn = u.cpu().numpy(), d.cpu().numpy(), z.cpu().numpy()
