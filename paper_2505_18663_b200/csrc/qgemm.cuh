@@ -10,6 +10,8 @@
 //   qgemm_ss.cuh   one scale per token: activation codes one int8 each (TMA writes the operand stages)
 //                  or packed 4 / 6 bits each (widened into the stages by warps, like the weights)
 //   qgemm_fat.cuh  block-wise scales, and the epilogue that is the next layer's rotate-quantize
+// Each of them either widens the 4-bit weight codes itself, tile by tile, or (handle with an operand:
+// dvdq_widen_weights) reads them one int8 each with TMA.
 // A 4-bit two's-complement nibble masked into the HIGH half of a byte is the int8 value 16 x code, a
 // 6-bit code shifted to the top of a byte is 4 x code; the factor (16 x 16, 4 x 16 or 16 per
 // product) is an exact shift of the int32 accumulator in the epilogue.  Weights are stored as

@@ -26,7 +26,13 @@
 //               takes 128 of the 256 columns.  With one warp per quarter the epilogue, not the MMA,
 //               sets the pace of layers with a short K or a GELU (+13..25 % there); where the
 //               mainloop sets it, the extra warps only compete with the widening warps (-2..7 %).
-//   warps 16-23 (packed codes) widen activation codes into the operand stage (two groups).
+//   warps 16-23 (packed codes, EW = 4) widen activation codes into the operand stage (two groups);
+//               with EW = 8 the weight warps 6-13 widen both operands of their k-block instead.
+// WOP (the weight handle carries the codes one int8 each, dvdq_widen_weights): warp 15's TMA copies
+// go straight into a ring of six weight operand stages and no warp widens weights; one warp
+// (14 with packed codes, 6 otherwise) tells the leader that this CTA's weight rows have landed.
+// With codes in bytes no warp touches an operand at all then; with packed codes and EW = 8 warps
+// 6-13 widen the activation codes only.
 // Every wait is bounded (mbar_wait).
 #pragma once
 
