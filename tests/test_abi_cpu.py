@@ -39,6 +39,8 @@ def test_size_queries():
     n = B.dvdq_weight_blob_bytes(3072, 3072)
     assert n >= 3072 * 1536 + 8 * 3072 and n % 256 == 0
     assert B.dvdq_weight_blob_bytes(3071, 3072) == 0
+    assert B.dvdq_weight_operand_bytes(3072, 12288) == 3072 * 12288       # one int8 per code
+    assert B.dvdq_weight_operand_bytes(3071, 3072) == 0 and B.dvdq_weight_operand_bytes(3072, 100) == 0
     q = B.ActQuant(4, 1024, 0)
     ws = B.dvdq_qlinear_workspace_bytes(1000, 3072, q)
     assert ws >= 1000 * 1536 + 8000 and ws % 256 == 0
@@ -122,6 +124,21 @@ def test_validation_happens_before_any_cuda_call():
     assert lib.dvdq_quantize_weights_symmetric(one, 9, 256, 256, 64, one, C.byref(B.Weights()), None) == B.ERR_SHAPE   # N % 8
     assert lib.dvdq_quantize_weights_symmetric(one, 8, 256, 256, 64, one, None, None) == B.ERR_NULL
     assert lib.dvdq_quantize_weights_symmetric(one, 8, 256, 256, 64, C.c_void_p(64), C.byref(B.Weights()), None) == B.ERR_ALIGN
+    # the int8 weight operand: the handle is validated first, then the caller's buffer
+    wh = B.Weights(0x51445644, 1, 256, 256, 256, 0, 4096, B.dvdq_weight_blob_bytes(256, 256))
+    wo = B.Weights()
+    nk = 256 * 256
+    assert lib.dvdq_widen_weights(C.byref(wh), C.c_void_p(4096), nk, None, None) == B.ERR_NULL
+    assert lib.dvdq_widen_weights(None, C.c_void_p(4096), nk, C.byref(wo), None) == B.ERR_NULL
+    assert lib.dvdq_widen_weights(C.byref(B.Weights()), C.c_void_p(4096), nk, C.byref(wo), None) == B.ERR_BLOB
+    assert lib.dvdq_widen_weights(C.byref(wh), None, nk, C.byref(wo), None) == B.ERR_NULL
+    assert lib.dvdq_widen_weights(C.byref(wh), C.c_void_p(4096), nk - 1, C.byref(wo), None) == B.ERR_WORKSPACE
+    assert lib.dvdq_widen_weights(C.byref(wh), C.c_void_p(4096 + 16), nk, C.byref(wo), None) == B.ERR_ALIGN
+    # a handle whose operand does not fit its shape, or is misaligned, is refused by the GEMM
+    wh.operand, wh.operand_bytes = 8192, nk - 64
+    assert lib.dvdq_qgemm(one, one, one, 4, C.byref(B.ActQuant(4, 256, 0)), C.byref(wh), None, 0, one, 256, None) == B.ERR_BLOB
+    wh.operand, wh.operand_bytes = 8192 + 16, nk
+    assert lib.dvdq_qgemm(one, one, one, 4, C.byref(B.ActQuant(4, 256, 0)), C.byref(wh), None, 0, one, 256, None) == B.ERR_ALIGN
     assert lib.dvdq_int8_mma_ceiling(0, None, None) == B.ERR_SHAPE
     assert lib.dvdq_debug_wait_timeout(0, None) == B.ERR_SHAPE
 
