@@ -155,7 +155,9 @@ dvdq_status dvdq_pack_weights(const uint8_t* Wq, const float* delta, const int32
  * to those with `w`.  The blob stays the format of record (the
  * scales, zero points and 4-bit codes are still read from it); the buffer may be a scratch area
  * that is rewritten before every launch (one call per layer and step costs about 1 % of a GEMM
- * over 65536 tokens) or kept for the life of the weights (at 8 more bits per weight).  w and out
+ * over 65536 tokens) or kept for the life of the weights (at 8 more bits per weight).  A scratch
+ * area shared by several layers is safe only while the calls that write and read it are ordered
+ * (one stream, or events between streams): nothing in the library orders them.  w and out
  * may be the same object.  dvdq_qgemm_int32 always reads the 4-bit codes. */
 dvdq_status dvdq_widen_weights(const dvdq_weights* w /* host */, void* operand_out, size_t operand_bytes,
                                dvdq_weights* out /* host */, void* cuda_stream);
