@@ -31,8 +31,9 @@
 // WOP (the weight handle carries the codes one int8 each, dvdq_widen_weights): warp 15's TMA copies
 // go straight into a ring of six weight operand stages and no warp widens weights; one warp
 // (14 with packed codes, 6 otherwise) tells the leader that this CTA's weight rows have landed.
-// With codes in bytes no warp touches an operand at all then; with packed codes and EW = 8 warps
-// 6-13 widen the activation codes only.
+// With codes in bytes no warp touches an operand at all then, and one "full" / "empty" barrier per
+// stage serves both operands' rings (half the waits and commits of the MMA warp); with packed codes
+// and EW = 8 warps 6-13 widen the activation codes only.
 // Every wait is bounded (mbar_wait).
 #pragma once
 
@@ -120,6 +121,9 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     // packed codes with the second set of epilogue warps (layers whose epilogue sets the pace): the
     // eight weight warps widen both operands of their k-block instead of eight more warps
     constexpr bool kWidenBoth = kPackedA && EW == 8;
+    // both operands by TMA into rings of the same depth: one "full" and one "empty" barrier per stage serve both
+    constexpr bool kOneRing = WOP && !kPackedA;
+    static_assert(!kOneRing || S::kAStages == S::kWStages, "one ring: the operands' stages advance together");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -151,7 +155,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (threadIdx.x == 0) {
         for (int s = 0; s < AST; ++s) {
             mbar_init(a_full(s), 1);
-            mbar_init(a_ready(s), kPackedA ? 2 * (kSsAWarps / kUnpackGroups) : 2);
+            mbar_init(a_ready(s), kPackedA ? 2 * (kSsAWarps / kUnpackGroups) : kOneRing ? 4 : 2);
             mbar_init(a_empty(s), 1);
         }
         for (int s = 0; s < APS; ++s) { mbar_init(apk_full(s), 1); mbar_init(apk_empty(s), kSsAWarps / kUnpackGroups); }
@@ -179,7 +183,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
             for (int kb = 0; kb < KB; ++kb) {
                 if (!mbar_wait_warp(wp_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(st), 0));
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(kOneRing ? a_ready(st) : ops_full(st), 0));
                 __syncwarp();
                 if (++st == WST) { st = 0; ph ^= 1u; }
             }
@@ -234,7 +238,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int n0 = (tile % num_n) * BN + (int)rank * BNh;
                 for (int kb = 0; ok && kb < KB; ++kb) {
                     if (WOP) {  // straight into the operand stage, which the MMA's commit frees
-                        if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                        if (!mbar_wait(kOneRing ? a_empty(wst) : ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
                         mbar_arrive_expect_tx(wp_full(wst), S::kW);
                         tma_load_2d(sbase + S::kWOff + wst * S::kW, &tmW, wp_full(wst), kb * kBK, n0);
                     } else {
@@ -272,9 +276,9 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     // the activation ring may have an odd number of stages: its second stage of the trip can wrap
                     const uint32_t sa1 = sa + 1 == AST ? 0u : sa + 1, pa1 = sa + 1 == AST ? pa ^ 1u : pa;
                     if (!mbar_wait_warp(a_ready(sa), pa, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                    if (!mbar_wait_warp(ops_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
+                    if (!kOneRing && !mbar_wait_warp(ops_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     if (!mbar_wait_warp(a_ready(sa1), pa1, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                    if (!mbar_wait_warp(ops_full(st + 1), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
+                    if (!kOneRing && !mbar_wait_warp(ops_full(st + 1), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                     tc_fence_after();
                     if (elect_one()) {
 #pragma unroll
@@ -284,7 +288,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 #pragma unroll
                             for (int k = 0; k < kBK / 32; ++k)  // +32 int8 along K = +2 in the 16-byte address field
                                 tc_mma_i8_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (kb | h | k) != 0 ? 1u : 0u);
-                            tc_commit_pair(ops_empty(st + h), 3);
+                            if (!kOneRing) tc_commit_pair(ops_empty(st + h), 3);
                             tc_commit_pair(a_empty(h ? sa1 : sa), 3);
                         }
                         if (kb + 2 >= KB) tc_commit_pair(acc_full(a), 3);
