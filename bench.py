@@ -198,7 +198,7 @@ def config_of(wl, args):
 # layout (container_bits); None where no capture of that kernel in its present form exists.
 # (16384-token capture x 4: traffic grows with M; mean of the four launches of a step; the GEMM with
 # its weight operand written before every launch, the default)
-QGEMM_DRAM_TRAFFIC_PER_LAUNCH = {0: 1.15e9, 8: 1.53e9}
+QGEMM_DRAM_TRAFFIC_PER_LAUNCH = {0: 1.17e9, 8: 1.52e9}
 RQ_DRAM_TRAFFIC_PER_LAUNCH = {0: 0.82e9, 8: 0.94e9}
 
 
