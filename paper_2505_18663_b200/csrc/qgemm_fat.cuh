@@ -291,104 +291,104 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // first of these warps forwards "weight rows landed", as warp 2 does for the activation rows
             if (warp == kFatFirstWWarp) forward_w();
         } else {
-        // ------------------------------------------------------------ widen weight codes -> shared memory
-        const uint32_t grp = (uint32_t)(warp - kFatFirstWWarp) >> 2;
-        const int u = (threadIdx.x - kFatFirstWWarp * 32) & 127;  // thread of its group of four warps
-        uint32_t j = 0;
-        bool ok = true;
-        const uint32_t rt_zero = runtime_zero();
-        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-            for (int kb = 0; kb < KB; ++kb) {
-                const uint32_t jj = j++;
-                if (jj % kUnpackGroups != grp) continue;
-                if constexpr (kPackedA) {
-                    // this CTA's 128 token rows of the k-block first: the same job on the activation rings
-                    const uint32_t apst = jj % APS, apph = (jj / APS) & 1u;
-                    const uint32_t awst = jj % AST, awph = (jj / AST) & 1u;
-                    if (!mbar_wait(apk_full(apst), apph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                    const uint32_t pa = sbase + S::kAPackedOff + apst * S::kAPacked;
-                    const uint32_t wd = sbase + S::kAOff + awst * S::kA;
-                    constexpr int kAPieces = (kBM * 4) / 128;
-                    uint4 pl[kAPieces];
-                    uint2 ph2[kAPieces];
-                    uint32_t got = 0u;
+            // ------------------------------------------------------------ widen weight codes -> shared memory
+            const uint32_t grp = (uint32_t)(warp - kFatFirstWWarp) >> 2;
+            const int u = (threadIdx.x - kFatFirstWWarp * 32) & 127;  // thread of its group of four warps
+            uint32_t j = 0;
+            bool ok = true;
+            const uint32_t rt_zero = runtime_zero();
+            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
+                for (int kb = 0; kb < KB; ++kb) {
+                    const uint32_t jj = j++;
+                    if (jj % kUnpackGroups != grp) continue;
+                    if constexpr (kPackedA) {
+                        // this CTA's 128 token rows of the k-block first: the same job on the activation rings
+                        const uint32_t apst = jj % APS, apph = (jj / APS) & 1u;
+                        const uint32_t awst = jj % AST, awph = (jj / AST) & 1u;
+                        if (!mbar_wait(apk_full(apst), apph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                        const uint32_t pa = sbase + S::kAPackedOff + apst * S::kAPacked;
+                        const uint32_t wd = sbase + S::kAOff + awst * S::kA;
+                        constexpr int kAPieces = (kBM * 4) / 128;
+                        uint4 pl[kAPieces];
+                        uint2 ph2[kAPieces];
+                        uint32_t got = 0u;
 #pragma unroll
-                    for (int it = 0; it < kAPieces; ++it) {
-                        const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
-                        pl[it] = lds128(pa + row * (kBK / 2) + ck * 16);
-                        got ^= pl[it].w;
-                        if (ABITS == 6) {
-                            ph2[it] = lds64(pa + S::kALo + row * (kBK / 4) + ck * 8);
-                            got ^= ph2[it].y;
-                        }
-                    }
-                    got &= rt_zero;
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_after_loads(apk_empty(apst), got);
-                    if (!mbar_wait(a_empty(awst), awph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-                    tc_fence_after();
-#pragma unroll
-                    for (int it = 0; it < kAPieces; ++it) {
-                        const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
-                        const uint32_t w[4] = {pl[it].x, pl[it].y, pl[it].z, pl[it].w};
-                        uint32_t e[4], o[4];
-#pragma unroll
-                        for (int jw = 0; jw < 4; ++jw) {
-                            if (ABITS == 4) {
-                                e[jw] = (w[jw] << 4) & 0xF0F0F0F0u;
-                                o[jw] = w[jw] & 0xF0F0F0F0u;
-                            } else {
-                                const uint32_t hh = (jw >> 1) ? ph2[it].y : ph2[it].x;
-                                const int a2 = 2 * (jw & 1);
-                                e[jw] = ((w[jw] << 2) & 0x3C3C3C3Cu) | ((hh << (6 - 2 * a2)) & 0xC0C0C0C0u);
-                                o[jw] = ((w[jw] >> 2) & 0x3C3C3C3Cu) | ((hh << (4 - 2 * a2)) & 0xC0C0C0C0u);
+                        for (int it = 0; it < kAPieces; ++it) {
+                            const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                            pl[it] = lds128(pa + row * (kBK / 2) + ck * 16);
+                            got ^= pl[it].w;
+                            if (ABITS == 6) {
+                                ph2[it] = lds64(pa + S::kALo + row * (kBK / 4) + ck * 8);
+                                got ^= ph2[it].y;
                             }
                         }
-                        const uint32_t drow = wd + (row >> 3) * 1024 + (row & 7) * 128;
-                        sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[0], o[0], e[1], o[1]);
-                        sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[2], o[2], e[3], o[3]);
+                        got &= rt_zero;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_after_loads(apk_empty(apst), got);
+                        if (!mbar_wait(a_empty(awst), awph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                        tc_fence_after();
+#pragma unroll
+                        for (int it = 0; it < kAPieces; ++it) {
+                            const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                            const uint32_t w[4] = {pl[it].x, pl[it].y, pl[it].z, pl[it].w};
+                            uint32_t e[4], o[4];
+#pragma unroll
+                            for (int jw = 0; jw < 4; ++jw) {
+                                if (ABITS == 4) {
+                                    e[jw] = (w[jw] << 4) & 0xF0F0F0F0u;
+                                    o[jw] = w[jw] & 0xF0F0F0F0u;
+                                } else {
+                                    const uint32_t hh = (jw >> 1) ? ph2[it].y : ph2[it].x;
+                                    const int a2 = 2 * (jw & 1);
+                                    e[jw] = ((w[jw] << 2) & 0x3C3C3C3Cu) | ((hh << (6 - 2 * a2)) & 0xC0C0C0C0u);
+                                    o[jw] = ((w[jw] >> 2) & 0x3C3C3C3Cu) | ((hh << (4 - 2 * a2)) & 0xC0C0C0C0u);
+                                }
+                            }
+                            const uint32_t drow = wd + (row >> 3) * 1024 + (row & 7) * 128;
+                            sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[0], o[0], e[1], o[1]);
+                            sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[2], o[2], e[3], o[3]);
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(awst), 0));
                     }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(awst), 0));
-                }
-                if constexpr (!WOP) {
-                const uint32_t pst = jj % WPB, pph = (jj / WPB) & 1u;
-                const uint32_t wst = jj % WST, wph = (jj / WST) & 1u;
-                if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                const uint32_t pw = sbase + S::kWPackedOff + pst * S::kWPacked;
-                const uint32_t wdW = sbase + S::kWOff + wst * S::kW;
-                // BNh rows x 4 chunks of 32 nibbles, stored as (u - 8): the packed rows go into registers
-                // before the operand stage is known to be free, and are widened on their way out
-                constexpr int kPieces = (BNh * 4) / 128;
-                uint4 p[kPieces];
-                uint32_t loaded = 0u;
+                    if constexpr (!WOP) {
+                        const uint32_t pst = jj % WPB, pph = (jj / WPB) & 1u;
+                        const uint32_t wst = jj % WST, wph = (jj / WST) & 1u;
+                        if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                        const uint32_t pw = sbase + S::kWPackedOff + pst * S::kWPacked;
+                        const uint32_t wdW = sbase + S::kWOff + wst * S::kW;
+                        // BNh rows x 4 chunks of 32 nibbles, stored as (u - 8): the packed rows go into registers
+                        // before the operand stage is known to be free, and are widened on their way out
+                        constexpr int kPieces = (BNh * 4) / 128;
+                        uint4 p[kPieces];
+                        uint32_t loaded = 0u;
 #pragma unroll
-                for (int it = 0; it < kPieces; ++it) {
-                    const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
-                    p[it] = lds128(pw + row * (kBK / 2) + ck * 16);
-                    loaded ^= p[it].w;
-                }
-                loaded &= rt_zero;
-                __syncwarp();
-                if (lane == 0) mbar_arrive_after_loads(wp_empty(pst), loaded);  // the packed rows are in registers
-                if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-                tc_fence_after();
+                        for (int it = 0; it < kPieces; ++it) {
+                            const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                            p[it] = lds128(pw + row * (kBK / 2) + ck * 16);
+                            loaded ^= p[it].w;
+                        }
+                        loaded &= rt_zero;
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_after_loads(wp_empty(pst), loaded);  // the packed rows are in registers
+                        if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                        tc_fence_after();
 #pragma unroll
-                for (int it = 0; it < kPieces; ++it) {
-                    const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
-                    const uint32_t drow = wdW + (row >> 3) * 1024 + (row & 7) * 128;
-                    sts128(drow + (((2 * ck) ^ (row & 7)) << 4), (p[it].x << 4) & 0xF0F0F0F0u, p[it].x & 0xF0F0F0F0u,
-                           (p[it].y << 4) & 0xF0F0F0F0u, p[it].y & 0xF0F0F0F0u);
-                    sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), (p[it].z << 4) & 0xF0F0F0F0u, p[it].z & 0xF0F0F0F0u,
-                           (p[it].w << 4) & 0xF0F0F0F0u, p[it].w & 0xF0F0F0F0u);
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(wst), 0));
+                        for (int it = 0; it < kPieces; ++it) {
+                            const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                            const uint32_t drow = wdW + (row >> 3) * 1024 + (row & 7) * 128;
+                            sts128(drow + (((2 * ck) ^ (row & 7)) << 4), (p[it].x << 4) & 0xF0F0F0F0u, p[it].x & 0xF0F0F0F0u,
+                                   (p[it].y << 4) & 0xF0F0F0F0u, p[it].y & 0xF0F0F0F0u);
+                            sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), (p[it].z << 4) & 0xF0F0F0F0u, p[it].z & 0xF0F0F0F0u,
+                                   (p[it].w << 4) & 0xF0F0F0F0u, p[it].w & 0xF0F0F0F0u);
+                        }
+                        fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(wst), 0));
+                    }
                 }
             }
-        }
         }
     } else {
         regs_take<kFatRegsEpilogue>();

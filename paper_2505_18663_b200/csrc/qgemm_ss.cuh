@@ -500,40 +500,40 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(awst), 0));
             }
             if constexpr (!WOP) {
-            const uint32_t pst = jj % WPB, pph = (jj / WPB) & 1u;
-            const uint32_t wst = jj % WST, wph = (jj / WST) & 1u;
-            if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-            const uint32_t pw = sbase + S::kWPackedOff + pst * S::kWPacked;
-            const uint32_t wdW = sbase + S::kWOff + wst * S::kW;
-            // BNh rows x 4 chunks of 32 nibbles, stored as (u - 8); widened in registers before the
-            // wide stage is known to be free
-            constexpr int kPieces = (BNh * 4) / 128;
-            uint32_t e[kPieces][4], o[kPieces][4];
-            uint32_t loaded = 0u;
+                const uint32_t pst = jj % WPB, pph = (jj / WPB) & 1u;
+                const uint32_t wst = jj % WST, wph = (jj / WST) & 1u;
+                if (!mbar_wait(wp_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                const uint32_t pw = sbase + S::kWPackedOff + pst * S::kWPacked;
+                const uint32_t wdW = sbase + S::kWOff + wst * S::kW;
+                // BNh rows x 4 chunks of 32 nibbles, stored as (u - 8); widened in registers before the
+                // wide stage is known to be free
+                constexpr int kPieces = (BNh * 4) / 128;
+                uint32_t e[kPieces][4], o[kPieces][4];
+                uint32_t loaded = 0u;
 #pragma unroll
-            for (int it = 0; it < kPieces; ++it) {
-                const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
-                const uint4 p = lds128(pw + row * (kBK / 2) + ck * 16);
-                const uint32_t w[4] = {p.x, p.y, p.z, p.w};
-                loaded ^= p.w;
+                for (int it = 0; it < kPieces; ++it) {
+                    const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                    const uint4 p = lds128(pw + row * (kBK / 2) + ck * 16);
+                    const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+                    loaded ^= p.w;
 #pragma unroll
-                for (int jw = 0; jw < 4; ++jw) { e[it][jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[it][jw] = w[jw] & 0xF0F0F0F0u; }
-            }
-            loaded &= rt_zero;
-            __syncwarp();
-            if (lane == 0) mbar_arrive_after_loads(wp_empty(pst), loaded);  // the packed rows are in registers
-            if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-            tc_fence_after();
+                    for (int jw = 0; jw < 4; ++jw) { e[it][jw] = (w[jw] << 4) & 0xF0F0F0F0u; o[it][jw] = w[jw] & 0xF0F0F0F0u; }
+                }
+                loaded &= rt_zero;
+                __syncwarp();
+                if (lane == 0) mbar_arrive_after_loads(wp_empty(pst), loaded);  // the packed rows are in registers
+                if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                tc_fence_after();
 #pragma unroll
-            for (int it = 0; it < kPieces; ++it) {
-                const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
-                const uint32_t drow = wdW + (row >> 3) * 1024 + (row & 7) * 128;
-                sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[it][0], o[it][0], e[it][1], o[it][1]);
-                sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[it][2], o[it][2], e[it][3], o[it][3]);
-            }
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(wst), 0));
+                for (int it = 0; it < kPieces; ++it) {
+                    const int qi = it * 128 + u, row = qi >> 2, ck = qi & 3;
+                    const uint32_t drow = wdW + (row >> 3) * 1024 + (row & 7) * 128;
+                    sts128(drow + (((2 * ck) ^ (row & 7)) << 4), e[it][0], o[it][0], e[it][1], o[it][1]);
+                    sts128(drow + (((2 * ck + 1) ^ (row & 7)) << 4), e[it][2], o[it][2], e[it][3], o[it][3]);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(wst), 0));
             }
             }
         }
