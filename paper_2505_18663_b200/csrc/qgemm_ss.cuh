@@ -20,8 +20,10 @@
 //   warps 2-5   epilogue (tcgen05.ld, zero-point term, scales, bias, GELU, bf16, TMA stores), one
 //               warp per tensor-memory lane quarter.
 //   warps 6-13  widen weight codes into the operand stage (two groups, alternate k-blocks).
-//   warp 14     (codes in bytes) tells the leader that this CTA's activation rows of a stage have
-//               landed (a TMA copy completes on a barrier of its own CTA).
+//   warp 14     idle but for one case (below): the TMA copies of activation rows of BOTH CTAs of a
+//               pair count their bytes on the leader's barrier of the stage (cp.async.bulk.tensor with
+//               .cta_group::2), which the leader's producer arms for both, so nobody has to tell the
+//               leader that the peer's rows have landed (+2-3 % over a forwarding warp).
 //   warps 16-19 (codes in bytes, EW = 8 only) a second epilogue warp per lane quarter; each then
 //               takes 128 of the 256 columns.  With one warp per quarter the epilogue, not the MMA,
 //               sets the pace of layers with a short K or a GELU (+13..25 % there); where the
@@ -29,8 +31,9 @@
 //   warps 16-23 (packed codes, EW = 4) widen activation codes into the operand stage (two groups);
 //               with EW = 8 the weight warps 6-13 widen both operands of their k-block instead.
 // WOP (the weight handle carries the codes one int8 each, dvdq_widen_weights): warp 15's TMA copies
-// go straight into a ring of six weight operand stages and no warp widens weights; one warp
-// (14 with packed codes, 6 otherwise) tells the leader that this CTA's weight rows have landed.
+// go straight into a ring of six weight operand stages and no warp widens weights; with codes in
+// bytes they are counted on the leader's barrier like the activation rows, with packed codes on a
+// barrier of their own CTA, and warp 14 tells the leader.
 // With codes in bytes no warp touches an operand at all then, and one "full" / "empty" barrier per
 // stage serves both operands' rings (half the waits and commits of the MMA warp); with packed codes
 // and EW = 8 warps 6-13 widen the activation codes only.
@@ -155,7 +158,9 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     if (threadIdx.x == 0) {
         for (int s = 0; s < AST; ++s) {
             mbar_init(a_full(s), 1);
-            mbar_init(a_ready(s), kPackedA ? 2 * (kSsAWarps / kUnpackGroups) : kOneRing ? 4 : 2);
+            // packed codes: the widening warps of both CTAs; codes in bytes: the leader's producer arms it for the
+            // TMA copies of both CTAs (in the one-ring mode its weight producer as well)
+            mbar_init(a_ready(s), kPackedA ? 2 * (kSsAWarps / kUnpackGroups) : kOneRing ? 2 : 1);
             mbar_init(a_empty(s), 1);
         }
         for (int s = 0; s < APS; ++s) { mbar_init(apk_full(s), 1); mbar_init(apk_empty(s), kSsAWarps / kUnpackGroups); }
@@ -176,19 +181,6 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     tc_fence_after();
     const uint32_t tmem_base = misc[0];
 
-    // WOP: "this CTA's weight rows of a stage have landed" -> leader (a TMA copy completes on a barrier of its own CTA)
-    auto forward_w = [&]() {
-        uint32_t st = 0, ph = 0;
-        bool ok = true;
-        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-            for (int kb = 0; kb < KB; ++kb) {
-                if (!mbar_wait_warp(wp_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                if (lane == 0) mbar_arrive_cluster(map_to_cta(kOneRing ? a_ready(st) : ops_full(st), 0));
-                __syncwarp();
-                if (++st == WST) { st = 0; ph ^= 1u; }
-            }
-        }
-    };
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer, activation rows
         if (lane == 0) {
@@ -205,6 +197,14 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
                 for (int kb = 0; ok && kb < KB; ++kb) {
                     if (!mbar_wait(ring_empty(st), ph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                    if (!kPackedA) {
+                        // both CTAs' copies count their bytes on the leader's "full" barrier of the stage
+                        if (rank == 0) mbar_arrive_expect_tx(a_ready(st), 2 * S::kA);
+                        tma_load_2d_pair(sbase + S::kAOff + st * S::kA, &tmA, map_to_cta(a_ready(st), 0), kb * kBK, m0);
+                        ++issued;
+                        if (++st == kRing) { st = 0; ph ^= 1u; }
+                        continue;
+                    }
                     mbar_arrive_expect_tx(ring_full(st), kBytes);
                     if (kPackedA) {
                         const uint32_t dst = sbase + S::kAPackedOff + st * S::kAPacked;
@@ -217,7 +217,11 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (++st == kRing) { st = 0; ph ^= 1u; }
                 }
             }
-            if (!ok) {
+            if (!ok && !kPackedA) {
+                // Giving up (some wait ran out after seconds): copies issued before that have long landed;
+                // a short bounded pause covers the last ones, whose barrier is not this CTA's to poll.
+                for (int it = 0; it < 64; ++it) __nanosleep(1000);
+            } else if (!ok) {
                 // Giving up: let copies already in flight land before the CTA exits (bounded).
                 const uint32_t n_out = issued < (uint32_t)kRing ? issued : (uint32_t)kRing;
                 for (uint32_t i = 0; i < n_out; ++i) {
@@ -237,8 +241,15 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 const int n0 = (tile % num_n) * BN + (int)rank * BNh;
                 for (int kb = 0; ok && kb < KB; ++kb) {
-                    if (WOP) {  // straight into the operand stage, which the MMA's commit frees
-                        if (!mbar_wait(kOneRing ? a_empty(wst) : ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                    if (kOneRing) {
+                        // straight into the operand stage, counted on the leader's "full" barrier like the activation rows
+                        if (!mbar_wait(a_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                        if (rank == 0) mbar_arrive_expect_tx(a_ready(wst), 2 * S::kW);
+                        tma_load_2d_pair(sbase + S::kWOff + wst * S::kW, &tmW, map_to_cta(a_ready(wst), 0), kb * kBK, n0);
+                    } else if (WOP) {
+                        // (packed activation codes) into the operand stage on a barrier of this CTA; warp 14
+                        // tells the leader: the pair form measured 0.5-1 % slower here
+                        if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
                         mbar_arrive_expect_tx(wp_full(wst), S::kW);
                         tma_load_2d(sbase + S::kWOff + wst * S::kW, &tmW, wp_full(wst), kb * kBK, n0);
                     } else {
@@ -250,7 +261,9 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (++wst == WPB) { wst = 0; wph ^= 1u; }
                 }
             }
-            if (!ok) {
+            if (!ok && kOneRing) {
+                for (int it = 0; it < 64; ++it) __nanosleep(1000);
+            } else if (!ok) {
                 const uint32_t w_out = wissued < (uint32_t)WPB ? wissued : (uint32_t)WPB;
                 for (uint32_t i = 0; i < w_out; ++i) {
                     const uint32_t s = (wst + WPB - 1 - i) % WPB;
@@ -434,9 +447,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         __syncwarp();
 
     } else if (WOP && !kWidenBoth && warp < kSsFwdWarp) {
-        // the weight operand comes by TMA: these warps have no work, but for one when the forwarding
-        // warp already forwards activation rows
-        if (!kPackedA && warp == kSsFirstWWarp) forward_w();
+        // the weight operand comes by TMA: these warps have no work
     } else if (warp < kSsFwdWarp) {
         // ------------------------------------------------------------ widen weight codes -> shared memory
         const uint32_t grp = (uint32_t)(warp - kSsFirstWWarp) >> 2;
@@ -538,21 +549,19 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
         }
     } else if (warp == kSsFwdWarp) {
-        // ------------------------------------------------------------ "activation rows landed" -> leader
-        // (codes in bytes only: a TMA copy completes on a barrier of its own CTA; widening warps arrive on the leader's themselves)
-        if constexpr (!kPackedA) {
+        // ------------------------------------------------------------ "weight rows landed" -> leader
+        // (packed activation codes with the weight operand by TMA only)
+        if constexpr (WOP && kPackedA) {
             uint32_t st = 0, ph = 0;
             bool ok = true;
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_wait_warp(a_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                    if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(st), 0));
+                    if (!mbar_wait_warp(wp_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
+                    if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(st), 0));
                     __syncwarp();
-                    if (++st == AST) { st = 0; ph ^= 1u; }
+                    if (++st == WST) { st = 0; ph ^= 1u; }
                 }
             }
-        } else if constexpr (WOP) {
-            forward_w();
         }
     } else if (kPackedA && EW == 4 && warp >= kSsFirstAWarp) {
         // ------------------------------------------------------------ widen activation codes -> shared memory
