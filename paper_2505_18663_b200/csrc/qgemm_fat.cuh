@@ -13,8 +13,8 @@
 // warps, one row and 128 columns per thread, with the register file re-divided between the roles
 // (setmaxnreg: the loaders and the widening warps give registers up, the epilogue warps take them).
 // Roles are aligned to groups of four warps, as that instruction requires:
-//   warps 0-3    TMA producer of activation tiles | MMA issuer (leader CTA) | "rows landed"
-//                forwarder | TMA producer of packed weight rows
+//   warps 0-3    TMA producer of activation tiles | MMA issuer (leader CTA) | "weight rows landed"
+//                forwarder (one mode only) | TMA producer of weight rows
 //   warps 4-11   widen weight codes into the operand stages (two groups, alternate k-blocks)
 //   warps 12-19  epilogue: warp w reads tensor-memory lanes 32 * (w % 4).., columns 128 * ((w - 12) / 4)..
 // Every wait is bounded, as in qgemm.cuh.
@@ -71,6 +71,10 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     constexpr int BN = S::BN, BNh = S::BNh;
     constexpr bool kPackedA = S::kPackedA;  // packed activation codes: the widening warps widen both operands
     constexpr int AST = S::kAStages, APS = S::kAPackedStages, WST = S::kWStages, WPB = S::kWpBars;
+    // both operands by TMA into rings of the same depth: one "full" and one "empty" barrier per stage
+    // serve both, and the copies of both CTAs count their bytes on the leader's (see qgemm_ss.cuh)
+    constexpr bool kOneRing = WOP && !kPackedA;
+    static_assert(!kOneRing || S::kAStages == S::kWStages, "one ring: the operands' stages advance together");
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
@@ -104,7 +108,7 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int s = 0; s < AST; ++s) {
             mbar_init(a_full(s), 1);
-            mbar_init(a_ready(s), kPackedA ? 2 * (kSsWWarps / kUnpackGroups) : 2);
+            mbar_init(a_ready(s), kPackedA ? 2 * (kSsWWarps / kUnpackGroups) : kOneRing ? 2 : 1);
             mbar_init(a_empty(s), 1);
         }
         for (int s = 0; s < APS; ++s) { mbar_init(apk_full(s), 1); mbar_init(apk_empty(s), kSsWWarps / kUnpackGroups); }
@@ -155,6 +159,14 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     const int m0 = (tile / num_n) * (2 * kBM) + (int)rank * kBM;
                     for (int kb = 0; ok && kb < KB; ++kb) {
                         if (!mbar_wait(ring_empty(st), ph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                        if (!kPackedA) {
+                            // both CTAs' copies count their bytes on the leader's "full" barrier of the stage
+                            if (rank == 0) mbar_arrive_expect_tx(a_ready(st), 2 * S::kA);
+                            tma_load_2d_pair(sbase + S::kAOff + st * S::kA, &tmA, map_to_cta(a_ready(st), 0), kb * kBK, m0);
+                            ++issued;
+                            if (++st == kRing) { st = 0; ph ^= 1u; }
+                            continue;
+                        }
                         mbar_arrive_expect_tx(ring_full(st), kBytes);
                         if (kPackedA) {
                             const uint32_t dst = sbase + S::kAPackedOff + st * S::kAPacked;
@@ -167,7 +179,11 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         if (++st == kRing) { st = 0; ph ^= 1u; }
                     }
                 }
-                if (!ok) {  // giving up: let copies already in flight land before the CTA exits (bounded)
+                if (!ok && !kPackedA) {
+                    // giving up (some wait ran out after seconds): copies issued before that have long landed;
+                    // a short bounded pause covers the last ones, whose barrier is not this CTA's to poll
+                    for (int it = 0; it < 64; ++it) __nanosleep(1000);
+                } else if (!ok) {  // giving up: let copies already in flight land before the CTA exits (bounded)
                     const uint32_t n_out = issued < (uint32_t)kRing ? issued : (uint32_t)kRing;
                     for (uint32_t i = 0; i < n_out; ++i) {
                         const uint32_t s = (st + kRing - 1 - i) % kRing;
@@ -186,7 +202,11 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                     const int n0 = (tile % num_n) * BN + (int)rank * BNh;
                     for (int kb = 0; ok && kb < KB; ++kb) {
-                        if (WOP) {  // straight into the operand stage, which the MMA's commit frees
+                        if (kOneRing) {  // as the activation rows: bytes counted on the leader's "full" barrier
+                            if (!mbar_wait(a_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                            if (rank == 0) mbar_arrive_expect_tx(a_ready(wst), 2 * S::kW);
+                            tma_load_2d_pair(sbase + S::kWOff + wst * S::kW, &tmW, map_to_cta(a_ready(wst), 0), kb * kBK, n0);
+                        } else if (WOP) {  // straight into the operand stage, which the MMA's commit frees
                             if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
                             mbar_arrive_expect_tx(wp_full(wst), S::kW);
                             tma_load_2d(sbase + S::kWOff + wst * S::kW, &tmW, wp_full(wst), kb * kBK, n0);
@@ -199,7 +219,9 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         if (++wst == WPB) { wst = 0; wph ^= 1u; }
                     }
                 }
-                if (!ok) {
+                if (!ok && kOneRing) {
+                    for (int it = 0; it < 64; ++it) __nanosleep(1000);
+                } else if (!ok) {
                     const uint32_t w_out = wissued < (uint32_t)WPB ? wissued : (uint32_t)WPB;
                     for (uint32_t i = 0; i < w_out; ++i) {
                         const uint32_t s = (wst + WPB - 1 - i) % WPB;
@@ -234,10 +256,10 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         if (last) kin = 0;
                         const uint32_t sa1 = sa + 1 == AST ? 0u : sa + 1, pa1 = sa + 1 == AST ? pa ^ 1u : pa;
                         if (!mbar_wait_warp(a_ready(sa), pa, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                        if (!mbar_wait_warp(ops_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
+                        if (!kOneRing && !mbar_wait_warp(ops_full(st), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                         if (step == 2) {
                             if (!mbar_wait_warp(a_ready(sa1), pa1, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                            if (!mbar_wait_warp(ops_full(st + 1), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
+                            if (!kOneRing && !mbar_wait_warp(ops_full(st + 1), ph, abort_flag, kWaitWideFull)) { ok = false; break; }
                         }
                         tc_fence_after();
                         if (elect_one()) {
@@ -249,7 +271,7 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                                 for (int k = 0; k < kBK / 32; ++k)
                                     tc_mma_i8_ss_pair(d_tmem, adesc + 2u * k, bdesc + 2u * k, idesc, (first && h == 0 && k == 0) ? 0u : 1u);
-                                tc_commit_pair(ops_empty(st + h), 3);
+                                if (!kOneRing) tc_commit_pair(ops_empty(st + h), 3);
                                 tc_commit_pair(a_empty(sah), 3);
                             }
                             if (last) tc_commit_pair(acc_full(acc), 3);
@@ -267,29 +289,15 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
             __syncwarp();
         } else {
-            // ------------------------------------------------------------ "activation rows landed" -> leader
-            // (codes in bytes only; packed codes are widened by warps that arrive on the leader's barrier themselves)
-            if constexpr (!kPackedA) {
-                uint32_t st = 0, ph = 0;
-                bool ok = true;
-                for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-                    for (int kb = 0; kb < KB; ++kb) {
-                        if (!mbar_wait_warp(a_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                        if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ready(st), 0));
-                        __syncwarp();
-                        if (++st == AST) { st = 0; ph ^= 1u; }
-                    }
-                }
-            } else if constexpr (WOP) {
-                forward_w();
-            }
+            // ------------------------------------------------------------ "weight rows landed" -> leader
+            // (packed activation codes with the weight operand by TMA only: TMA copies into operand stages
+            // otherwise count their bytes on the leader's barrier themselves, and widening warps arrive there)
+            if constexpr (WOP && kPackedA) forward_w();
         }
     } else if (warp < kFatFirstEpilogueWarp) {
         regs_give<kFatRegsWiden>();
         if constexpr (WOP && !kPackedA) {
-            // the weight operand comes by TMA and the activation codes are bytes: nothing to widen; the
-            // first of these warps forwards "weight rows landed", as warp 2 does for the activation rows
-            if (warp == kFatFirstWWarp) forward_w();
+            // the weight operand comes by TMA and the activation codes are bytes: nothing to widen
         } else {
             // ------------------------------------------------------------ widen weight codes -> shared memory
             const uint32_t grp = (uint32_t)(warp - kFatFirstWWarp) >> 2;
