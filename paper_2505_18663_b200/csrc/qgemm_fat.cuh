@@ -13,8 +13,8 @@
 // warps, one row and 128 columns per thread, with the register file re-divided between the roles
 // (setmaxnreg: the loaders and the widening warps give registers up, the epilogue warps take them).
 // Roles are aligned to groups of four warps, as that instruction requires:
-//   warps 0-3    TMA producer of activation tiles | MMA issuer (leader CTA) | "weight rows landed"
-//                forwarder (one mode only) | TMA producer of weight rows
+//   warps 0-3    TMA producer of activation tiles | MMA issuer (leader CTA) | idle | TMA producer of
+//                weight rows
 //   warps 4-11   widen weight codes into the operand stages (two groups, alternate k-blocks)
 //   warps 12-19  epilogue: warp w reads tensor-memory lanes 32 * (w % 4).., columns 128 * ((w - 12) / 4)..
 // Every wait is bounded, as in qgemm.cuh.
@@ -112,7 +112,7 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             mbar_init(a_empty(s), 1);
         }
         for (int s = 0; s < APS; ++s) { mbar_init(apk_full(s), 1); mbar_init(apk_empty(s), kSsWWarps / kUnpackGroups); }
-        for (int s = 0; s < WST; ++s) { mbar_init(ops_full(s), WOP ? 2 : 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
+        for (int s = 0; s < WST; ++s) { mbar_init(ops_full(s), WOP ? 1 : 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * 8); }
         mbar_init(drain_bar, 1);
         for (int s = 0; s < WPB; ++s) { mbar_init(wp_full(s), 1); mbar_init(wp_empty(s), kSsWWarps / kUnpackGroups); }
@@ -129,19 +129,6 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = misc[0];
 
-    // WOP: "this CTA's weight rows of a stage have landed" -> leader (a TMA copy completes on a barrier of its own CTA)
-    auto forward_w = [&]() {
-        uint32_t st = 0, ph = 0;
-        bool ok = true;
-        for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-            for (int kb = 0; kb < KB; ++kb) {
-                if (!mbar_wait_warp(wp_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(st), 0));
-                __syncwarp();
-                if (++st == WST) { st = 0; ph ^= 1u; }
-            }
-        }
-    };
     if (warp < kFatFirstWWarp) {
         regs_give<kFatRegsLoader>();
         if (warp == 0) {
@@ -202,14 +189,13 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                     const int n0 = (tile % num_n) * BN + (int)rank * BNh;
                     for (int kb = 0; ok && kb < KB; ++kb) {
-                        if (kOneRing) {  // as the activation rows: bytes counted on the leader's "full" barrier
-                            if (!mbar_wait(a_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-                            if (rank == 0) mbar_arrive_expect_tx(a_ready(wst), 2 * S::kW);
-                            tma_load_2d_pair(sbase + S::kWOff + wst * S::kW, &tmW, map_to_cta(a_ready(wst), 0), kb * kBK, n0);
-                        } else if (WOP) {  // straight into the operand stage, which the MMA's commit frees
-                            if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-                            mbar_arrive_expect_tx(wp_full(wst), S::kW);
-                            tma_load_2d(sbase + S::kWOff + wst * S::kW, &tmW, wp_full(wst), kb * kBK, n0);
+                        if (WOP) {
+                            // straight into the operand stage, which the MMA's commit frees; both CTAs' copies
+                            // count their bytes on the leader's "full" barrier of the stage
+                            const uint32_t full = kOneRing ? a_ready(wst) : ops_full(wst);
+                            if (!mbar_wait(kOneRing ? a_empty(wst) : ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                            if (rank == 0) mbar_arrive_expect_tx(full, 2 * S::kW);
+                            tma_load_2d_pair(sbase + S::kWOff + wst * S::kW, &tmW, map_to_cta(full, 0), kb * kBK, n0);
                         } else {
                             if (!mbar_wait(wp_empty(wst), wph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
                             mbar_arrive_expect_tx(wp_full(wst), S::kWPacked);
@@ -219,7 +205,7 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         if (++wst == WPB) { wst = 0; wph ^= 1u; }
                     }
                 }
-                if (!ok && kOneRing) {
+                if (!ok && WOP) {
                     for (int it = 0; it < 64; ++it) __nanosleep(1000);
                 } else if (!ok) {
                     const uint32_t w_out = wissued < (uint32_t)WPB ? wissued : (uint32_t)WPB;
@@ -289,10 +275,8 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
             __syncwarp();
         } else {
-            // ------------------------------------------------------------ "weight rows landed" -> leader
-            // (packed activation codes with the weight operand by TMA only: TMA copies into operand stages
-            // otherwise count their bytes on the leader's barrier themselves, and widening warps arrive there)
-            if constexpr (WOP && kPackedA) forward_w();
+            // idle: TMA copies into operand stages count their bytes on the leader's barrier themselves,
+            // and widening warps arrive there
         }
     } else if (warp < kFatFirstEpilogueWarp) {
         regs_give<kFatRegsWiden>();

@@ -20,10 +20,10 @@
 //   warps 2-5   epilogue (tcgen05.ld, zero-point term, scales, bias, GELU, bf16, TMA stores), one
 //               warp per tensor-memory lane quarter.
 //   warps 6-13  widen weight codes into the operand stage (two groups, alternate k-blocks).
-//   warp 14     idle but for one case (below): the TMA copies of activation rows of BOTH CTAs of a
-//               pair count their bytes on the leader's barrier of the stage (cp.async.bulk.tensor with
-//               .cta_group::2), which the leader's producer arms for both, so nobody has to tell the
-//               leader that the peer's rows have landed (+2-3 % over a forwarding warp).
+//   warp 14     idle: the TMA copies into operand stages of BOTH CTAs of a pair count their bytes on
+//               the leader's barrier of the stage (cp.async.bulk.tensor with .cta_group::2), which
+//               the leader's producer arms for both, so nobody has to tell the leader that the
+//               peer's rows have landed (+1-3 % over a forwarding warp).
 //   warps 16-19 (codes in bytes, EW = 8 only) a second epilogue warp per lane quarter; each then
 //               takes 128 of the 256 columns.  With one warp per quarter the epilogue, not the MMA,
 //               sets the pace of layers with a short K or a GELU (+13..25 % there); where the
@@ -31,9 +31,8 @@
 //   warps 16-23 (packed codes, EW = 4) widen activation codes into the operand stage (two groups);
 //               with EW = 8 the weight warps 6-13 widen both operands of their k-block instead.
 // WOP (the weight handle carries the codes one int8 each, dvdq_widen_weights): warp 15's TMA copies
-// go straight into a ring of six weight operand stages and no warp widens weights; with codes in
-// bytes they are counted on the leader's barrier like the activation rows, with packed codes on a
-// barrier of their own CTA, and warp 14 tells the leader.
+// go straight into a ring of six weight operand stages, counted on the leader's barrier, and no
+// warp widens weights.
 // With codes in bytes no warp touches an operand at all then, and one "full" / "empty" barrier per
 // stage serves both operands' rings (half the waits and commits of the MMA warp); with packed codes
 // and EW = 8 warps 6-13 widen the activation codes only.
@@ -164,7 +163,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             mbar_init(a_empty(s), 1);
         }
         for (int s = 0; s < APS; ++s) { mbar_init(apk_full(s), 1); mbar_init(apk_empty(s), kSsAWarps / kUnpackGroups); }
-        for (int s = 0; s < WST; ++s) { mbar_init(ops_full(s), WOP ? 2 : 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
+        for (int s = 0; s < WST; ++s) { mbar_init(ops_full(s), WOP ? 1 : 2 * (kSsWWarps / kUnpackGroups)); mbar_init(ops_empty(s), 1); }
         for (int s = 0; s < 2; ++s) { mbar_init(acc_full(s), 1); mbar_init(acc_empty(s), 2 * EW); }
         mbar_init(drain_bar, 1);
         for (int s = 0; s < WPB; ++s) { mbar_init(wp_full(s), 1); mbar_init(wp_empty(s), kSsWWarps / kUnpackGroups); }
@@ -241,17 +240,13 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 const int n0 = (tile % num_n) * BN + (int)rank * BNh;
                 for (int kb = 0; ok && kb < KB; ++kb) {
-                    if (kOneRing) {
-                        // straight into the operand stage, counted on the leader's "full" barrier like the activation rows
-                        if (!mbar_wait(a_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-                        if (rank == 0) mbar_arrive_expect_tx(a_ready(wst), 2 * S::kW);
-                        tma_load_2d_pair(sbase + S::kWOff + wst * S::kW, &tmW, map_to_cta(a_ready(wst), 0), kb * kBK, n0);
-                    } else if (WOP) {
-                        // (packed activation codes) into the operand stage on a barrier of this CTA; warp 14
-                        // tells the leader: the pair form measured 0.5-1 % slower here
-                        if (!mbar_wait(ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
-                        mbar_arrive_expect_tx(wp_full(wst), S::kW);
-                        tma_load_2d(sbase + S::kWOff + wst * S::kW, &tmW, wp_full(wst), kb * kBK, n0);
+                    if (WOP) {
+                        // straight into the operand stage, which the MMA's commit frees; both CTAs' copies
+                        // count their bytes on the leader's "full" barrier of the stage, like the activation rows
+                        const uint32_t full = kOneRing ? a_ready(wst) : ops_full(wst);
+                        if (!mbar_wait(kOneRing ? a_empty(wst) : ops_empty(wst), wph ^ 1u, abort_flag, kWaitWideEmpty)) { ok = false; break; }
+                        if (rank == 0) mbar_arrive_expect_tx(full, 2 * S::kW);
+                        tma_load_2d_pair(sbase + S::kWOff + wst * S::kW, &tmW, map_to_cta(full, 0), kb * kBK, n0);
                     } else {
                         if (!mbar_wait(wp_empty(wst), wph ^ 1u, abort_flag, kWaitPackedEmpty)) { ok = false; break; }
                         mbar_arrive_expect_tx(wp_full(wst), S::kWPacked);
@@ -261,7 +256,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (++wst == WPB) { wst = 0; wph ^= 1u; }
                 }
             }
-            if (!ok && kOneRing) {
+            if (!ok && WOP) {
                 for (int it = 0; it < 64; ++it) __nanosleep(1000);
             } else if (!ok) {
                 const uint32_t w_out = wissued < (uint32_t)WPB ? wissued : (uint32_t)WPB;
@@ -546,21 +541,6 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 __syncwarp();
                 if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(wst), 0));
             }
-            }
-        }
-    } else if (warp == kSsFwdWarp) {
-        // ------------------------------------------------------------ "weight rows landed" -> leader
-        // (packed activation codes with the weight operand by TMA only)
-        if constexpr (WOP && kPackedA) {
-            uint32_t st = 0, ph = 0;
-            bool ok = true;
-            for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
-                for (int kb = 0; kb < KB; ++kb) {
-                    if (!mbar_wait_warp(wp_full(st), ph, abort_flag, kWaitPackedFull)) { ok = false; break; }
-                    if (lane == 0) mbar_arrive_cluster(map_to_cta(ops_full(st), 0));
-                    __syncwarp();
-                    if (++st == WST) { st = 0; ph ^= 1u; }
-                }
             }
         }
     } else if (kPackedA && EW == 4 && warp >= kSsFirstAWarp) {
