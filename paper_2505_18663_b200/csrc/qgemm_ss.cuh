@@ -32,7 +32,7 @@
 //               with EW = 8 the weight warps 6-13 widen both operands of their k-block instead.
 // WOP (the weight handle carries the codes one int8 each, dvdq_widen_weights): warp 15's TMA copies
 // go straight into a ring of six weight operand stages, counted on the leader's barrier, and no
-// warp widens weights.
+// warp widens weights; next to packed activation codes warps 6-9 then widen those, as a third group.
 // With codes in bytes no warp touches an operand at all then, and one "full" / "empty" barrier per
 // stage serves both operands' rings (half the waits and commits of the MMA warp); with packed codes
 // and EW = 8 warps 6-13 widen the activation codes only.
@@ -441,9 +441,10 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         if (!RAW && lane == 0) tma_store_wait_all();
         __syncwarp();
 
-    } else if (WOP && !kWidenBoth && warp < kSsFwdWarp) {
-        // the weight operand comes by TMA: these warps have no work
-    } else if (warp < kSsFwdWarp) {
+    } else if (WOP && !kWidenBoth && warp < kSsFwdWarp && !(kPackedA && warp < kSsFirstWWarp + 4)) {
+        // the weight operand comes by TMA: these warps have no work (but for the first four next to
+        // packed activation codes, which join the activation warps below)
+    } else if (!(WOP && !kWidenBoth) && warp < kSsFwdWarp) {
         // ------------------------------------------------------------ widen weight codes -> shared memory
         const uint32_t grp = (uint32_t)(warp - kSsFirstWWarp) >> 2;
         const int u = (threadIdx.x - kSsFirstWWarp * 32) & 127;  // thread of its group of four warps
@@ -543,20 +544,23 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             }
             }
         }
-    } else if (kPackedA && EW == 4 && warp >= kSsFirstAWarp) {
+    } else if (kPackedA && EW == 4 && (warp >= kSsFirstAWarp || (WOP && warp >= kSsFirstWWarp && warp < kSsFirstWWarp + 4))) {
         // ------------------------------------------------------------ widen activation codes -> shared memory
         // The same job as the weight warps': this CTA's 128 token rows x 128 codes of a k-block, 16 bytes
         // of packed low bits (and 8 bytes of high bits) per piece, into the K-major 128-byte-swizzled stage.
         if constexpr (kPackedA && EW == 4) {
-            const uint32_t grp = (uint32_t)(warp - kSsFirstAWarp) >> 2;
-            const int u = (threadIdx.x - kSsFirstAWarp * 32) & 127;
+            // with the weight operand by TMA four of the idle weight warps are a third group: +3 % with 6-bit
+            // codes, whose widening is the longest chain (next to weight warps at work a third group cost 3 %)
+            constexpr uint32_t kAGroups = WOP ? 3 : 2;
+            const uint32_t grp = warp >= kSsFirstAWarp ? (uint32_t)(warp - kSsFirstAWarp) >> 2 : 2u;
+            const int u = warp >= kSsFirstAWarp ? (threadIdx.x - kSsFirstAWarp * 32) & 127 : (threadIdx.x - kSsFirstWWarp * 32) & 127;
             uint32_t j = 0;
             bool ok = true;
             const uint32_t rt_zero = runtime_zero();
             for (int tile = pair; ok && tile < num_tiles; tile += num_pairs) {
                 for (int kb = 0; kb < KB; ++kb) {
                     const uint32_t jj = j++;
-                    if (jj % kUnpackGroups != grp) continue;
+                    if (jj % kAGroups != grp) continue;
                     const uint32_t pst = jj % APS, pph = (jj / APS) & 1u;
                     const uint32_t wst = jj % AST, wph = (jj / AST) & 1u;
                     if (!mbar_wait(apk_full(pst), pph, abort_flag, kWaitPackedFull)) { ok = false; break; }
