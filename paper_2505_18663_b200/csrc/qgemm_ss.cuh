@@ -351,14 +351,32 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 }
             }
             __syncwarp();
-            if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) break;
-            tc_fence_after();
-            const int row = m0 + q * 32 + lane;
-            const bool row_ok = row < M;
-            const float s_i = (!RAW && row_ok) ? scales[row] : 0.f;
-            int32_t S_i = row_ok ? sums[(int64_t)row * spr] : 0;
-            if (RAW && row_ok)
-                for (int g = 1; g < spr; ++g) S_i += sums[(int64_t)row * spr + g];  // spr == 1 unless the scales are block-wise
+            int row;
+            bool row_ok;
+            float s_i;
+            int32_t S_i;
+            // With eight epilogue warps the epilogue sets the pace, and a global-memory latency after the
+            // wait for the accumulator would be on every tile's critical path: the row's scale and code
+            // sum are loaded before it (+1.5-3.5 % on K = 1536).  With four, the mainloop sets the pace.
+            if constexpr (EW == 8) {
+                row = m0 + q * 32 + lane;
+                row_ok = row < M;
+                s_i = (!RAW && row_ok) ? scales[row] : 0.f;
+                S_i = row_ok ? sums[(int64_t)row * spr] : 0;
+                if (RAW && row_ok)
+                    for (int g = 1; g < spr; ++g) S_i += sums[(int64_t)row * spr + g];  // spr == 1 unless the scales are block-wise
+                if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) break;
+                tc_fence_after();
+            } else {
+                if (!mbar_wait(acc_full(a), aph, abort_flag, kWaitAccFull)) break;
+                tc_fence_after();
+                row = m0 + q * 32 + lane;
+                row_ok = row < M;
+                s_i = (!RAW && row_ok) ? scales[row] : 0.f;
+                S_i = row_ok ? sums[(int64_t)row * spr] : 0;
+                if (RAW && row_ok)
+                    for (int g = 1; g < spr; ++g) S_i += sums[(int64_t)row * spr + g];
+            }
             const float S_f = (float)S_i;  // |sum of codes| <= K * 32 < 2^24: exact
             const float s_k = s_i * (1.0f / (float)(1 << kShift)), nS_k = -S_f * (float)(1 << kShift);
             const uint64_t s2 = f2_pack(s_k, s_k), negS2 = f2_pack(nS_k, nS_k);
