@@ -89,7 +89,7 @@ qgemm_fat_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int KBG = KB / NG;  // k-blocks per group: 1, 2 or 8
 
     const uint32_t bar0 = sbase + S::kBarOff;
-    auto a_full = [&](int s) { return bar0 + 8u * s; };
+    auto a_full = [&](int s) { return bar0 + 8u * s; };  // a slot kept for the layout's sake: copies count on a_ready
     auto a_ready = [&](int s) { return bar0 + 8u * (AST + s); };
     auto a_empty = [&](int s) { return bar0 + 8u * (2 * AST + s); };
     const uint32_t barw = bar0 + 8u * (3 * AST);

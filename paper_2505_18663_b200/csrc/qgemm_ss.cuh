@@ -138,7 +138,7 @@ qgemm_ss_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int KB = 2 * ((K + 2 * kBK - 1) / (2 * kBK));  // even; a k-block past K reads zeros
 
     const uint32_t bar0 = sbase + S::kBarOff;
-    auto a_full = [&](int s) { return bar0 + 8u * s; };                          // this CTA's TMA copy of the stage
+    auto a_full = [&](int s) { return bar0 + 8u * s; };                          // a slot kept for the layout's sake: copies count on a_ready
     auto a_ready = [&](int s) { return bar0 + 8u * (AST + s); };                 // leader's copy: both CTAs' rows of the stage are in place
     auto a_empty = [&](int s) { return bar0 + 8u * (2 * AST + s); };             // one per CTA
     const uint32_t barw = bar0 + 8u * (3 * AST);
